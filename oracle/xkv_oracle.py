@@ -1,0 +1,337 @@
+"""CPU oracle for xKV cross-layer factorisation and the Selective Reconstruction decode step.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain statement of what the
+CUDA library must compute.  It shares no code with the CUDA path and imports
+nothing from the product package; only tests, the smoke check and the
+benchmark's CPU-baseline leg may call it.
+
+Conventions
+-----------
+* Every tensor that the library receives in bf16 is handed to the oracle as the
+  same bf16 values widened to float32/float64 (no extra rounding happens here
+  except where a function says it produces a bf16 tensor).
+* Floating point is fp64 everywhere except `landmark_scores`, whose fp32
+  sequential accumulation is part of the contract: the scores decide an integer
+  result (the selected indices), so both sides must take that decision in the
+  same precision and the same order.
+* Symbols follow the paper: L (here T) context rows, W (here G) layers per
+  window, H_q / H_kv heads, d_h head width, d = H_kv*d_h, c chunk size,
+  k token budget, k_ch = ceil(k/c), n_c = ceil(T/c), rho(h) = h // n_rep.
+
+Parity pins (tests/test_oracle_*.py): every function below is pinned by closed
+forms, invariants, brute force on tiny inputs, a library routine it must reduce
+to, or numbers the paper prints; none is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+# --------------------------------------------------------------------------
+# bf16 helper (the oracle's own; round-to-nearest-even on the fp32 bit pattern)
+# --------------------------------------------------------------------------
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); returns float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    lsb = (u >> np.uint64(16)) & np.uint64(1)
+    u = (u + np.uint64(0x7FFF) + lsb) & np.uint64(0xFFFF0000)
+    return u.astype(np.uint32).view(np.float32).reshape(x.shape)
+
+
+# --------------------------------------------------------------------------
+# O1  Cross-Layer Factorization  (Sec. 3.1, Eq. 1)
+# --------------------------------------------------------------------------
+
+
+def clf_factorize(X_layers, r: int):
+    """Rank-r factorisation of the column-wise concatenation of a window's caches.
+
+    X_layers: list of W arrays (T x d), the pre-RoPE key cache or the value cache
+    of the W adjacent layers of one window (Eq. 1).  Returns (A, [B_l], sigma):
+    A = U_r Sigma_r (T x r) is the shared token basis, B_l (r x d) is the l-th
+    column block of V_r^T, sigma are all singular values of the concatenation.
+    No centring is applied (Eq. 1 has none).  This is the exact optimum the
+    paper approximates with a randomised SVD.
+    """
+    X_cat = np.concatenate([np.asarray(x, dtype=np.float64) for x in X_layers], axis=1)
+    U, s, Vt = np.linalg.svd(X_cat, full_matrices=False)
+    if not (1 <= r <= s.shape[0]):
+        raise ValueError("rank out of range")
+    A = U[:, :r] * s[:r][None, :]
+    d = X_layers[0].shape[1]
+    B = [Vt[:r, i * d:(i + 1) * d].copy() for i in range(len(X_layers))]
+    return A, B, s
+
+
+# --------------------------------------------------------------------------
+# RoPE (rotate-half convention).  The paper factorises pre-RoPE keys while
+# landmarks and queries are post-RoPE, so reconstructed key rows must be
+# rotated at their token position before they meet the query.
+# --------------------------------------------------------------------------
+
+
+def rope_rotate(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
+    """Rotate rows of x (n x d_h) at integer positions pos (n,), fp64.
+
+    theta_i = base^(-2i/d_h) for i < d_h/2, phi = pos*theta_i,
+    y[i] = x[i] cos(phi) - x[i+d_h/2] sin(phi),
+    y[i+d_h/2] = x[i+d_h/2] cos(phi) + x[i] sin(phi).   base <= 0: identity.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    if base <= 0:
+        return x.copy()
+    d_h = x.shape[-1]
+    half = d_h // 2
+    i = np.arange(half, dtype=np.float64)
+    theta = np.power(float(base), -2.0 * i / d_h)
+    phi = np.asarray(pos, dtype=np.float64)[:, None] * theta[None, :]
+    cs, sn = np.cos(phi), np.sin(phi)
+    x1, x2 = x[:, :half], x[:, half:]
+    return np.concatenate([x1 * cs - x2 * sn, x2 * cs + x1 * sn], axis=1)
+
+
+# --------------------------------------------------------------------------
+# O2  Landmark construction  (App. B.1, Algorithm 1, lines 1-3)
+# --------------------------------------------------------------------------
+
+
+def build_landmarks(K_pre: np.ndarray, c: int, rope_base: float) -> np.ndarray:
+    """Chunk means of the post-RoPE keys of one layer, rounded to bf16.
+
+    K_pre: (H_kv, T, d_h) pre-RoPE keys (the original cache, not a reconstruction).
+    Chunk j covers rows [c*j, min(c*j+c, T)); its landmark is the mean over the
+    rows actually present (the 1/|C_j| form, which also covers a ragged tail).
+    Returns (H_kv, n_c, d_h) float32 holding bf16 values.
+    """
+    H_kv, T, d_h = K_pre.shape
+    n_c = -(-T // c)
+    out = np.zeros((H_kv, n_c, d_h), dtype=np.float64)
+    pos = np.arange(T)
+    for g in range(H_kv):
+        Kr = rope_rotate(K_pre[g], pos, rope_base)
+        for j in range(n_c):
+            rows = Kr[c * j:min(c * j + c, T)]
+            out[g, j] = rows.sum(axis=0) / rows.shape[0]
+    return bf16_round(out.astype(np.float32))
+
+
+# --------------------------------------------------------------------------
+# O3  Landmark-guided top-k chunk selection  (App. B.1, Algorithm 2)
+# --------------------------------------------------------------------------
+
+
+def landmark_scores(q_heads: np.ndarray, L_g: np.ndarray) -> np.ndarray:
+    """Algorithm 2 line 2 for the query heads mapped to one KV head.
+
+    q_heads (n_rep x d_h) and L_g (n_c x d_h) hold bf16 values.  Canonical
+    arithmetic: acc = +0; for i = 0..d_h-1 in order acc = acc + q[i]*L[j][i]
+    in fp32 (each product of two bf16 values is exact in fp32, so only the
+    order matters); P = acc * s with s = 1/sqrt(d_h) computed in fp32.
+    """
+    q = np.asarray(q_heads, dtype=np.float32)
+    L = np.asarray(L_g, dtype=np.float32)
+    n_rep, d_h = q.shape
+    s = np.float32(1.0) / np.sqrt(np.float32(d_h))
+    P = np.empty((n_rep, L.shape[0]), dtype=np.float32)
+    for h in range(n_rep):
+        acc = np.zeros(L.shape[0], dtype=np.float32)
+        for i in range(d_h):
+            acc = acc + q[h, i] * L[:, i]
+        P[h] = acc * s
+    return P
+
+
+def pool_scores(P: np.ndarray) -> np.ndarray:
+    """Algorithm 2 line 3: max over the query heads of one KV head."""
+    return P.max(axis=0)
+
+
+def topk_chunks(S: np.ndarray, k_ch: int) -> np.ndarray:
+    """Algorithm 2 line 4 with a fixed tie rule.
+
+    Total order: score descending, then chunk index ascending (-0 equals +0).
+    Returns the first k_ch chunk ids of that order, sorted ascending.
+    """
+    order = np.argsort(-(S.astype(np.float32) + np.float32(0.0)), kind="stable")
+    return np.sort(order[:k_ch]).astype(np.int64)
+
+
+def expand_chunks(chunks: np.ndarray, c: int, T: int) -> np.ndarray:
+    """Chunk ids -> token rows c*j .. min(c*j+c, T)-1, ascending."""
+    rows = []
+    for j in chunks:
+        rows.extend(range(int(j) * c, min(int(j) * c + c, T)))
+    return np.asarray(rows, dtype=np.int32)
+
+
+def sr_select(q_heads: np.ndarray, L_g: np.ndarray, k: int, c: int, T: int) -> np.ndarray:
+    """Selected token rows for one (layer, sequence, KV head): Algorithm 2 without outliers."""
+    n_c = L_g.shape[0]
+    k_ch = min(-(-k // c), n_c)
+    S = pool_scores(landmark_scores(q_heads, L_g))
+    return expand_chunks(topk_chunks(S, k_ch), c, T)
+
+
+# --------------------------------------------------------------------------
+# O4  Selective reconstruction  (Sec. 3.2, Eq. 3)
+# --------------------------------------------------------------------------
+
+
+def sr_reconstruct(A: np.ndarray, B_head: np.ndarray, rows: np.ndarray) -> np.ndarray:
+    """X_hat[S,:] = A[S,:] @ B_{l,g}   (A: T x r, B_head: r x d_h), fp64."""
+    return np.asarray(A, dtype=np.float64)[np.asarray(rows, dtype=np.int64)] @ np.asarray(B_head, dtype=np.float64)
+
+
+def sr_reconstruct_keys(A_k, B_k_head, rows, rope_base: float) -> np.ndarray:
+    """Reconstructed key rows rotated at their token positions (position = row index)."""
+    return rope_rotate(sr_reconstruct(A_k, B_k_head, rows), np.asarray(rows), rope_base)
+
+
+# --------------------------------------------------------------------------
+# O5  Attention over the reconstructed rows
+# --------------------------------------------------------------------------
+
+
+def attend(q_heads: np.ndarray, K_hat: np.ndarray, V_hat: np.ndarray, scale: float):
+    """softmax(q K_hat^T * scale) V_hat per query head; returns (o, lse) in fp64.
+
+    An empty row set gives o = 0 and lse = -inf.
+    """
+    q = np.asarray(q_heads, dtype=np.float64)
+    n_rep = q.shape[0]
+    d_v = V_hat.shape[1] if V_hat.ndim == 2 else 0
+    if K_hat.shape[0] == 0:
+        return np.zeros((n_rep, d_v)), np.full((n_rep,), -np.inf)
+    z = (q @ np.asarray(K_hat, dtype=np.float64).T) * float(scale)
+    m = z.max(axis=1, keepdims=True)
+    w = np.exp(z - m)
+    l = w.sum(axis=1, keepdims=True)
+    o = (w @ np.asarray(V_hat, dtype=np.float64)) / l
+    lse = (m + np.log(l))[:, 0]
+    return o, lse
+
+
+def dense_attend(q_heads, K_all, V_all, scale: float):
+    """Plain softmax attention over every row, written separately from `attend`
+    (row by row, no max subtraction shared with it) so that the two can pin each other."""
+    q = np.asarray(q_heads, dtype=np.float64)
+    K = np.asarray(K_all, dtype=np.float64)
+    V = np.asarray(V_all, dtype=np.float64)
+    out = np.zeros((q.shape[0], V.shape[1]))
+    for h in range(q.shape[0]):
+        z = np.array([float(np.dot(q[h], K[j])) * float(scale) for j in range(K.shape[0])])
+        e = np.exp(z - z.max())
+        out[h] = (e[:, None] * V).sum(axis=0) / e.sum()
+    return out
+
+
+def merge_partials(parts):
+    """Merge attention results over disjoint row sets by log-sum-exp.
+
+    parts: list of (o, lse) as returned by `attend`.  Equals `attend` on the union.
+    """
+    lses = np.stack([p[1] for p in parts])            # (n_parts, n_rep)
+    m = lses.max(axis=0)
+    w = np.exp(lses - m[None, :])                     # weight of each part
+    o = sum(w[i][:, None] * parts[i][0] for i in range(len(parts))) / w.sum(axis=0)[:, None]
+    return o, m + np.log(w.sum(axis=0))
+
+
+# --------------------------------------------------------------------------
+# The decode step of one window: select -> reconstruct -> RoPE -> attend
+# --------------------------------------------------------------------------
+
+
+def sr_decode_problem(q_heads, L_g, A_k, A_v, B_k_head, B_v_head, k, c, T, rope_base, scale,
+                      rows=None):
+    """One (layer, sequence, KV head) problem.  rows=None: use Algorithm 2."""
+    if rows is None:
+        rows = sr_select(q_heads, L_g, k, c, T)
+    K_hat = sr_reconstruct_keys(A_k, B_k_head, rows, rope_base)
+    V_hat = sr_reconstruct(A_v, B_v_head, rows)
+    o, lse = attend(q_heads, K_hat, V_hat, scale)
+    return rows, o, lse
+
+
+def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scale=None,
+                   sel_idx=None, sel_cnt=None, problems=None):
+    """Whole-window decode step in the library's tensor layouts.
+
+    A_k (B,T,r_k)  A_v (B,T,r_v)  B_k (B,G,r_k,d)  B_v (B,G,r_v,d)
+    landmarks (B,G,H_kv,n_c,d_h)  q (G,B,H_q,d_h)
+    Returns sel_idx (G,B,H_kv,k_cap) int32 padded with -1, sel_cnt (G,B,H_kv),
+    out (G,B,H_q,d_h) fp64, lse (G,B,H_q) fp64.
+    If sel_idx/sel_cnt are given the selection is taken from them (any order,
+    duplicates allowed) and Algorithm 2 is skipped.  `problems` restricts the
+    work to a list of (l, b, g) triples (the rest of the outputs stay zero).
+    """
+    Bsz, T, _ = A_k.shape
+    G = B_k.shape[1]
+    H_q, d_h = q.shape[2], q.shape[3]
+    n_rep = H_q // H_kv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d_h)
+    k_cap = (-(-k // c)) * c if sel_idx is None else sel_idx.shape[-1]
+    o_idx = np.full((G, Bsz, H_kv, k_cap), -1, dtype=np.int32)
+    o_cnt = np.zeros((G, Bsz, H_kv), dtype=np.int32)
+    out = np.zeros((G, Bsz, H_q, d_h))
+    lse = np.zeros((G, Bsz, H_q))
+    if problems is None:
+        problems = [(l, b, g) for l in range(G) for b in range(Bsz) for g in range(H_kv)]
+    for (l, b, g) in problems:
+        qh = q[l, b, g * n_rep:(g + 1) * n_rep]
+        rows = None
+        if sel_idx is not None:
+            rows = np.asarray(sel_idx[l, b, g, :int(sel_cnt[l, b, g])], dtype=np.int32)
+        rows, o, ls = sr_decode_problem(
+            qh, None if landmarks is None else landmarks[b, l, g], A_k[b], A_v[b],
+            B_k[b, l][:, g * d_h:(g + 1) * d_h], B_v[b, l][:, g * d_h:(g + 1) * d_h],
+            k, c, T, rope_base, scale, rows)
+        o_idx[l, b, g, :len(rows)] = rows
+        o_cnt[l, b, g] = len(rows)
+        out[l, b, g * n_rep:(g + 1) * n_rep] = o
+        lse[l, b, g * n_rep:(g + 1) * n_rep] = ls
+    return o_idx, o_cnt, out, lse
+
+
+# --------------------------------------------------------------------------
+# Cost and memory accounting  (App. C, "FLOPs & Memory Cost")
+# --------------------------------------------------------------------------
+
+
+def flops_dense(L: int, r_k: int, r_v: int, d: int) -> int:
+    """Dense reconstruction cost of one layer (multiply-add counted once, as the paper does)."""
+    return L * r_k * d + L * r_v * d
+
+
+def flops_sr(M_per_head, d_h: int, r_k: int, r_v: int) -> int:
+    """Selective reconstruction cost of one layer: sum_g M_g * d_h * (r_K + r_V)."""
+    return sum(int(M) * d_h * (r_k + r_v) for M in M_per_head)
+
+
+def factor_scalars(N: int, W: int, L: int, r_k: int, r_v: int, d: int) -> int:
+    """Stored scalars of the CLF factors: one basis per window, one B per layer."""
+    Gw = -(-N // W)
+    return (Gw * L * r_k + N * r_k * d) + (Gw * L * r_v + N * r_v * d)
+
+
+def landmark_scalars(N: int, L: int, c: int, d: int) -> int:
+    return N * (-(-L // c)) * d
+
+
+def compression_ratios(N: int, W: int, L: int, d: int, r_k: int, r_v: int, c: int) -> dict:
+    """Compression ratios relative to the full cache of 2*N*L*d scalars."""
+    Gw = -(-N // W)
+    C_K = N * L * d / (Gw * L * r_k + N * r_k * d)
+    C_V = N * L * d / (Gw * L * r_v + N * r_v * d) if r_v else float("inf")
+    alpha = (-(-L // c)) / L
+    return {
+        "xkv": 2.0 / (1.0 / C_K + 1.0 / C_V),
+        "xkv_sr": 2.0 / (1.0 / C_K + 1.0 / C_V + alpha),
+        "xk_sr_gpu": 2.0 / (1.0 / C_K + alpha),
+        "xk_sr_total": 2.0 / (1.0 / C_K + alpha + 1.0),
+    }
