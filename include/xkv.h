@@ -1,0 +1,167 @@
+/*
+ * xkv.h -- C ABI of the xKV selective-reconstruction (SR) decode library for NVIDIA B200 (sm_100a).
+ *
+ * One handle describes one window of G adjacent transformer layers whose pre-RoPE key cache and
+ * value cache were factorised across layers (paper Sec. 3.1, Eq. 1):
+ *     [X_l0 ... X_l0+G-1] ~= A [B_l0 ... B_l0+G-1],   A = U Sigma (T x r),  B_l (r x d),  d = H_kv*d_h
+ * once for keys (A_k, B_k, rank r_k) and once for values (A_v, B_v, rank r_v).
+ *
+ * A decode step for the layers of the window is two calls:
+ *   xkv_sr_select              landmark-guided top-k chunk selection (App. B.1, Algorithm 2)
+ *   xkv_sr_reconstruct_attend  X_hat[S,:] = A[S,:] B_{l,g} for keys and values (Sec. 3.2, Eq. 3),
+ *                              rotary embedding of the rebuilt key rows, softmax attention over them.
+ *
+ * General rules
+ *   - Every function returns an xkv_status; nothing throws, aborts or traps the GPU.
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The config struct,
+ *     the handle and the out-parameters of create/status/bytes are host memory.
+ *   - All work is enqueued on the CUDA stream passed in (a cudaStream_t cast to void*; NULL is the
+ *     legacy default stream).  No call synchronises the device except create and destroy.
+ *   - The handle BORROWS A_k, A_v, landmarks (the caller keeps them alive and unchanged while the
+ *     handle is used) and copies B_k, B_v into a repacked buffer that it owns, together with its
+ *     scratch (pooled scores, attention partials, rotary tables).  Calls on one handle must not
+ *     overlap on the GPU: they share that scratch.
+ *   - Conditions detected on the device (an index outside [0,T), a bounded wait that ran out) do not
+ *     fault: the offending row is skipped or the tile abandoned, a bit is set in a device word, and
+ *     xkv_group_status reports it after the caller has synchronised.
+ *   - Index arithmetic is 64-bit; T < 2^24, d_h in {64,128}, r_k and r_v multiples of 8,
+ *     H_q a multiple of H_kv with H_q/H_kv <= 16.
+ */
+#ifndef XKV_H_
+#define XKV_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define XKV_API __attribute__((visibility("default")))
+#else
+#define XKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xkv_group xkv_group; /* opaque */
+
+typedef enum {
+  XKV_OK = 0,
+  XKV_ERR_INVALID_ARG = -1, /* NULL pointer, bad struct_size, sizes that break a rule above */
+  XKV_ERR_UNSUPPORTED = -2, /* a legal but unimplemented combination */
+  XKV_ERR_ARCH = -3,        /* current device is not compute capability 10.x */
+  XKV_ERR_CUDA = -4,        /* a CUDA runtime call failed; see xkv_last_cuda_error */
+  XKV_ERR_OOM = -5,         /* device allocation for the handle failed */
+  XKV_ERR_INDEX_RANGE = -6, /* device flag: a selected row was outside [0,T) and was skipped */
+  XKV_ERR_TIMEOUT = -7      /* device flag: a bounded wait inside a kernel ran out */
+} xkv_status;
+
+/* Bits of the device flag word returned by xkv_group_status. */
+#define XKV_FLAG_INDEX_RANGE 1u
+#define XKV_FLAG_TIMEOUT 2u
+
+/*
+ * Problem statement for one window (names follow the paper; T is its L, G its W).
+ * Layouts are row-major with the last index fastest; bf16 means the upper 16 bits of an IEEE fp32.
+ */
+typedef struct {
+  uint32_t struct_size; /* sizeof(xkv_group_config); checked for ABI agreement */
+  int32_t G;            /* layers in the window (paper W), >= 1 */
+  int32_t batch;        /* sequences; each has its own factors (the SVD is computed per prompt) */
+  int32_t T;            /* context rows (paper L), 1 <= T < 2^24 */
+  int32_t H_kv, H_q;    /* KV heads and query heads; GQA map rho(h) = h / (H_q/H_kv) */
+  int32_t d_h;          /* head width: 64 or 128 */
+  int32_t r_k, r_v;     /* ranks of the key and value factorisation; multiples of 8 */
+  int32_t chunk;        /* landmark chunk size c (0 means 8); n_c = ceil(T/c) */
+  int32_t k_max;        /* largest token budget k that xkv_sr_select will be given */
+  float rope_base;      /* > 0: rotate rebuilt key rows (rotate-half, theta_i = base^(-2i/d_h),
+                           position = token row); <= 0: keys are used as reconstructed */
+  float softmax_scale;  /* logit scale of the attention; 0 means 1/sqrt(d_h) */
+  const void* A_k;      /* bf16 [batch][T][r_k]   shared token basis of the keys    (borrowed) */
+  const void* A_v;      /* bf16 [batch][T][r_v]   shared token basis of the values  (borrowed) */
+  const void* B_k;      /* bf16 [batch][G][r_k][H_kv*d_h]  per-layer reconstruction matrices; head g
+                           owns columns g*d_h .. g*d_h+d_h-1 (Eq. 2).  Copied at create. */
+  const void* B_v;      /* bf16 [batch][G][r_v][H_kv*d_h]  same for values.  Copied at create. */
+  const void* landmarks; /* bf16 [batch][G][H_kv][n_c][d_h] chunk means of the post-RoPE keys
+                            (Algorithm 1, lines 1-3); borrowed.  May be NULL if xkv_sr_select is
+                            never called on this handle. */
+} xkv_group_config;
+
+/*
+ * Validate the configuration, allocate the handle's device memory on the current device, repack
+ * B_k/B_v and build the rotary tables (this work is enqueued on `stream` and waited for).
+ * On success *out receives the handle.  Errors: INVALID_ARG, ARCH, OOM, CUDA.
+ */
+XKV_API int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out);
+
+/*
+ * Algorithm 2 (App. B.1) for layers layer_begin <= l < layer_end of the window, every sequence and
+ * every KV head g:
+ *   P[h,j] = (sum_{i=0}^{d_h-1} q[h,i]*L[g,j,i]) * (1/sqrt(d_h))   fp32, i in ascending order
+ *   S[j]   = max over the H_q/H_kv query heads h with rho(h) = g
+ *   take the k_ch = min(ceil(k/c), n_c) chunks first in the order (S descending, j ascending;
+ *   -0 equals +0), sort them ascending, expand chunk j to rows c*j .. min(c*j+c, T)-1.
+ * q        bf16 [G][batch][H_q][d_h], post-RoPE decode queries (rows of layers outside the range are
+ *          not read).
+ * k        token budget, 1 <= k <= k_max.  k_cap = ceil(k/c)*c is the row stride of sel_idx.
+ * sel_idx  out, int32 [G][batch][H_kv][k_cap]; entries at and beyond sel_cnt are set to -1.
+ * sel_cnt  out, int32 [G][batch][H_kv]; number of rows (k_ch*c, less if the ragged last chunk is in).
+ * Scores must be finite; the result for NaN inputs is unspecified (but in range).
+ * Errors: INVALID_ARG (NULL, bad range, k out of range, handle without landmarks), CUDA.
+ */
+XKV_API int xkv_sr_select(xkv_group* grp, int layer_begin, int layer_end, const void* q, int32_t k,
+                  int32_t* sel_idx, int32_t* sel_cnt, void* stream);
+
+/*
+ * Eq. 3 plus attention for layers layer_begin <= l < layer_end, every sequence, every KV head g:
+ *   K_hat[S,:] = rope(A_k[S,:] B_k_{l,g}),  V_hat[S,:] = A_v[S,:] B_v_{l,g},
+ *   out_h = softmax(scale * q_h K_hat^T) V_hat  for the query heads h with rho(h) = g.
+ * sel_idx  int32 [G][batch][H_kv][k_cap], the first sel_cnt entries of each row list the token rows
+ *          S.  They need not be sorted or chunk aligned; a repeated row counts as often as it
+ *          appears.  A row outside [0,T) is skipped and XKV_FLAG_INDEX_RANGE is raised.
+ * sel_cnt  int32 [G][batch][H_kv], 0 <= sel_cnt <= k_cap.  With sel_cnt = 0 the head's output is 0
+ *          and its lse is -inf.
+ * k_cap    row stride of sel_idx, 1 <= k_cap <= ceil(k_max/c)*c (the handle's scratch is sized by k_max).
+ * out      bf16 [G][batch][H_q][d_h].
+ * lse      optional (may be NULL) fp32 [G][batch][H_q]: natural-log sum of exp of the scaled logits,
+ *          for merging with attention over rows kept outside the factorised cache.
+ * Accumulation is fp32 from bf16 operands.  Errors: INVALID_ARG, CUDA.
+ */
+XKV_API int xkv_sr_reconstruct_attend(xkv_group* grp, int layer_begin, int layer_end, const void* q,
+                              const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_cap,
+                              void* out, float* lse, void* stream);
+
+/* Free the handle and the device memory it owns (synchronises the device first). NULL is allowed. */
+XKV_API int xkv_group_destroy(xkv_group* grp);
+
+/*
+ * Read the device flag word (host out-parameter, may be NULL) with a blocking copy on `stream`
+ * and clear it.  Returns XKV_OK, or the status of the most severe flag (TIMEOUT over INDEX_RANGE).
+ */
+XKV_API int xkv_group_status(xkv_group* grp, uint32_t* device_flags, void* stream);
+
+/*
+ * Memory accounting of one window (App. C, "Compressed-cache memory" and "Landmark memory"),
+ * in bytes of bf16 storage: factor_bytes = batch*2*(T*r_k + G*r_k*d + T*r_v + G*r_v*d),
+ * landmark_bytes = batch*2*G*ceil(T/c)*d.  Host-only; needs no device.  Out-pointers may be NULL.
+ */
+XKV_API int xkv_group_bytes(const xkv_group_config* cfg, uint64_t* factor_bytes, uint64_t* landmark_bytes);
+
+/*
+ * Scratch bytes the handle owns on the device (pooled scores, attention partials, rotary tables,
+ * repacked B), host out-parameter.
+ */
+XKV_API int xkv_group_workspace_bytes(const xkv_group* grp, uint64_t* bytes);
+
+/* Static, human-readable name of a status code. Never NULL. */
+XKV_API const char* xkv_strerror(int status);
+
+/* The last CUDA runtime error code seen by this library on the calling thread (0 if none). */
+XKV_API int xkv_last_cuda_error(void);
+
+/* Number of kernels the library has launched since load (all handles); for launch accounting. */
+XKV_API uint64_t xkv_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XKV_H_ */

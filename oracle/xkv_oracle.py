@@ -183,7 +183,8 @@ def sr_select(q_heads: np.ndarray, L_g: np.ndarray, k: int, c: int, T: int) -> n
 
 def sr_reconstruct(A: np.ndarray, B_head: np.ndarray, rows: np.ndarray) -> np.ndarray:
     """X_hat[S,:] = A[S,:] @ B_{l,g}   (A: T x r, B_head: r x d_h), fp64."""
-    return np.asarray(A, dtype=np.float64)[np.asarray(rows, dtype=np.int64)] @ np.asarray(B_head, dtype=np.float64)
+    gathered = np.asarray(A)[np.asarray(rows, dtype=np.int64)].astype(np.float64)
+    return gathered @ np.asarray(B_head, dtype=np.float64)
 
 
 def sr_reconstruct_keys(A_k, B_k_head, rows, rope_base: float) -> np.ndarray:

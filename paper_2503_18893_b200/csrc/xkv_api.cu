@@ -1,0 +1,258 @@
+// C ABI of libxkv: argument checking, handle life cycle, dispatch to the kernels.
+#include <cuda.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <atomic>
+#include <new>
+
+#include "xkv_internal.cuh"
+
+namespace xkv {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<uint64_t> g_launches{0};
+
+void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static int check_config(const xkv_group_config* c, bool need_ptrs) {
+  if (!c) return XKV_ERR_INVALID_ARG;
+  if (c->struct_size != sizeof(xkv_group_config)) return XKV_ERR_INVALID_ARG;
+  if (c->G < 1 || c->batch < 1 || c->T < 1 || c->T >= (1 << 24)) return XKV_ERR_INVALID_ARG;
+  if (c->H_kv < 1 || c->H_q < 1 || c->H_q % c->H_kv != 0) return XKV_ERR_INVALID_ARG;
+  if (c->H_q / c->H_kv > kMaxRep) return XKV_ERR_INVALID_ARG;
+  if (c->d_h != 64 && c->d_h != 128) return XKV_ERR_INVALID_ARG;
+  if (c->r_k < 8 || c->r_v < 8 || c->r_k % 8 || c->r_v % 8) return XKV_ERR_INVALID_ARG;
+  if (c->r_k > 8192 || c->r_v > 8192) return XKV_ERR_INVALID_ARG;
+  if (c->chunk < 0 || c->chunk > 4096) return XKV_ERR_INVALID_ARG;
+  if (c->k_max < 1) return XKV_ERR_INVALID_ARG;
+  if (!(c->softmax_scale >= 0.0f) || isinf(c->softmax_scale)) return XKV_ERR_INVALID_ARG;
+  if (isnan(c->rope_base) || isinf(c->rope_base)) return XKV_ERR_INVALID_ARG;
+  if (need_ptrs) {
+    if (!c->A_k || !c->A_v || !c->B_k || !c->B_v) return XKV_ERR_INVALID_ARG;
+    const uintptr_t m = (uintptr_t)c->A_k | (uintptr_t)c->A_v | (uintptr_t)c->B_k | (uintptr_t)c->B_v |
+                        (uintptr_t)c->landmarks;
+    if (m & 15u) return XKV_ERR_INVALID_ARG;   // 16-byte vector loads and TMA need this
+  }
+  return XKV_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols fastest), box = box_rows x 64 columns, 128-byte swizzle.
+static bool encode_rows64(void* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace xkv
+
+using namespace xkv;
+
+#define XKV_TRY_CUDA(expr)                 \
+  do {                                     \
+    cudaError_t e_ = (expr);               \
+    if (e_ != cudaSuccess) {               \
+      set_cuda_error(e_);                  \
+      (void)cudaGetLastError();            \
+      st = (e_ == cudaErrorMemoryAllocation) ? XKV_ERR_OOM : XKV_ERR_CUDA; \
+      goto fail;                           \
+    }                                      \
+  } while (0)
+
+extern "C" {
+
+const char* xkv_strerror(int s) {
+  switch (s) {
+    case XKV_OK: return "ok";
+    case XKV_ERR_INVALID_ARG: return "invalid argument";
+    case XKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case XKV_ERR_ARCH: return "device is not sm_100 (B200)";
+    case XKV_ERR_CUDA: return "CUDA runtime error";
+    case XKV_ERR_OOM: return "out of device memory";
+    case XKV_ERR_INDEX_RANGE: return "a selected row index was outside [0,T) and was skipped";
+    case XKV_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    default: return "unknown status";
+  }
+}
+
+int xkv_last_cuda_error(void) { return g_last_cuda_error; }
+uint64_t xkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int xkv_group_bytes(const xkv_group_config* cfg, uint64_t* factor_bytes, uint64_t* landmark_bytes) {
+  int st = check_config(cfg, false);
+  if (st != XKV_OK) return st;
+  const uint64_t c = cfg->chunk ? cfg->chunk : 8;
+  const uint64_t d = (uint64_t)cfg->H_kv * cfg->d_h, T = cfg->T, G = cfg->G, B = cfg->batch;
+  if (factor_bytes)
+    *factor_bytes = B * 2 * (T * cfg->r_k + G * cfg->r_k * d + T * cfg->r_v + G * cfg->r_v * d);
+  if (landmark_bytes) *landmark_bytes = B * 2 * G * ((T + c - 1) / c) * d;
+  return XKV_OK;
+}
+
+int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out) {
+  if (!out) return XKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  int st = check_config(cfg, true);
+  if (st != XKV_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  xkv_group* g = new (std::nothrow) xkv_group();
+  if (!g) return XKV_ERR_OOM;
+  memset(g, 0, sizeof(*g));
+  g->cfg = *cfg;
+  if (g->cfg.chunk == 0) g->cfg.chunk = 8;
+  {
+    cudaDeviceProp prop;
+    XKV_TRY_CUDA(cudaGetDevice(&g->device));
+    XKV_TRY_CUDA(cudaGetDeviceProperties(&prop, g->device));
+    if (prop.major != 10) { st = XKV_ERR_ARCH; goto fail; }
+    g->sm_count = prop.multiProcessorCount;
+  }
+  {
+    GroupDev& d = g->dev;
+    const xkv_group_config& c = g->cfg;
+    d.G = c.G; d.batch = c.batch; d.T = c.T; d.H_kv = c.H_kv; d.H_q = c.H_q; d.d_h = c.d_h;
+    d.r_k = c.r_k; d.r_v = c.r_v; d.c = c.chunk; d.n_c = (c.T + c.chunk - 1) / c.chunk;
+    d.n_rep = c.H_q / c.H_kv;
+    d.n_hi = (c.T + kRopeLo - 1) / kRopeLo;
+    d.sel_scale = 1.0f / sqrtf((float)c.d_h);
+    d.att_scale = c.softmax_scale > 0.0f ? c.softmax_scale : 1.0f / sqrtf((float)c.d_h);
+    d.use_rope = c.rope_base > 0.0f;
+    d.A_k = (const __nv_bfloat16*)c.A_k; d.A_v = (const __nv_bfloat16*)c.A_v;
+    d.landmarks = (const __nv_bfloat16*)c.landmarks;
+    g->k_cap_max = (int)(((int64_t)c.k_max + c.chunk - 1) / c.chunk) * c.chunk;
+
+    const size_t heads = (size_t)c.batch * c.G * c.H_kv;
+    const size_t btk = heads * kDP * c.r_k * sizeof(__nv_bfloat16);
+    const size_t btv = heads * kDP * c.r_v * sizeof(__nv_bfloat16);
+    const size_t pooled = c.landmarks ? heads * d.n_c * sizeof(float) : 0;
+    const size_t hi = (size_t)d.n_hi * (c.d_h / 2) * sizeof(float2);
+    const size_t lo = (size_t)kRopeLo * (c.d_h / 2) * sizeof(float2);
+    const size_t part = attend_part_floats(g) * sizeof(float);
+    void* p = nullptr;
+#define XKV_ALLOC(dst, type, bytes)                        \
+    do {                                                   \
+      XKV_TRY_CUDA(cudaMalloc(&p, (bytes) ? (bytes) : 16)); \
+      g->owned[g->n_owned++] = p;                          \
+      dst = (type)p;                                       \
+      g->workspace_bytes += (bytes);                       \
+    } while (0)
+    __nv_bfloat16 *Bt_k, *Bt_v; float2 *rhi, *rlo;
+    XKV_ALLOC(Bt_k, __nv_bfloat16*, btk);
+    XKV_ALLOC(Bt_v, __nv_bfloat16*, btv);
+    XKV_ALLOC(d.pooled, float*, pooled);
+    XKV_ALLOC(rhi, float2*, hi);
+    XKV_ALLOC(rlo, float2*, lo);
+    XKV_ALLOC(d.part, float*, part);
+    XKV_ALLOC(d.flags, unsigned int*, 256);
+#undef XKV_ALLOC
+    d.Bt_k = Bt_k; d.Bt_v = Bt_v; d.rope_hi = rhi; d.rope_lo = rlo;
+    XKV_TRY_CUDA(cudaMemsetAsync(d.flags, 0, 256, s));
+    XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_k, Bt_k, c.batch, c.G, c.r_k, c.H_kv, c.d_h, s));
+    XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_v, Bt_v, c.batch, c.G, c.r_v, c.H_kv, c.d_h, s));
+    XKV_TRY_CUDA(launch_rope_tables(rhi, rlo, d.n_hi, c.d_h, c.rope_base > 0 ? (double)c.rope_base : 1.0, s));
+    XKV_TRY_CUDA(cudaStreamSynchronize(s));
+
+    if (c.landmarks) {
+      const uint64_t rows = (uint64_t)heads * d.n_c;
+      g->has_lm_tmap = encode_rows64(g->lm_tmap, c.landmarks, rows, (uint64_t)c.d_h, 256) ? 1 : 0;
+      if (!g->has_lm_tmap) { st = XKV_ERR_CUDA; goto fail; }
+    }
+    // Tensor maps over the repacked B blocks need 16-byte row pitch and at least one 64-wide box.
+    if (c.r_k % 64 == 0 && c.r_v % 64 == 0) {
+      g->has_b_tmap = encode_rows64(g->bk_tmap, Bt_k, heads * kDP, (uint64_t)c.r_k, kDP) &&
+                      encode_rows64(g->bv_tmap, Bt_v, heads * kDP, (uint64_t)c.r_v, kDP);
+    }
+  }
+  *out = g;
+  return XKV_OK;
+fail:
+  for (int i = 0; i < g->n_owned; ++i) cudaFree(g->owned[i]);
+  delete g;
+  return st;
+}
+
+int xkv_group_destroy(xkv_group* g) {
+  if (!g) return XKV_OK;
+  int st = XKV_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { set_cuda_error(e); st = XKV_ERR_CUDA; }
+  for (int i = 0; i < g->n_owned; ++i) cudaFree(g->owned[i]);
+  delete g;
+  return st;
+}
+
+int xkv_group_workspace_bytes(const xkv_group* g, uint64_t* bytes) {
+  if (!g || !bytes) return XKV_ERR_INVALID_ARG;
+  *bytes = g->workspace_bytes;
+  return XKV_OK;
+}
+
+int xkv_group_status(xkv_group* g, uint32_t* device_flags, void* stream) {
+  if (!g) return XKV_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned int f = 0;
+  cudaError_t e = cudaMemcpyAsync(&f, g->dev.flags, sizeof(f), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(g->dev.flags, 0, sizeof(f), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+  if (device_flags) *device_flags = f;
+  if (f & XKV_FLAG_TIMEOUT) return XKV_ERR_TIMEOUT;
+  if (f & XKV_FLAG_INDEX_RANGE) return XKV_ERR_INDEX_RANGE;
+  return XKV_OK;
+}
+
+int xkv_sr_select(xkv_group* g, int layer_begin, int layer_end, const void* q, int32_t k, int32_t* sel_idx,
+                  int32_t* sel_cnt, void* stream) {
+  if (!g || !q || !sel_idx || !sel_cnt) return XKV_ERR_INVALID_ARG;
+  if (!g->cfg.landmarks) return XKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
+  if (k < 1 || k > g->cfg.k_max) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15u) || ((uintptr_t)sel_idx & 3u) || ((uintptr_t)sel_cnt & 3u)) return XKV_ERR_INVALID_ARG;
+  cudaError_t e = launch_select(g, layer_begin, layer_end, (const __nv_bfloat16*)q, k, sel_idx, sel_cnt,
+                                (cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, const void* q,
+                              const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_cap, void* out,
+                              float* lse, void* stream) {
+  if (!g || !q || !sel_idx || !sel_cnt || !out) return XKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
+  if (k_cap < 1 || k_cap > g->k_cap_max) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) ||
+      ((uintptr_t)sel_cnt & 3u) || ((uintptr_t)lse & 3u))
+    return XKV_ERR_INVALID_ARG;
+  cudaError_t e = launch_reconstruct_attend(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx,
+                                            sel_cnt, k_cap, (__nv_bfloat16*)out, lse, (cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Internal declarations shared by the translation units of libxkv (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "xkv.h"
+
+namespace xkv {
+
+constexpr int kDP = 128;          // rows of a repacked B head block (d_h padded to 128 with zeros)
+constexpr int kRopeLo = 64;       // positions covered by the fine rotary table
+constexpr int kMaxRep = 16;       // query heads per KV head
+constexpr int kAttTile = 128;     // selected rows per attention tile
+constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, head) problem
+
+// Device-side description of one window; a copy lives in the handle and is passed by value.
+struct GroupDev {
+  int G, batch, T, H_kv, H_q, d_h, r_k, r_v, c, n_c, n_rep;
+  int n_hi;                         // rows of the coarse rotary table: ceil(T / kRopeLo)
+  float sel_scale;                  // 1/sqrt(d_h) computed on the host (Algorithm 2, line 2)
+  float att_scale;                  // softmax scale of the attention
+  int use_rope;
+  const __nv_bfloat16* A_k;         // [batch][T][r_k]
+  const __nv_bfloat16* A_v;         // [batch][T][r_v]
+  const __nv_bfloat16* landmarks;   // [batch][G][H_kv][n_c][d_h]
+  const __nv_bfloat16* Bt_k;        // [batch][G][H_kv][kDP][r_k]  transposed head blocks, zero padded
+  const __nv_bfloat16* Bt_v;        // [batch][G][H_kv][kDP][r_v]
+  const float2* rope_hi;            // [n_hi][d_h/2]   (cos, sin) of (64*p_hi) * theta_i
+  const float2* rope_lo;            // [kRopeLo][d_h/2] (cos, sin) of p_lo * theta_i
+  float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
+  float* part;                      // attention partials, see xkv_attend.cu
+  unsigned int* flags;              // device flag word
+};
+
+}  // namespace xkv
+
+struct xkv_group {
+  xkv_group_config cfg;
+  xkv::GroupDev dev;
+  int device;
+  int sm_count;
+  int k_cap_max;                    // ceil(k_max/c)*c
+  size_t workspace_bytes;
+  void* owned[8];
+  int n_owned;
+  alignas(64) unsigned char lm_tmap[128];   // CUtensorMap for the landmark scan
+  int has_lm_tmap;
+  alignas(64) unsigned char bk_tmap[128];   // CUtensorMap over Bt_k rows
+  alignas(64) unsigned char bv_tmap[128];   // CUtensorMap over Bt_v rows
+  int has_b_tmap;
+};
+
+namespace xkv {
+
+void set_cuda_error(cudaError_t e);
+void count_launch(int n = 1);
+
+// xkv_prep.cu
+cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch, int G, int r, int H_kv,
+                            int d_h, cudaStream_t s);
+cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int d_h, double base, cudaStream_t s);
+
+// xkv_select.cu
+cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
+                          int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
+
+// xkv_attend.cu
+size_t attend_part_floats(const xkv_group* grp);
+cudaError_t launch_reconstruct_attend(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q,
+                                      const int32_t* sel_idx, const int32_t* sel_cnt, int k_cap,
+                                      __nv_bfloat16* out, float* lse, cudaStream_t s);
+
+}  // namespace xkv

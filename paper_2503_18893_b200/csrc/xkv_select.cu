@@ -1,0 +1,337 @@
+// Landmark-guided top-k chunk selection (App. B.1, Algorithm 2) in two kernels:
+//   score_pool_kernel  lines 2-3: streams every landmark once (HBM bound), fp32 scores in the canonical
+//                      order, max-pool over the query heads of each KV head;
+//   topk_kernel        lines 1,4: exact k_ch-th largest pooled score by radix select, then an ordered
+//                      compaction (ties to the lowest chunk index, output ascending) and expansion of
+//                      chunk ids to token rows.
+#include <cuda.h>
+
+#include "xkv_internal.cuh"
+
+namespace xkv {
+
+namespace {
+
+constexpr int kScoreRows = 256;      // landmark rows (chunks) per CTA
+constexpr int kScoreThreads = 128;   // two rows per thread
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+// One pass over the staged tile for HB query heads; returns per-row max of the scaled scores.
+template <int DH, int HB>
+__device__ __forceinline__ void score_pass(uint32_t tile, const float* __restrict__ qs, int row0, float s,
+                                           float& best0, float& best1) {
+  float acc0[HB], acc1[HB];
+#pragma unroll
+  for (int h = 0; h < HB; ++h) { acc0[h] = 0.0f; acc1[h] = 0.0f; }
+  const uint32_t sw = (uint32_t)(row0 & 7);
+  const uint32_t a0 = tile + (uint32_t)row0 * 128u;
+  const uint32_t a1 = a0 + (uint32_t)kScoreThreads * 128u;
+#pragma unroll 2
+  for (int cc = 0; cc < DH / 8; ++cc) {
+    const uint32_t off = (uint32_t)(cc >> 3) * (kScoreRows * 128u) + ((((uint32_t)cc & 7u) ^ sw) << 4);
+    const uint4 va = lds128(a0 + off);
+    const uint4 vb = lds128(a1 + off);
+    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+    const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+    for (int h = 0; h < HB; ++h) {
+      const float4 q0 = *reinterpret_cast<const float4*>(qs + h * DH + cc * 8);
+      const float4 q1 = *reinterpret_cast<const float4*>(qs + h * DH + cc * 8 + 4);
+      const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        // element 2w is the low half of word w, element 2w+1 the high half; ascending i
+        acc0[h] = fmaf(qv[2 * w], __uint_as_float(wa[w] << 16), acc0[h]);
+        acc1[h] = fmaf(qv[2 * w], __uint_as_float(wb[w] << 16), acc1[h]);
+        acc0[h] = fmaf(qv[2 * w + 1], __uint_as_float(wa[w] & 0xffff0000u), acc0[h]);
+        acc1[h] = fmaf(qv[2 * w + 1], __uint_as_float(wb[w] & 0xffff0000u), acc1[h]);
+      }
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < HB; ++h) {
+    best0 = fmaxf(best0, acc0[h] * s);
+    best1 = fmaxf(best1, acc1[h] * s);
+  }
+}
+
+// grid.x = ceil(n_c / 256) tiles, grid.y = (layers in call) * batch * H_kv problems.
+template <int DH>
+__global__ void __launch_bounds__(kScoreThreads)
+score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const __nv_bfloat16* __restrict__ q,
+                  int l0) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_storage;
+  const uint32_t tile = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  float* qs = reinterpret_cast<float*>(smem_raw + (tile - smem_u32(smem_raw)) + (DH / 64) * kScoreRows * 128);
+  const uint32_t bar = smem_u32(&bar_storage);
+
+  const int g = blockIdx.y % dev.H_kv;
+  const int b = (blockIdx.y / dev.H_kv) % dev.batch;
+  const int l = l0 + blockIdx.y / (dev.H_kv * dev.batch);
+  const int j0 = blockIdx.x * kScoreRows;
+  const long long prob_lm = ((long long)b * dev.G + l) * dev.H_kv + g;       // landmark order
+  const long long prob_out = ((long long)l * dev.batch + b) * dev.H_kv + g;  // [G][batch][H_kv] order
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
+    const int y = (int)(prob_lm * dev.n_c + j0);
+#pragma unroll
+    for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar);
+  }
+  // queries of this KV head, widened to fp32 while the landmarks are in flight
+  const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * dev.n_rep) * DH;
+  for (int i = threadIdx.x; i < dev.n_rep * DH; i += kScoreThreads) qs[i] = __bfloat162float(qg[i]);
+  __syncthreads();
+
+  if (!mbar_wait_bounded(bar, 0)) {
+    if (threadIdx.x == 0) atomicOr(dev.flags, XKV_FLAG_TIMEOUT);
+    return;
+  }
+  float best0 = -INFINITY, best1 = -INFINITY;
+  const int row0 = threadIdx.x;
+  for (int h0 = 0; h0 < dev.n_rep; h0 += 4) {
+    const int hb = min(4, dev.n_rep - h0);
+    const float* qh = qs + h0 * DH;
+    if (hb == 4) score_pass<DH, 4>(tile, qh, row0, dev.sel_scale, best0, best1);
+    else if (hb == 3) score_pass<DH, 3>(tile, qh, row0, dev.sel_scale, best0, best1);
+    else if (hb == 2) score_pass<DH, 2>(tile, qh, row0, dev.sel_scale, best0, best1);
+    else score_pass<DH, 1>(tile, qh, row0, dev.sel_scale, best0, best1);
+  }
+  float* dst = dev.pooled + prob_out * dev.n_c;
+  if (j0 + row0 < dev.n_c) dst[j0 + row0] = best0;
+  if (j0 + row0 + kScoreThreads < dev.n_c) dst[j0 + row0 + kScoreThreads] = best1;
+}
+
+// ---------------------------------------------------------------------------------------------
+
+constexpr int kTopkThreads = 1024;
+constexpr int kTopkItems = 16;   // consecutive chunks per thread in the compaction
+
+// Order-preserving map float -> uint32 (larger float = larger key), with -0 folded onto +0.
+__device__ __forceinline__ uint32_t score_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  if (u == 0x80000000u) u = 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// One CTA per (layer, sequence, KV head).  grid.x = problems of the call.
+__global__ void __launch_bounds__(kTopkThreads)
+topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel_idx,
+            int32_t* __restrict__ sel_cnt) {
+  __shared__ uint32_t whist[kTopkThreads / 32][256];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t warp_tot[kTopkThreads / 32];
+  __shared__ uint32_t sh_prefix, sh_need;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_layer = dev.batch * dev.H_kv;
+  const long long prob = (long long)l0 * per_layer + blockIdx.x;     // [G][batch][H_kv] order
+  const float* __restrict__ S = dev.pooled + prob * dev.n_c;
+  int32_t* __restrict__ out = sel_idx + prob * k_cap;
+  const int n_c = dev.n_c, c = dev.c, T = dev.T;
+
+  uint32_t thr = 0, need_eq = 0;
+  const bool all = (k_ch >= n_c);
+  if (!all) {
+    uint32_t prefix = 0, mask = 0, need = (uint32_t)k_ch;
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int i = tid; i < (kTopkThreads / 32) * 256; i += kTopkThreads) (&whist[0][0])[i] = 0;
+      __syncthreads();
+      for (int j = tid; j < n_c; j += kTopkThreads) {
+        const uint32_t key = score_key(S[j]);
+        if ((key & mask) == prefix) atomicAdd(&whist[warp][(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 256) {
+        uint32_t s = 0;
+#pragma unroll 8
+        for (int w = 0; w < kTopkThreads / 32; ++w) s += whist[w][tid];
+        hist[tid] = s;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // lane owns bins 8*lane .. 8*lane+7; suffix sums from the top bin downwards
+        uint32_t loc[8], tot = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { loc[i] = hist[lane * 8 + i]; tot += loc[i]; }
+        uint32_t above = tot;                       // inclusive suffix over lanes >= lane
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
+          if (lane + o < 32) above += v;
+        }
+        above -= tot;                               // elements in bins of higher lanes
+        // exactly one lane holds the bin where the running count crosses `need`
+        if (above < need && above + tot >= need) {
+          uint32_t run = above;
+          int bsel = 0;
+#pragma unroll
+          for (int i = 7; i >= 0; --i) {
+            if (run < need && run + loc[i] >= need) { bsel = i; break; }
+            run += loc[i];
+          }
+          sh_prefix = prefix | ((uint32_t)(lane * 8 + bsel) << shift);
+          sh_need = need - run;
+        }
+      }
+      __syncthreads();
+      prefix = sh_prefix;
+      need = sh_need;
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+    thr = prefix;
+    need_eq = need;
+  }
+
+  // Ordered compaction: chunk j is taken if key > thr, or key == thr and fewer than need_eq equal
+  // keys precede it.  Positions follow ascending j.
+  uint32_t run_gt = 0, run_eq = 0;                  // totals of the super-blocks already done
+  const int super = kTopkThreads * kTopkItems;
+  for (int base = 0; base < n_c; base += super) {
+    const int j0 = base + tid * kTopkItems;
+    uint32_t gtm = 0, eqm = 0;                      // bit i set: item i is > / == thr
+    if (all) {
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) if (j0 + i < n_c) gtm |= 1u << i;
+    } else {
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) {
+        if (j0 + i < n_c) {
+          const uint32_t key = score_key(S[j0 + i]);
+          gtm |= (key > thr ? 1u : 0u) << i;
+          eqm |= (key == thr ? 1u : 0u) << i;
+        }
+      }
+    }
+    const uint32_t mine = (uint32_t)__popc(gtm) | ((uint32_t)__popc(eqm) << 16);
+    uint32_t inc = mine;                            // inclusive warp scan of packed (gt, eq) counts
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t t = warp_tot[lane];
+      uint32_t ti = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, ti, o);
+        if (lane >= o) ti += v;
+      }
+      warp_tot[lane] = ti - t;                      // exclusive prefix of warp totals
+      if (lane == 31) { sh_prefix = ti; }           // super-block total
+    }
+    __syncthreads();
+    const uint32_t excl = inc - mine + warp_tot[warp];
+    uint32_t gt_before = run_gt + (excl & 0xffffu);
+    uint32_t eq_before = run_eq + (excl >> 16);
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) {
+      const bool is_gt = (gtm >> i) & 1u, is_eq = (eqm >> i) & 1u;
+      const bool take = is_gt || (is_eq && eq_before < need_eq);
+      if (take) {
+        const uint32_t pos = gt_before + min(eq_before, need_eq);
+        const int j = j0 + i;
+        const int rows = min(c, T - j * c);
+        for (int t = 0; t < rows; ++t) out[(size_t)pos * c + t] = j * c + t;
+      }
+      gt_before += is_gt ? 1u : 0u;
+      eq_before += is_eq ? 1u : 0u;
+    }
+    run_gt += sh_prefix & 0xffffu;
+    run_eq += sh_prefix >> 16;
+    __syncthreads();
+  }
+  // Row count: k_ch whole chunks unless the ragged last chunk was taken (it is then the last one).
+  const int taken = all ? n_c : k_ch;
+  int cnt = taken * c;
+  {
+    bool last_in = all;
+    if (!all) {
+      const uint32_t key = score_key(S[n_c - 1]);
+      // the last chunk has the highest index, so it wins a tie only if every equal key fits
+      last_in = key > thr || (key == thr && run_eq <= need_eq);
+    }
+    if (last_in) cnt -= (n_c * c - T);
+  }
+  for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
+  if (tid == 0) sel_cnt[prob] = cnt;
+}
+
+}  // namespace
+
+cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
+                          int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
+  const GroupDev& dev = grp->dev;
+  const int problems = (l1 - l0) * dev.batch * dev.H_kv;
+  const int tiles = (dev.n_c + kScoreRows - 1) / kScoreRows;
+  const int c = dev.c;
+  const int k_ch_raw = (k + c - 1) / c;
+  const int k_ch = k_ch_raw < dev.n_c ? k_ch_raw : dev.n_c;
+  const int k_cap = k_ch_raw * c;
+  CUtensorMap tmap;
+  memcpy(&tmap, grp->lm_tmap, sizeof(tmap));
+  const size_t smem = 1024 + (size_t)(dev.d_h / 64) * kScoreRows * 128 + (size_t)dev.n_rep * dev.d_h * 4;
+  dim3 grid(tiles, problems);
+  cudaError_t e;
+  if (dev.d_h == 128) {
+    e = cudaFuncSetAttribute(score_pool_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    score_pool_kernel<128><<<grid, kScoreThreads, smem, s>>>(tmap, dev, q, l0);
+  } else {
+    e = cudaFuncSetAttribute(score_pool_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    score_pool_kernel<64><<<grid, kScoreThreads, smem, s>>>(tmap, dev, q, l0);
+  }
+  count_launch();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  topk_kernel<<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace xkv

@@ -1,0 +1,152 @@
+"""Synthetic long-context workloads for tests and the benchmark.
+
+Everything here prepares INPUTS of the decode path (it plays the role of the prefill side, which
+is outside the library): factors drawn by `synth.make_factors`, and chunk landmarks computed from
+the keys those factors represent (App. B.1, Algorithm 1 lines 1-3) with plain torch ops on
+whatever device the factors live on.  The decode step itself is only ever run through the
+C ABI (`xkv.py`).
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import torch
+
+from . import synth
+
+
+def rope_angles(T: int, d_h: int, base: float, device, start: int = 0):
+    """cos/sin of p*theta_i (fp64 angles, returned as fp32), p in [start, start+T), i < d_h/2."""
+    half = d_h // 2
+    theta = torch.pow(torch.tensor(float(base), dtype=torch.float64, device=device),
+                      -torch.arange(half, dtype=torch.float64, device=device) / half)
+    phi = torch.arange(start, start + T, dtype=torch.float64, device=device)[:, None] * theta[None, :]
+    return torch.cos(phi).float(), torch.sin(phi).float()
+
+
+def landmarks_from_factors(A_k: torch.Tensor, B_k: torch.Tensor, H_kv: int, c: int, rope_base: float,
+                           rows_per_pass: int = 16384) -> torch.Tensor:
+    """Chunk means of the post-RoPE keys K_l = rope(A_k @ B_k[l]) of every layer and sequence.
+
+    A_k (batch,T,r) bf16, B_k (batch,G,r,d) bf16  ->  bf16 (batch,G,H_kv,n_c,d_h).
+    The mean of a ragged last chunk runs over the rows present.  fp32 arithmetic.
+    """
+    batch, T, r = A_k.shape
+    G, d = B_k.shape[1], B_k.shape[3]
+    d_h = d // H_kv
+    half = d_h // 2
+    n_c = -(-T // c)
+    dev = A_k.device
+    out = torch.empty((batch, G, H_kv, n_c, d_h), dtype=torch.bfloat16, device=dev)
+    step = max(c, (rows_per_pass // c) * c)
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        for b in range(batch):
+            for l in range(G):
+                Bl = B_k[b, l].float()
+                for t0 in range(0, T, step):
+                    t1 = min(T, t0 + step)
+                    K = (A_k[b, t0:t1].float() @ Bl).view(t1 - t0, H_kv, d_h)
+                    if rope_base > 0:
+                        cs, sn = rope_angles(t1 - t0, d_h, rope_base, dev, start=t0)
+                        x1, x2 = K[..., :half], K[..., half:]
+                        K = torch.cat([x1 * cs[:, None, :] - x2 * sn[:, None, :],
+                                       x2 * cs[:, None, :] + x1 * sn[:, None, :]], dim=-1)
+                    n_full = (t1 - t0) // c
+                    j0 = t0 // c
+                    if n_full:
+                        m = K[:n_full * c].view(n_full, c, H_kv, d_h).mean(dim=1)
+                        out[b, l, :, j0:j0 + n_full] = m.permute(1, 0, 2).to(torch.bfloat16)
+                    if n_full * c < t1 - t0:
+                        m = K[n_full * c:].mean(dim=0)
+                        out[b, l, :, j0 + n_full] = m.to(torch.bfloat16)
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+    return out
+
+
+@dataclasses.dataclass
+class GroupInputs:
+    A_k: torch.Tensor
+    A_v: torch.Tensor
+    B_k: torch.Tensor
+    B_v: torch.Tensor
+    landmarks: torch.Tensor
+    q: torch.Tensor          # (n_steps, G, batch, H_q, d_h)
+
+
+def make_group_inputs(shape: synth.SRShape, group: int = 0, n_steps: int = 1, device="cpu") -> GroupInputs:
+    """Factors, landmarks and queries of one window, drawn directly (no factorisation is run)."""
+    A_k, A_v, B_k, B_v = synth.make_factors(shape, group, device)
+    lm = landmarks_from_factors(A_k, B_k, shape.H_kv, shape.c, shape.rope_base)
+    q = synth.make_queries(shape, n_steps, group, device)
+    return GroupInputs(A_k, A_v, B_k, B_v, lm, q)
+
+
+def algorithmic_bytes(shape: synth.SRShape, unique_rows=None) -> dict:
+    """Bytes one window-step has to move (bf16 storage), per term.
+
+    landmarks: every landmark is read once;  rows_issued: every selected row of A_k and A_v;
+    rows_unique: the rows of the union over the (layer, head) problems of each sequence
+    (pass the measured count; default = min(issued, T));  B: both reconstruction matrices.
+    """
+    problems = shape.G * shape.H_kv * shape.batch
+    M = min(shape.k_cap, shape.T)
+    lm = shape.batch * shape.G * shape.n_c * shape.d * 2
+    issued = problems * M * (shape.r_k + shape.r_v) * 2
+    if unique_rows is None:
+        unique_rows = shape.batch * min(shape.G * shape.H_kv * M, shape.T)
+    uniq = unique_rows * (shape.r_k + shape.r_v) * 2
+    Bm = shape.batch * shape.G * (shape.r_k + shape.r_v) * shape.d * 2
+    small = shape.G * shape.batch * shape.H_q * shape.d_h * 2 * 2 + problems * (M + 1) * 4 * 2
+    return {"landmarks": lm, "rows_issued": issued, "rows_unique": uniq, "B": Bm, "small": small,
+            "bytes_min": lm + uniq + Bm + small, "bytes_issued": lm + issued + Bm + small}
+
+
+def algorithmic_flops(shape: synth.SRShape) -> float:
+    """2 * sum over problems of M * d_h * (r_K + r_V)  (the paper's SR cost with the multiply-add factor)."""
+    problems = shape.G * shape.H_kv * shape.batch
+    M = min(shape.k_cap, shape.T)
+    return 2.0 * problems * M * shape.d_h * (shape.r_k + shape.r_v)
+
+
+class DeviceWorkload:
+    """All windows of a configuration resident on one GPU, with their handles and output buffers."""
+
+    def __init__(self, shape: synth.SRShape, n_steps: int = 4, device="cuda", groups=None):
+        from . import xkv  # loads the CUDA library; raises if it is not built
+        self.xkv = xkv
+        self.shape = shape
+        self.device = device
+        self.groups = []
+        self.inputs = []
+        ids = range(shape.n_groups) if groups is None else groups
+        for gi in ids:
+            inp = make_group_inputs(shape, gi, n_steps, device)
+            grp = xkv.create_from_tensors(inp.A_k, inp.A_v, inp.B_k, inp.B_v, inp.landmarks, H_kv=shape.H_kv,
+                                          H_q=shape.H_q, k_max=shape.k, chunk=shape.c, rope_base=shape.rope_base)
+            self.inputs.append(inp)
+            self.groups.append(grp)
+        n = len(self.groups)
+        s = shape
+        self.sel_idx = torch.empty((n, s.G, s.batch, s.H_kv, s.k_cap), dtype=torch.int32, device=device)
+        self.sel_cnt = torch.empty((n, s.G, s.batch, s.H_kv), dtype=torch.int32, device=device)
+        self.out = torch.empty((n, s.G, s.batch, s.H_q, s.d_h), dtype=torch.bfloat16, device=device)
+        self.lse = torch.empty((n, s.G, s.batch, s.H_q), dtype=torch.float32, device=device)
+        self.n_steps = n_steps
+
+    def step(self, i: int, q_override=None) -> None:
+        """One decode step: every window, select then reconstruct+attend, on the current stream."""
+        s, x = self.shape, self.xkv
+        for gi, grp in enumerate(self.groups):
+            q = self.inputs[gi].q[i % self.n_steps] if q_override is None else q_override[gi]
+            x.xkv_sr_select(grp, 0, s.G, q, s.k, self.sel_idx[gi], self.sel_cnt[gi])
+            x.xkv_sr_reconstruct_attend(grp, 0, s.G, q, self.sel_idx[gi], self.sel_cnt[gi], s.k_cap,
+                                        self.out[gi], self.lse[gi])
+
+    def close(self):
+        for g in self.groups:
+            self.xkv.xkv_group_destroy(g)
+        self.groups = []

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of libxkv (argument marshalling only; every step runs in the CUDA library).
+
+The functions carry the names of the C ABI (include/xkv.h).  Tensors are torch CUDA tensors used
+for their device memory; the stream is torch's current stream unless one is given.  Importing this
+module loads libxkv.so from the package directory and raises if it has not been built: there is no
+CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libxkv.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2503_18893_b200.build` "
+        "(nvcc, sm_100a). There is no fallback path.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+XKV_OK = 0
+XKV_ERR_INVALID_ARG = -1
+XKV_ERR_UNSUPPORTED = -2
+XKV_ERR_ARCH = -3
+XKV_ERR_CUDA = -4
+XKV_ERR_OOM = -5
+XKV_ERR_INDEX_RANGE = -6
+XKV_ERR_TIMEOUT = -7
+XKV_FLAG_INDEX_RANGE = 1
+XKV_FLAG_TIMEOUT = 2
+
+
+class xkv_group_config(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("G", ctypes.c_int32), ("batch", ctypes.c_int32), ("T", ctypes.c_int32),
+        ("H_kv", ctypes.c_int32), ("H_q", ctypes.c_int32), ("d_h", ctypes.c_int32),
+        ("r_k", ctypes.c_int32), ("r_v", ctypes.c_int32), ("chunk", ctypes.c_int32),
+        ("k_max", ctypes.c_int32),
+        ("rope_base", ctypes.c_float), ("softmax_scale", ctypes.c_float),
+        ("A_k", ctypes.c_void_p), ("A_v", ctypes.c_void_p),
+        ("B_k", ctypes.c_void_p), ("B_v", ctypes.c_void_p),
+        ("landmarks", ctypes.c_void_p),
+    ]
+
+
+_P = ctypes.c_void_p
+_lib.xkv_group_create.argtypes = [ctypes.POINTER(xkv_group_config), _P, ctypes.POINTER(_P)]
+_lib.xkv_group_create.restype = ctypes.c_int
+_lib.xkv_sr_select.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, ctypes.c_int32, _P, _P, _P]
+_lib.xkv_sr_select.restype = ctypes.c_int
+_lib.xkv_sr_reconstruct_attend.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, ctypes.c_int32, _P, _P, _P]
+_lib.xkv_sr_reconstruct_attend.restype = ctypes.c_int
+_lib.xkv_group_destroy.argtypes = [_P]
+_lib.xkv_group_destroy.restype = ctypes.c_int
+_lib.xkv_group_status.argtypes = [_P, ctypes.POINTER(ctypes.c_uint32), _P]
+_lib.xkv_group_status.restype = ctypes.c_int
+_lib.xkv_group_bytes.argtypes = [ctypes.POINTER(xkv_group_config), ctypes.POINTER(ctypes.c_uint64),
+                                 ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_group_bytes.restype = ctypes.c_int
+_lib.xkv_group_workspace_bytes.argtypes = [_P, ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_group_workspace_bytes.restype = ctypes.c_int
+_lib.xkv_strerror.argtypes = [ctypes.c_int]
+_lib.xkv_strerror.restype = ctypes.c_char_p
+_lib.xkv_last_cuda_error.restype = ctypes.c_int
+_lib.xkv_kernel_launch_count.restype = ctypes.c_uint64
+
+
+class XKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {xkv_strerror(status)} (status {status}, cuda error {xkv_last_cuda_error()})")
+
+
+def xkv_strerror(status: int) -> str:
+    return _lib.xkv_strerror(int(status)).decode()
+
+
+def xkv_last_cuda_error() -> int:
+    return int(_lib.xkv_last_cuda_error())
+
+
+def xkv_kernel_launch_count() -> int:
+    return int(_lib.xkv_kernel_launch_count())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def make_config(*, G, batch, T, H_kv, H_q, d_h, r_k, r_v, k_max, chunk=8, rope_base=10000.0,
+                softmax_scale=0.0, A_k=None, A_v=None, B_k=None, B_v=None, landmarks=None) -> xkv_group_config:
+    """Fill an xkv_group_config; tensor arguments contribute their device addresses only."""
+    cfg = xkv_group_config()
+    cfg.struct_size = ctypes.sizeof(xkv_group_config)
+    cfg.G, cfg.batch, cfg.T, cfg.H_kv, cfg.H_q, cfg.d_h = G, batch, T, H_kv, H_q, d_h
+    cfg.r_k, cfg.r_v, cfg.chunk, cfg.k_max = r_k, r_v, chunk, k_max
+    cfg.rope_base, cfg.softmax_scale = rope_base, softmax_scale
+    cfg.A_k, cfg.A_v, cfg.B_k, cfg.B_v, cfg.landmarks = _ptr(A_k), _ptr(A_v), _ptr(B_k), _ptr(B_v), _ptr(landmarks)
+    return cfg
+
+
+def xkv_group_bytes(cfg: xkv_group_config):
+    """(factor_bytes, landmark_bytes) of one window; host only."""
+    f, l = ctypes.c_uint64(), ctypes.c_uint64()
+    st = _lib.xkv_group_bytes(ctypes.byref(cfg), ctypes.byref(f), ctypes.byref(l))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_group_bytes")
+    return f.value, l.value
+
+
+class Group:
+    """Owner of one xkv_group handle.  Keeps the borrowed tensors alive."""
+
+    def __init__(self, handle: int, cfg: xkv_group_config, keep):
+        self.handle, self.cfg, self._keep = handle, cfg, keep
+
+    @property
+    def k_cap_max(self) -> int:
+        c = self.cfg.chunk or 8
+        return -(-self.cfg.k_max // c) * c
+
+    def __del__(self):
+        try:
+            xkv_group_destroy(self)
+        except Exception:
+            pass
+
+
+def xkv_group_create(cfg: xkv_group_config, stream=None, keep=None) -> Group:
+    h = _P()
+    st = _lib.xkv_group_create(ctypes.byref(cfg), _stream(stream), ctypes.byref(h))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_group_create")
+    return Group(h.value, cfg, keep)
+
+
+def xkv_group_destroy(grp: Group) -> None:
+    if grp.handle:
+        h, grp.handle = grp.handle, 0
+        st = _lib.xkv_group_destroy(h)
+        if st != XKV_OK:
+            raise XKVError(st, "xkv_group_destroy")
+
+
+def xkv_sr_select(grp: Group, layer_begin: int, layer_end: int, q, k: int, sel_idx, sel_cnt, stream=None) -> None:
+    st = _lib.xkv_sr_select(grp.handle, layer_begin, layer_end, _ptr(q), k, _ptr(sel_idx), _ptr(sel_cnt),
+                            _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_sr_select")
+
+
+def xkv_sr_reconstruct_attend(grp: Group, layer_begin: int, layer_end: int, q, sel_idx, sel_cnt, k_cap: int,
+                              out, lse=None, stream=None) -> None:
+    st = _lib.xkv_sr_reconstruct_attend(grp.handle, layer_begin, layer_end, _ptr(q), _ptr(sel_idx), _ptr(sel_cnt),
+                                        k_cap, _ptr(out), _ptr(lse), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_sr_reconstruct_attend")
+
+
+def xkv_group_status(grp: Group, stream=None):
+    """(status, flags): reads and clears the device flag word (blocks on the stream)."""
+    f = ctypes.c_uint32()
+    st = _lib.xkv_group_status(grp.handle, ctypes.byref(f), _stream(stream))
+    return st, f.value
+
+
+def xkv_group_workspace_bytes(grp: Group) -> int:
+    b = ctypes.c_uint64()
+    st = _lib.xkv_group_workspace_bytes(grp.handle, ctypes.byref(b))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_group_workspace_bytes")
+    return b.value
+
+
+def create_from_tensors(A_k, A_v, B_k, B_v, landmarks, *, H_kv, H_q, k_max, chunk=8, rope_base=10000.0,
+                        softmax_scale=0.0, stream=None) -> Group:
+    """Convenience: read the sizes off the tensors (layouts of xkv_group_config) and create the handle."""
+    batch, T, r_k = A_k.shape
+    r_v = A_v.shape[2]
+    G = B_k.shape[1]
+    d_h = B_k.shape[3] // H_kv
+    for t in (A_k, A_v, B_k, B_v, landmarks):
+        if t is not None:
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
+    cfg = make_config(G=G, batch=batch, T=T, H_kv=H_kv, H_q=H_q, d_h=d_h, r_k=r_k, r_v=r_v, k_max=k_max,
+                      chunk=chunk, rope_base=rope_base, softmax_scale=softmax_scale, A_k=A_k, A_v=A_v,
+                      B_k=B_k, B_v=B_v, landmarks=landmarks)
+    return xkv_group_create(cfg, stream, keep=(A_k, A_v, landmarks))
