@@ -139,7 +139,10 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     d.G = c.G; d.batch = c.batch; d.T = c.T; d.H_kv = c.H_kv; d.H_q = c.H_q; d.d_h = c.d_h;
     d.r_k = c.r_k; d.r_v = c.r_v; d.c = c.chunk; d.n_c = (c.T + c.chunk - 1) / c.chunk;
     d.n_rep = c.H_q / c.H_kv;
-    d.n_hi = (c.T + kRopeLo - 1) / kRopeLo;
+    // fine table of 8 positions (one landmark chunk); coarser splits keep the coarse table under 64 MB
+    d.rope_shift = 3;
+    while (((size_t)((c.T >> d.rope_shift) + 1) * (c.d_h / 2) * sizeof(float2)) > ((size_t)64 << 20)) d.rope_shift += 3;
+    d.n_hi = (c.T + (1 << d.rope_shift) - 1) >> d.rope_shift;
     d.sel_scale = 1.0f / sqrtf((float)c.d_h);
     d.att_scale = c.softmax_scale > 0.0f ? c.softmax_scale : 1.0f / sqrtf((float)c.d_h);
     d.use_rope = c.rope_base > 0.0f;
@@ -152,8 +155,9 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     const size_t btv = heads * kDP * c.r_v * sizeof(__nv_bfloat16);
     const size_t pooled = c.landmarks ? heads * d.n_c * sizeof(float) : 0;
     const size_t hi = (size_t)d.n_hi * (c.d_h / 2) * sizeof(float2);
-    const size_t lo = (size_t)kRopeLo * (c.d_h / 2) * sizeof(float2);
-    const size_t part = attend_part_floats(g) * sizeof(float);
+    const size_t lo = ((size_t)1 << d.rope_shift) * (c.d_h / 2) * sizeof(float2);
+    const size_t pf0 = attend_part_floats(g), pf1 = fused_part_floats(g);
+    const size_t part = (pf0 > pf1 ? pf0 : pf1) * sizeof(float);
     void* p = nullptr;
 #define XKV_ALLOC(dst, type, bytes)                        \
     do {                                                   \
@@ -175,7 +179,7 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     XKV_TRY_CUDA(cudaMemsetAsync(d.flags, 0, 256, s));
     XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_k, Bt_k, c.batch, c.G, c.r_k, c.H_kv, c.d_h, s));
     XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_v, Bt_v, c.batch, c.G, c.r_v, c.H_kv, c.d_h, s));
-    XKV_TRY_CUDA(launch_rope_tables(rhi, rlo, d.n_hi, c.d_h, c.rope_base > 0 ? (double)c.rope_base : 1.0, s));
+    XKV_TRY_CUDA(launch_rope_tables(rhi, rlo, d.n_hi, d.rope_shift, c.d_h, c.rope_base > 0 ? (double)c.rope_base : 1.0, s));
     XKV_TRY_CUDA(cudaStreamSynchronize(s));
 
     if (c.landmarks) {
@@ -183,10 +187,14 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
       g->has_lm_tmap = encode_rows64(g->lm_tmap, c.landmarks, rows, (uint64_t)c.d_h, 256) ? 1 : 0;
       if (!g->has_lm_tmap) { st = XKV_ERR_CUDA; goto fail; }
     }
-    // Tensor maps over the repacked B blocks need 16-byte row pitch and at least one 64-wide box.
-    if (c.r_k % 64 == 0 && c.r_v % 64 == 0) {
-      g->has_b_tmap = encode_rows64(g->bk_tmap, Bt_k, heads * kDP, (uint64_t)c.r_k, kDP) &&
-                      encode_rows64(g->bv_tmap, Bt_v, heads * kDP, (uint64_t)c.r_v, kDP);
+    // Tensor maps over the repacked B blocks (row pitch r*2 bytes is a multiple of 16 because r % 8 == 0;
+    // a slab that reaches past column r is zero-filled by the copy engine).
+    g->has_b_tmap = encode_rows64(g->bk_tmap, Bt_k, heads * kDP, (uint64_t)c.r_k, kDP) &&
+                    encode_rows64(g->bv_tmap, Bt_v, heads * kDP, (uint64_t)c.r_v, kDP);
+    if (!g->has_b_tmap) { st = XKV_ERR_CUDA; goto fail; }
+    {
+      const char* e = getenv("XKV_ATTEND_IMPL");
+      g->attend_impl = (e && e[0] == 't') ? 1 : 0;
     }
   }
   *out = g;
@@ -249,8 +257,11 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) ||
       ((uintptr_t)sel_cnt & 3u) || ((uintptr_t)lse & 3u))
     return XKV_ERR_INVALID_ARG;
-  cudaError_t e = launch_reconstruct_attend(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx,
-                                            sel_cnt, k_cap, (__nv_bfloat16*)out, lse, (cudaStream_t)stream);
+  cudaError_t e = g->attend_impl
+                      ? launch_reconstruct_attend(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt,
+                                                  k_cap, (__nv_bfloat16*)out, lse, (cudaStream_t)stream)
+                      : launch_fused(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt, k_cap,
+                                     (__nv_bfloat16*)out, lse, (cudaStream_t)stream);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }

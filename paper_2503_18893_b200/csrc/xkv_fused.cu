@@ -1,0 +1,536 @@
+// Selective reconstruction (Sec. 3.2, Eq. 3) fused with decode attention over the rebuilt rows: the
+// tensor-core path.  One persistent CTA per SM walks a contiguous range of 128-row tiles of the selected
+// sets; a problem is one (layer, sequence, KV head).
+//
+// Per tile (128 selected rows S_t of one problem):
+//   K_hat   [j][d] = sum_m A_k[S_t[j]][m] * B_k[m][d]     tcgen05.mma, M = rows, N = d_h, accumulator in TMEM
+//   logits  z[h][j] = scale * <q_h, rope(K_hat[j])>         thread j owns TMEM lane j (one rebuilt key row)
+//   V_hat^T [d][j] = sum_m B_v[m][d] * A_v[S_t[j]][m]     tcgen05.mma, M = d_h, N = rows
+//   o[h][d] += sum_j p[h][j] * V_hat^T[d][j]                thread d owns TMEM lane d; online softmax
+// Rebuilt K/V never leave the SM.  Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-11 gather
+// producers (cp.async of the selected rows, TMA of the B slabs), 12 MMA issue.
+// Every wait is bounded; a wait that runs out raises XKV_FLAG_TIMEOUT and the CTA winds down.
+#include <cuda.h>
+
+#include "xkv_internal.cuh"
+#include "xkv_ptx.cuh"
+
+namespace xkv {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kTile = 128;                       // selected rows per tile
+constexpr int kSlabBytes = kTile * 128;          // 128 rows x 64 bf16 (one 128-byte swizzle row each)
+constexpr int kStageBytes = 2 * kSlabBytes;      // gathered rows + B slab
+constexpr int kLag = 3;                          // cp.async groups a producer thread keeps in flight
+constexpr int kThreads = 13 * 32;
+constexpr int kPosBufs = 4;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct Sched {
+  int l0;            // first layer of the call
+  int tpp;           // tiles per problem = ceil(k_cap / 128)
+  int n_tiles;       // problems * tpp
+  int n_ctas;
+  int n_slots;       // partial slots per problem
+  int k_cap;
+  int stages;
+};
+
+struct Bars {        // offsets (in 8-byte words) into the barrier array
+  int full, empty, kfull, kempty, vfull, vempty, pfull, pempty, grp, total;
+};
+__host__ __device__ inline Bars bar_layout(int stages) {
+  Bars b;
+  b.full = 0; b.empty = stages; b.kfull = 2 * stages; b.kempty = b.kfull + 2; b.vfull = b.kempty + 2;
+  b.vempty = b.vfull + 2; b.pfull = b.vempty + 2; b.pempty = b.pfull + 2; b.grp = b.pempty + 2; b.total = b.grp + 1;
+  return b;
+}
+
+// cta that owns global tile t when cta i owns tiles [i*N/C, (i+1)*N/C)
+__device__ __forceinline__ int cta_of_tile(long long t, int C, int N) { return (int)(((t + 1) * C - 1) / N); }
+
+struct Ctx {
+  volatile int* abort;
+  unsigned int* flags;
+};
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait on an mbarrier phase.  Returns false if another thread of the CTA has given up, or if the
+// phase does not complete within kWaitLimitNs (then this thread raises the flag and makes the others give up).
+__device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 0u) {
+      if (*c.abort) return false;
+      if (global_ns() - t0 > kWaitLimitNs) break;
+    }
+  }
+  *c.abort = 1;
+  atomicOr(c.flags, XKV_FLAG_TIMEOUT);
+  return false;
+}
+
+template <int DH, int NR>
+__global__ void __launch_bounds__(kThreads, 1)
+sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constant__ CUtensorMap bv_map, GroupDev dev,
+                Sched sc, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ sel_idx,
+                const int32_t* __restrict__ sel_cnt) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int HALF = DH / 2;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  const int S = sc.stages;
+  // carve-up after the stage ring
+  float* q_s = reinterpret_cast<float*>(gen + (size_t)S * kStageBytes);          // [NR][DH]
+  float* P_s = q_s + NR * DH;                                                    // [2][NR][128]
+  float* alpha_s = P_s + 2 * NR * kTile;                                         // [2][NR]
+  float* red_s = alpha_s + 2 * NR;                                               // [2][4][NR]
+  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [4][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(pos_s + kPosBufs * kTile);
+  const Bars bl = bar_layout(S);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + bl.total);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto BAR = [&](int word) { return bar0 + 8u * (uint32_t)word; };
+  Ctx ctx{abort_flag, dev.flags};
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 129); mbar_init(BAR(bl.empty + s), 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(BAR(bl.kfull + b), 1); mbar_init(BAR(bl.kempty + b), 128);
+      mbar_init(BAR(bl.vfull + b), 1); mbar_init(BAR(bl.vempty + b), 128);
+      mbar_init(BAR(bl.pfull + b), 128); mbar_init(BAR(bl.pempty + b), 128);
+    }
+    mbar_init(BAR(bl.grp), 128);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 12) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int C = sc.n_ctas, N = sc.n_tiles;
+  const long long t_begin = ((long long)blockIdx.x * N) / C, t_end = ((long long)(blockIdx.x + 1) * N) / C;
+  const int per_layer = dev.batch * dev.H_kv;
+  const int n_rep = dev.n_rep;
+
+  // decode a problem ordinal of the call into (l, b, g)
+  auto prob_of = [&](int py, int& l, int& b, int& g) {
+    g = py % dev.H_kv; b = (py / dev.H_kv) % dev.batch; l = sc.l0 + py / per_layer;
+    return ((long long)l * dev.batch + b) * dev.H_kv + g;
+  };
+
+  if (warp >= 8 && warp < 12) {
+    // =============================== producers: gather rows of A, TMA the B slabs ===============================
+    const int pt = tid - 256;
+    const uint32_t row_off = (uint32_t)pt * 128u, sw = (uint32_t)(pt & 7);
+    long long gs = 0;                 // stages issued so far (ring position)
+    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    long long prob = 0;
+    bool ok = true;
+    for (long long t = t_begin; t < t_end && ok; ++t) {
+      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
+      if (py != cur_py) { cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
+      const int row0 = ti * kTile;
+      if (row0 >= cnt) continue;
+      int p = -1;
+      if (row0 + pt < cnt) {
+        p = sel_idx[prob * sc.k_cap + row0 + pt];
+        if (p < 0 || p >= dev.T) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
+      }
+      pos_s[(it & (kPosBufs - 1)) * kTile + pt] = p;
+      const size_t row = (size_t)b * dev.T + (size_t)(p < 0 ? 0 : p);
+      const int head_row = (int)((((size_t)b * dev.G + l) * dev.H_kv + g) * kDP);
+#pragma unroll 1
+      for (int phase = 0; phase < 2 && ok; ++phase) {
+        const int r = phase ? dev.r_v : dev.r_k;
+        const __nv_bfloat16* src = (phase ? dev.A_v : dev.A_k) + row * r;
+        const CUtensorMap* map = phase ? &bv_map : &bk_map;
+        const int nks = (r + 63) >> 6;
+#pragma unroll 1
+        for (int ks = 0; ks < nks; ++ks, ++gs) {
+          const int s = (int)(gs % S);
+          if (!wait_bar(ctx, BAR(bl.empty + s), (uint32_t)(((gs / S) & 1) ^ 1))) { ok = false; break; }
+          const uint32_t st = base + (uint32_t)s * kStageBytes;
+          if (pt == 0) {
+            mbar_expect_tx(BAR(bl.full + s), kSlabBytes);
+            tma_load_2d(st + kSlabBytes, map, ks * 64, head_row, BAR(bl.full + s));
+          }
+#pragma unroll
+          for (int c8 = 0; c8 < 8; ++c8) {
+            const int col = ks * 64 + c8 * 8;
+            const bool in = col < r;
+            cp_async16(st + row_off + (((uint32_t)c8 ^ sw) << 4), src + (in ? col : 0), in ? 16u : 0u);
+          }
+          cp_async_commit();
+          if (gs >= kLag) { cp_async_wait<kLag>(); fence_proxy_async(); mbar_arrive(BAR(bl.full + (int)((gs - kLag) % S))); }
+        }
+      }
+      ++it;
+    }
+    // drain: the last kLag stages (fewer if less were issued)
+    cp_async_wait<0>();
+    fence_proxy_async();
+    if (ok) {
+      for (long long x = (gs > kLag ? gs - kLag : 0); x < gs; ++x) mbar_arrive(BAR(bl.full + (int)(x % S)));
+    }
+  } else if (warp == 12) {
+    // =============================== MMA issue ===============================
+    constexpr uint32_t idesc = idesc_bf16_f32(128, 128);
+    long long gs = 0;
+    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    bool ok = true;
+    for (long long t = t_begin; t < t_end && ok; ++t) {
+      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
+      if (py != cur_py) { cur_py = py; const long long prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
+      if (ti * kTile >= cnt) continue;
+      const int buf = it & 1;
+      const uint32_t par = (uint32_t)((it >> 1) & 1);
+#pragma unroll 1
+      for (int phase = 0; phase < 2 && ok; ++phase) {
+        const int r = phase ? dev.r_v : dev.r_k;
+        const int nks = (r + 63) >> 6;
+        const uint32_t acc = tmem + (uint32_t)(phase * 256 + buf * 128);
+        if (!wait_bar(ctx, BAR((phase ? bl.vempty : bl.kempty) + buf), par ^ 1u)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll 1
+        for (int ks = 0; ks < nks; ++ks, ++gs) {
+          const int s = (int)(gs % S);
+          if (!wait_bar(ctx, BAR(bl.full + s), (uint32_t)((gs / S) & 1))) { ok = false; break; }
+          tc_fence_after();
+          if (lane == 0) {
+            const uint32_t rows_tile = base + (uint32_t)s * kStageBytes;       // gathered rows of A
+            const uint32_t b_tile = rows_tile + kSlabBytes;                    // slab of the transposed B block
+            const uint32_t a_addr = phase ? b_tile : rows_tile;                // keys: M = rows; values: M = d
+            const uint32_t b_addr = phase ? rows_tile : b_tile;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              if (ks * 64 + kk * 16 < r) {
+                tc_mma_bf16(acc, smem_desc_sw128(a_addr, kk * 32), smem_desc_sw128(b_addr, kk * 32), idesc,
+                            (ks | kk) ? 1u : 0u);
+              }
+            }
+            tc_commit(BAR(bl.empty + s));
+            if (ks == nks - 1) tc_commit(BAR((phase ? bl.vfull : bl.kfull) + buf));
+          }
+          __syncwarp();
+        }
+      }
+      ++it;
+    }
+  } else if (warp < 4) {
+    // =============================== key epilogue: rope, logits, softmax statistics ===============================
+    const int j = tid;                                  // tile row = TMEM lane
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const float scale2 = dev.att_scale * kLog2e;
+    const int rmask = (1 << dev.rope_shift) - 1;
+    float m_run[NR], l_thr[NR];
+    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    long long prob = 0;
+    bool ok = true;
+    uint32_t grp_par = 0;
+    // barrier among the 128 threads of this role, with the same bounded wait as every other wait
+    auto group_sync = [&]() {
+      mbar_arrive(BAR(bl.grp));
+      if (!wait_bar(ctx, BAR(bl.grp), grp_par)) ok = false;
+      grp_par ^= 1u;
+    };
+    auto flush = [&]() {   // end of a segment: write (m, l) of every head to the problem's partial slot
+      float tot[NR];
+#pragma unroll
+      for (int h = 0; h < NR; ++h) {
+        float v = l_thr[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        tot[h] = v;
+      }
+      group_sync();                           // red_s[0] is free (last tile's readers are done)
+      if (lane == 0) {
+#pragma unroll
+        for (int h = 0; h < NR; ++h) red_s[warp * NR + h] = tot[h];
+      }
+      group_sync();
+      if (j < n_rep) {
+        const long long first = (long long)cur_py * sc.tpp;
+        const int seg = (int)blockIdx.x - cta_of_tile(first, C, N);
+        float* part = dev.part + (((size_t)prob * sc.n_slots + seg) * n_rep + j) * (DH + 2);
+        float ls = 0.0f, mm = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < NR; ++h) {
+          if (h == j) { ls = red_s[h] + red_s[NR + h] + red_s[2 * NR + h] + red_s[3 * NR + h]; mm = m_run[h]; }
+        }
+        part[DH] = mm;
+        part[DH + 1] = ls;
+      }
+    };
+    for (long long t = t_begin; t < t_end && ok; ++t) {
+      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
+      if (py != cur_py) {
+        if (cur_py >= 0) flush();
+        cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap);
+#pragma unroll
+        for (int h = 0; h < NR; ++h) { m_run[h] = -INFINITY; l_thr[h] = 0.0f; }
+        const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
+        for (int i = j; i < NR * DH; i += 128) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
+        group_sync();
+      }
+      if (ti * kTile >= cnt) continue;
+      const int buf = it & 1;
+      const uint32_t par = (uint32_t)((it >> 1) & 1);
+      if (!wait_bar(ctx, BAR(bl.kfull + buf), par)) { ok = false; break; }
+      tc_fence_after();
+      const int pos = pos_s[(it & (kPosBufs - 1)) * kTile + j];
+      const int pp = pos < 0 ? 0 : pos;
+      const float2* hi = dev.rope_hi + (pp >> dev.rope_shift);
+      const float2* lo = dev.rope_lo + (pp & rmask);
+      float z[NR];
+#pragma unroll
+      for (int h = 0; h < NR; ++h) z[h] = 0.0f;
+      const uint32_t acc = tmem + lane_base + (uint32_t)(buf * 128);
+#pragma unroll 1
+      for (int pass = 0; pass < HALF / 32; ++pass) {
+        float x1[32], x2[32];
+        tmem_ld32(acc + (uint32_t)(pass * 32), x1);
+        tmem_ld32(acc + (uint32_t)(HALF + pass * 32), x2);
+        tc_wait_ld();
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) {
+          float r1[4], r2[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int ii = pass * 32 + i4 * 4 + e;
+            float cs = 1.0f, sn = 0.0f;
+            if (dev.use_rope) {
+              const float2 a = __ldg(hi + (size_t)ii * dev.n_hi), c2 = __ldg(lo + ((size_t)ii << dev.rope_shift));
+              cs = a.x * c2.x - a.y * c2.y;
+              sn = a.y * c2.x + a.x * c2.y;
+            }
+            const float u = x1[i4 * 4 + e], v = x2[i4 * 4 + e];
+            r1[e] = u * cs - v * sn;
+            r2[e] = v * cs + u * sn;
+          }
+#pragma unroll
+          for (int h = 0; h < NR; ++h) {
+            const float4 qa = *reinterpret_cast<const float4*>(q_s + h * DH + pass * 32 + i4 * 4);
+            const float4 qb = *reinterpret_cast<const float4*>(q_s + h * DH + HALF + pass * 32 + i4 * 4);
+            z[h] = fmaf(qa.x, r1[0], z[h]); z[h] = fmaf(qb.x, r2[0], z[h]);
+            z[h] = fmaf(qa.y, r1[1], z[h]); z[h] = fmaf(qb.y, r2[1], z[h]);
+            z[h] = fmaf(qa.z, r1[2], z[h]); z[h] = fmaf(qb.z, r2[2], z[h]);
+            z[h] = fmaf(qa.w, r1[3], z[h]); z[h] = fmaf(qb.w, r2[3], z[h]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(BAR(bl.kempty + buf));                // accumulator may be overwritten
+      // tile max per head over the 128 rows
+      float tmax[NR];
+#pragma unroll
+      for (int h = 0; h < NR; ++h) {
+        z[h] = pos < 0 ? -INFINITY : z[h] * scale2;
+        float v = z[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+        tmax[h] = v;
+      }
+      float* red = red_s + (it & 1) * 4 * NR;
+      if (lane == 0) {
+#pragma unroll
+        for (int h = 0; h < NR; ++h) red[warp * NR + h] = tmax[h];
+      }
+      group_sync();
+      if (!wait_bar(ctx, BAR(bl.pempty + buf), par ^ 1u)) { ok = false; break; }
+#pragma unroll
+      for (int h = 0; h < NR; ++h) {
+        const float tm = fmaxf(fmaxf(red[h], red[NR + h]), fmaxf(red[2 * NR + h], red[3 * NR + h]));
+        const float m_new = fmaxf(m_run[h], tm);
+        const float alpha = (m_run[h] == -INFINITY) ? 0.0f : exp2f(m_run[h] - m_new);
+        const float p = (m_new == -INFINITY) ? 0.0f : exp2f(z[h] - m_new);
+        l_thr[h] = l_thr[h] * alpha + p;
+        m_run[h] = m_new;
+        P_s[(buf * NR + h) * kTile + j] = p;
+        if (j == h) alpha_s[buf * NR + h] = alpha;
+      }
+      mbar_arrive(BAR(bl.pfull + buf));
+      ++it;
+    }
+    if (ok && cur_py >= 0) flush();
+  } else {
+    // =============================== value epilogue: o += p * V_hat ===============================
+    const int dd = tid - 128;                           // output column = TMEM lane
+    const uint32_t lane_base = (uint32_t)((warp - 4) * 32) << 16;
+    float o[NR];
+    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    long long prob = 0;
+    bool ok = true;
+    auto flush = [&]() {
+      if (dd < DH) {
+        const long long first = (long long)cur_py * sc.tpp;
+        const int seg = (int)blockIdx.x - cta_of_tile(first, C, N);
+        float* part = dev.part + ((size_t)prob * sc.n_slots + seg) * n_rep * (DH + 2);
+#pragma unroll
+        for (int h = 0; h < NR; ++h) if (h < n_rep) part[h * (DH + 2) + dd] = o[h];
+      }
+    };
+    for (long long t = t_begin; t < t_end && ok; ++t) {
+      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
+      if (py != cur_py) {
+        if (cur_py >= 0) flush();
+        cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap);
+#pragma unroll
+        for (int h = 0; h < NR; ++h) o[h] = 0.0f;
+      }
+      if (ti * kTile >= cnt) continue;
+      const int buf = it & 1;
+      const uint32_t par = (uint32_t)((it >> 1) & 1);
+      if (!wait_bar(ctx, BAR(bl.pfull + buf), par)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.vfull + buf), par)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int h = 0; h < NR; ++h) o[h] *= alpha_s[buf * NR + h];
+      const uint32_t acc = tmem + lane_base + (uint32_t)(256 + buf * 128);
+      const float* P = P_s + buf * NR * kTile;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        float v[32];
+        tmem_ld32(acc + (uint32_t)(ch * 32), v);
+        tc_wait_ld();
+#pragma unroll
+        for (int j4 = 0; j4 < 8; ++j4) {
+#pragma unroll
+          for (int h = 0; h < NR; ++h) {
+            const float4 p4 = *reinterpret_cast<const float4*>(P + h * kTile + ch * 32 + j4 * 4);
+            o[h] = fmaf(p4.x, v[j4 * 4 + 0], o[h]);
+            o[h] = fmaf(p4.y, v[j4 * 4 + 1], o[h]);
+            o[h] = fmaf(p4.z, v[j4 * 4 + 2], o[h]);
+            o[h] = fmaf(p4.w, v[j4 * 4 + 3], o[h]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(BAR(bl.vempty + buf));
+      mbar_arrive(BAR(bl.pempty + buf));
+      ++it;
+    }
+    if (ok && cur_py >= 0) flush();
+  }
+
+  // wind down: nothing of this CTA may still touch shared or tensor memory
+  cp_async_wait<0>();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 12) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// Partials of a problem -> out, lse.  grid.x = problems * n_rep, blockDim = DH.  m is in log2 units.
+template <int DH>
+__global__ void __launch_bounds__(DH)
+merge_segments_kernel(GroupDev dev, Sched sc, const int32_t* __restrict__ sel_cnt, __nv_bfloat16* __restrict__ out,
+                      float* __restrict__ lse) {
+  const int n_rep = dev.n_rep;
+  const int h = blockIdx.x % n_rep, py = blockIdx.x / n_rep;
+  const int per_layer = dev.batch * dev.H_kv;
+  const int g = py % dev.H_kv, b = (py / dev.H_kv) % dev.batch, l = sc.l0 + py / per_layer;
+  const long long prob = ((long long)l * dev.batch + b) * dev.H_kv + g;
+  const long long first = (long long)py * sc.tpp;
+  const int c0 = cta_of_tile(first, sc.n_ctas, sc.n_tiles), c1 = cta_of_tile(first + sc.tpp - 1, sc.n_ctas, sc.n_tiles);
+  const int nseg = c1 - c0 + 1;
+  const float* part = dev.part + ((size_t)prob * sc.n_slots) * n_rep * (DH + 2) + (size_t)h * (DH + 2);
+  const size_t stride = (size_t)n_rep * (DH + 2);
+  float M = -INFINITY;
+  for (int s = 0; s < nseg; ++s) M = fmaxf(M, part[s * stride + DH]);
+  float L = 0.0f, o = 0.0f;
+  if (M != -INFINITY) {
+    for (int s = 0; s < nseg; ++s) {
+      const float ms = part[s * stride + DH];
+      if (ms == -INFINITY) continue;
+      const float w = exp2f(ms - M);
+      L += w * part[s * stride + DH + 1];
+      o += w * part[s * stride + threadIdx.x];
+    }
+  }
+  const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
+  out[qh * DH + threadIdx.x] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+  if (lse && threadIdx.x == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
+}
+
+template <int NR>
+size_t fused_smem_bytes(int stages, int DH) {
+  const Bars bl = bar_layout(stages);
+  return 1024 + (size_t)stages * kStageBytes + sizeof(float) * ((size_t)NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) +
+         sizeof(int) * kPosBufs * kTile + 8 * (size_t)bl.total + 16;
+}
+
+template <int DH, int NR>
+cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
+                           const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
+  const GroupDev& dev = grp->dev;
+  const int problems = (l1 - l0) * dev.batch * dev.H_kv;
+  Sched sc;
+  sc.l0 = l0;
+  sc.tpp = (k_cap + kTile - 1) / kTile;
+  sc.n_tiles = problems * sc.tpp;
+  sc.n_ctas = sc.n_tiles < grp->sm_count ? sc.n_tiles : grp->sm_count;
+  sc.n_slots = fused_slots(grp);
+  sc.k_cap = k_cap;
+  int stages = 6;
+  while (stages > 3 && fused_smem_bytes<NR>(stages, DH) > 227 * 1024) --stages;
+  sc.stages = stages;
+  const size_t smem = fused_smem_bytes<NR>(stages, DH);
+  cudaError_t e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  CUtensorMap mk, mv;
+  memcpy(&mk, grp->bk_tmap, sizeof(mk));
+  memcpy(&mv, grp->bv_tmap, sizeof(mv));
+  sr_fused_kernel<DH, NR><<<sc.n_ctas, kThreads, smem, s>>>(mk, mv, dev, sc, q, sel_idx, sel_cnt);
+  count_launch();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  merge_segments_kernel<DH><<<problems * dev.n_rep, DH, 0, s>>>(dev, sc, sel_cnt, out, lse);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int fused_slots(const xkv_group* grp) {
+  const int tpp_max = (grp->k_cap_max + kTile - 1) / kTile;
+  return (tpp_max < grp->sm_count ? tpp_max : grp->sm_count) + 1;
+}
+
+size_t fused_part_floats(const xkv_group* grp) {
+  const xkv_group_config& c = grp->cfg;
+  return (size_t)c.G * c.batch * c.H_kv * fused_slots(grp) * (size_t)(c.H_q / c.H_kv) * (c.d_h + 2);
+}
+
+cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
+                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
+  const int n_rep = grp->dev.n_rep;
+#define XKV_DISPATCH(DH)                                                                              \
+  if (n_rep <= 4) return launch_fused_t<DH, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
+  if (n_rep <= 8) return launch_fused_t<DH, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
+  return launch_fused_t<DH, 16>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);
+  if (grp->dev.d_h == 128) { XKV_DISPATCH(128) }
+  XKV_DISPATCH(64)
+#undef XKV_DISPATCH
+}
+
+}  // namespace xkv

@@ -10,7 +10,6 @@
 namespace xkv {
 
 constexpr int kDP = 128;          // rows of a repacked B head block (d_h padded to 128 with zeros)
-constexpr int kRopeLo = 64;       // positions covered by the fine rotary table
 constexpr int kMaxRep = 16;       // query heads per KV head
 constexpr int kAttTile = 128;     // selected rows per attention tile
 constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, head) problem
@@ -18,7 +17,8 @@ constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, 
 // Device-side description of one window; a copy lives in the handle and is passed by value.
 struct GroupDev {
   int G, batch, T, H_kv, H_q, d_h, r_k, r_v, c, n_c, n_rep;
-  int n_hi;                         // rows of the coarse rotary table: ceil(T / kRopeLo)
+  int rope_shift;                   // fine rotary table covers 2^rope_shift consecutive positions
+  int n_hi;                         // entries per frequency of the coarse table: ceil(T / 2^rope_shift)
   float sel_scale;                  // 1/sqrt(d_h) computed on the host (Algorithm 2, line 2)
   float att_scale;                  // softmax scale of the attention
   int use_rope;
@@ -27,8 +27,8 @@ struct GroupDev {
   const __nv_bfloat16* landmarks;   // [batch][G][H_kv][n_c][d_h]
   const __nv_bfloat16* Bt_k;        // [batch][G][H_kv][kDP][r_k]  transposed head blocks, zero padded
   const __nv_bfloat16* Bt_v;        // [batch][G][H_kv][kDP][r_v]
-  const float2* rope_hi;            // [n_hi][d_h/2]   (cos, sin) of (64*p_hi) * theta_i
-  const float2* rope_lo;            // [kRopeLo][d_h/2] (cos, sin) of p_lo * theta_i
+  const float2* rope_hi;            // [d_h/2][n_hi]          (cos, sin) of (p_hi << rope_shift) * theta_i
+  const float2* rope_lo;            // [d_h/2][2^rope_shift]  (cos, sin) of p_lo * theta_i
   float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
   float* part;                      // attention partials, see xkv_attend.cu
   unsigned int* flags;              // device flag word
@@ -50,6 +50,7 @@ struct xkv_group {
   alignas(64) unsigned char bk_tmap[128];   // CUtensorMap over Bt_k rows
   alignas(64) unsigned char bv_tmap[128];   // CUtensorMap over Bt_v rows
   int has_b_tmap;
+  int attend_impl;                  // 0: tensor-core fused kernel, 1: plain tile kernel
 };
 
 namespace xkv {
@@ -60,7 +61,8 @@ void count_launch(int n = 1);
 // xkv_prep.cu
 cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch, int G, int r, int H_kv,
                             int d_h, cudaStream_t s);
-cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int d_h, double base, cudaStream_t s);
+cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift, int d_h, double base,
+                               cudaStream_t s);
 
 // xkv_select.cu
 cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
@@ -71,5 +73,11 @@ size_t attend_part_floats(const xkv_group* grp);
 cudaError_t launch_reconstruct_attend(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q,
                                       const int32_t* sel_idx, const int32_t* sel_cnt, int k_cap,
                                       __nv_bfloat16* out, float* lse, cudaStream_t s);
+
+// xkv_fused.cu
+int fused_slots(const xkv_group* grp);
+size_t fused_part_floats(const xkv_group* grp);
+cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
+                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s);
 
 }  // namespace xkv

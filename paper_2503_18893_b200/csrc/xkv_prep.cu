@@ -34,25 +34,30 @@ cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch
   return cudaGetLastError();
 }
 
-// theta_i = base^(-2i/d_h); hi[p][i] = (cos, sin)(kRopeLo*p*theta_i), lo[p][i] = (cos, sin)(p*theta_i),
-// evaluated in fp64 so that the product of the two tables carries fp32 rounding only.
-__global__ void rope_tables_kernel(float2* hi, float2* lo, int n_hi, int half, double base) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  const int total = (n_hi + kRopeLo) * half;
+// theta_i = base^(-2i/d_h); position p = (p_hi << shift) + p_lo.  hi[i][p_hi] = (cos, sin)((p_hi << shift) * theta_i),
+// lo[i][p_lo] = (cos, sin)(p_lo * theta_i), evaluated in fp64 so that combining the two by the angle-addition
+// formulas carries fp32 rounding only.  Frequency-major layout: threads that hold consecutive token rows read
+// consecutive table entries.
+__global__ void rope_tables_kernel(float2* hi, float2* lo, int n_hi, int shift, int half, double base) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_lo = 1 << shift;
+  const long long total = (long long)(n_hi + n_lo) * half;
   if (idx >= total) return;
-  const int row = idx / half, i = idx % half;
+  const int i = (int)(idx / (n_hi + n_lo));
+  const int col = (int)(idx % (n_hi + n_lo));
   const double theta = pow(base, -(double)i / (double)half);
-  double p = row < n_hi ? (double)row * (double)kRopeLo : (double)(row - n_hi);
+  const double p = col < n_hi ? (double)((long long)col << shift) : (double)(col - n_hi);
   double sn, cs;
   sincos(p * theta, &sn, &cs);
-  float2 v = make_float2((float)cs, (float)sn);
-  if (row < n_hi) hi[(size_t)row * half + i] = v; else lo[(size_t)(row - n_hi) * half + i] = v;
+  const float2 v = make_float2((float)cs, (float)sn);
+  if (col < n_hi) hi[(size_t)i * n_hi + col] = v; else lo[(size_t)i * n_lo + (col - n_hi)] = v;
 }
 
-cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int d_h, double base, cudaStream_t s) {
+cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift, int d_h, double base,
+                               cudaStream_t s) {
   const int half = d_h / 2;
-  const int total = (n_hi + kRopeLo) * half;
-  rope_tables_kernel<<<(total + 255) / 256, 256, 0, s>>>(hi, lo, n_hi, half, base);
+  const long long total = (long long)(n_hi + (1 << rope_shift)) * half;
+  rope_tables_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(hi, lo, n_hi, rope_shift, half, base);
   count_launch();
   return cudaGetLastError();
 }
