@@ -125,10 +125,10 @@ recon_attend_tile_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__
     // thread (j, part) rotates a quarter of row j in place
     const int j = tid >> 2, part = tid & 3;
     const int p = rows_s[j];
-    const float2* hi = dev.rope_hi + (p >> dev.rope_shift);
-    const float2* lo = dev.rope_lo + (p & ((1 << dev.rope_shift) - 1));
+    const float2* hi = dev.rope_hi + (size_t)(p >> dev.rope_shift) * HALF;
+    const float2* lo = dev.rope_lo + (size_t)(p & ((1 << dev.rope_shift) - 1)) * HALF;
     for (int i = part; i < HALF; i += 4) {
-      const float2 a = hi[(size_t)i * dev.n_hi], c2 = lo[(size_t)i << dev.rope_shift];
+      const float2 a = hi[i], c2 = lo[i];
       const float cs = a.x * c2.x - a.y * c2.y, sn = a.y * c2.x + a.x * c2.y;
       const float x1 = Xs[j * (DH + 1) + i], x2 = Xs[j * (DH + 1) + i + HALF];
       Xs[j * (DH + 1) + i] = x1 * cs - x2 * sn;

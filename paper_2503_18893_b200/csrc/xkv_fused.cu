@@ -26,7 +26,7 @@ constexpr int kSlabBytes = kTile * 128;          // 128 rows x 64 bf16 (one 128-
 constexpr int kStageBytes = 2 * kSlabBytes;      // gathered rows + B slab
 constexpr int kLag = 3;                          // cp.async groups a producer thread keeps in flight
 constexpr int kThreads = 13 * 32;
-constexpr int kPosBufs = 4;
+constexpr int kRopeStride = 66;                  // float2 per staged rotary row (64 + pad against bank conflicts)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -42,12 +42,13 @@ struct Sched {
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, empty, kfull, kempty, vfull, vempty, pfull, pempty, grp, total;
+  int full, empty, kfull, kempty, vfull, vempty, pfull, pempty, rfree, grp, pgrp, total;
 };
 __host__ __device__ inline Bars bar_layout(int stages) {
   Bars b;
   b.full = 0; b.empty = stages; b.kfull = 2 * stages; b.kempty = b.kfull + 2; b.vfull = b.kempty + 2;
-  b.vempty = b.vfull + 2; b.pfull = b.vempty + 2; b.pempty = b.pfull + 2; b.grp = b.pempty + 2; b.total = b.grp + 1;
+  b.vempty = b.vfull + 2; b.pfull = b.vempty + 2; b.pempty = b.pfull + 2; b.rfree = b.pempty + 2;
+  b.grp = b.rfree + 2; b.pgrp = b.grp + 1; b.total = b.pgrp + 1;
   return b;
 }
 
@@ -80,6 +81,60 @@ __device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t pa
   return false;
 }
 
+// Logits of one rebuilt key row against NR query heads: rotate the (i, i+HALF) pairs, accumulate q . k.
+// hi/lo point at this row's coarse/fine rotary entries (cos, sin), in shared (SMEM) or global memory.
+template <int DH, int NR, bool ROPE, bool SMEM>
+__device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restrict__ hi, const float2* __restrict__ lo,
+                                           const float* __restrict__ q_s, float (&z)[NR]) {
+  constexpr int HALF = DH / 2;
+#pragma unroll 1
+  for (int pass = 0; pass < HALF / 32; ++pass) {
+    float x1[32], x2[32];
+    tmem_ld32(acc + (uint32_t)(pass * 32), x1);
+    tmem_ld32(acc + (uint32_t)(HALF + pass * 32), x2);
+    tc_wait_ld();
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+      float r1[4], r2[4];
+      const int ii = pass * 32 + i4 * 4;
+      if (ROPE) {
+        float2 a[4], c2[4];
+        if (SMEM) {
+          const float4 a01 = *reinterpret_cast<const float4*>(hi + ii), a23 = *reinterpret_cast<const float4*>(hi + ii + 2);
+          const float4 c01 = *reinterpret_cast<const float4*>(lo + ii), c23 = *reinterpret_cast<const float4*>(lo + ii + 2);
+          a[0] = make_float2(a01.x, a01.y); a[1] = make_float2(a01.z, a01.w);
+          a[2] = make_float2(a23.x, a23.y); a[3] = make_float2(a23.z, a23.w);
+          c2[0] = make_float2(c01.x, c01.y); c2[1] = make_float2(c01.z, c01.w);
+          c2[2] = make_float2(c23.x, c23.y); c2[3] = make_float2(c23.z, c23.w);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { a[e] = __ldg(hi + ii + e); c2[e] = __ldg(lo + ii + e); }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float cs = a[e].x * c2[e].x - a[e].y * c2[e].y;      // cos(x + y)
+          const float sn = a[e].y * c2[e].x + a[e].x * c2[e].y;      // sin(x + y)
+          const float u = x1[i4 * 4 + e], v = x2[i4 * 4 + e];
+          r1[e] = u * cs - v * sn;
+          r2[e] = v * cs + u * sn;
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { r1[e] = x1[i4 * 4 + e]; r2[e] = x2[i4 * 4 + e]; }
+      }
+#pragma unroll
+      for (int h = 0; h < NR; ++h) {
+        const float4 qa = *reinterpret_cast<const float4*>(q_s + h * DH + ii);
+        const float4 qb = *reinterpret_cast<const float4*>(q_s + h * DH + HALF + ii);
+        z[h] = fmaf(qa.x, r1[0], z[h]); z[h] = fmaf(qb.x, r2[0], z[h]);
+        z[h] = fmaf(qa.y, r1[1], z[h]); z[h] = fmaf(qb.y, r2[1], z[h]);
+        z[h] = fmaf(qa.z, r1[2], z[h]); z[h] = fmaf(qb.z, r2[2], z[h]);
+        z[h] = fmaf(qa.w, r1[3], z[h]); z[h] = fmaf(qb.w, r2[3], z[h]);
+      }
+    }
+  }
+}
+
 template <int DH, int NR>
 __global__ void __launch_bounds__(kThreads, 1)
 sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constant__ CUtensorMap bv_map, GroupDev dev,
@@ -92,18 +147,23 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   const int S = sc.stages;
   // carve-up after the stage ring
-  float* q_s = reinterpret_cast<float*>(gen + (size_t)S * kStageBytes);          // [NR][DH]
+  float2* hi_s = reinterpret_cast<float2*>(gen + (size_t)S * kStageBytes);       // [2][16][kRopeStride] coarse rotary rows
+  float2* lo_s = hi_s + 2 * 16 * kRopeStride;                                    // [8][kRopeStride]     fine rotary rows
+  float* q_s = reinterpret_cast<float*>(lo_s + 8 * kRopeStride);                 // [NR][DH]
   float* P_s = q_s + NR * DH;                                                    // [2][NR][128]
   float* alpha_s = P_s + 2 * NR * kTile;                                         // [2][NR]
   float* red_s = alpha_s + 2 * NR;                                               // [2][4][NR]
-  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [4][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(pos_s + kPosBufs * kTile);
+  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [2][128]
+  int* algn_s = pos_s + 2 * kTile;                                               // [2][4]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(algn_s + 8);
   const Bars bl = bar_layout(S);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + bl.total);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int word) { return bar0 + 8u * (uint32_t)word; };
   Ctx ctx{abort_flag, dev.flags};
+  // the staged rotary path needs the fine table to cover exactly 8 positions
+  const bool rope_smem = dev.use_rope && dev.rope_shift == 3;
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 129); mbar_init(BAR(bl.empty + s), 1); }
@@ -111,10 +171,15 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       mbar_init(BAR(bl.kfull + b), 1); mbar_init(BAR(bl.kempty + b), 128);
       mbar_init(BAR(bl.vfull + b), 1); mbar_init(BAR(bl.vempty + b), 128);
       mbar_init(BAR(bl.pfull + b), 128); mbar_init(BAR(bl.pempty + b), 128);
+      mbar_init(BAR(bl.rfree + b), 128);
     }
     mbar_init(BAR(bl.grp), 128);
+    mbar_init(BAR(bl.pgrp), 128);
     *abort_flag = 0;
     fence_mbar_init();
+  }
+  if (rope_smem) {
+    for (int i = tid; i < 8 * HALF; i += kThreads) lo_s[(i / HALF) * kRopeStride + (i % HALF)] = dev.rope_lo[i];
   }
   if (warp == 12) {
     tmem_alloc(smem_u32(tmem_slot), 512);
@@ -138,29 +203,64 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
 
   if (warp >= 8 && warp < 12) {
     // =============================== producers: gather rows of A, TMA the B slabs ===============================
-    const int pt = tid - 256;
-    const uint32_t row_off = (uint32_t)pt * 128u, sw = (uint32_t)(pt & 7);
+    // Eight consecutive lanes copy the eight 16-byte pieces of one 128-byte row slab, so that every
+    // request of a warp covers whole 128-byte lines; thread pt serves rows (pt>>3) + 16*i, i = 0..7.
+    const int pt = tid - 256, pw = warp - 8;
+    const uint32_t c8 = (uint32_t)(pt & 7);
     long long gs = 0;                 // stages issued so far (ring position)
     int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
     long long prob = 0;
     bool ok = true;
+    uint32_t pg_par = 0;
     for (long long t = t_begin; t < t_end && ok; ++t) {
       const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
       if (py != cur_py) { cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
       const int row0 = ti * kTile;
       if (row0 >= cnt) continue;
+      const int buf = it & 1;
+      // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
+      if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1))) { ok = false; break; }
       int p = -1;
       if (row0 + pt < cnt) {
         p = sel_idx[prob * sc.k_cap + row0 + pt];
         if (p < 0 || p >= dev.T) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
       }
-      pos_s[(it & (kPosBufs - 1)) * kTile + pt] = p;
-      const size_t row = (size_t)b * dev.T + (size_t)(p < 0 ? 0 : p);
+      pos_s[buf * kTile + pt] = p;
+      if (rope_smem) {
+        // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
+        const int hidx = p < 0 ? -1 : (p >> 3);
+        int gmax = hidx;
+        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 4));
+        const bool aligned = __all_sync(0xffffffffu, p < 0 || hidx == gmax);
+        if (lane == 0) algn_s[buf * 4 + pw] = aligned ? 1 : 0;
+        if (aligned) {
+#pragma unroll
+          for (int a = 0; a < 4; ++a) {
+            const int gm = __shfl_sync(0xffffffffu, gmax, a * 8);
+            if (lane * 2 < HALF) {
+              cp_async16(smem_u32(hi_s + (size_t)(buf * 16 + pw * 4 + a) * kRopeStride + lane * 2),
+                         dev.rope_hi + (size_t)(gm < 0 ? 0 : gm) * HALF + lane * 2, 16u);
+            }
+          }
+        }
+      }
+      // make every row position of the tile visible to all producer threads
+      mbar_arrive(BAR(bl.pgrp));
+      if (!wait_bar(ctx, BAR(bl.pgrp), pg_par)) { ok = false; break; }
+      pg_par ^= 1u;
+      long long rowidx[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int pr = pos_s[buf * kTile + i * 16 + (pt >> 3)];
+        rowidx[i] = (long long)b * dev.T + (pr < 0 ? 0 : pr);
+      }
       const int head_row = (int)((((size_t)b * dev.G + l) * dev.H_kv + g) * kDP);
 #pragma unroll 1
       for (int phase = 0; phase < 2 && ok; ++phase) {
         const int r = phase ? dev.r_v : dev.r_k;
-        const __nv_bfloat16* src = (phase ? dev.A_v : dev.A_k) + row * r;
+        const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
         const CUtensorMap* map = phase ? &bv_map : &bk_map;
         const int nks = (r + 63) >> 6;
 #pragma unroll 1
@@ -172,11 +272,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
             mbar_expect_tx(BAR(bl.full + s), kSlabBytes);
             tma_load_2d(st + kSlabBytes, map, ks * 64, head_row, BAR(bl.full + s));
           }
+          const int col = ks * 64 + (int)c8 * 8;
+          const bool in = col < r;
+          const uint32_t nbytes = in ? 16u : 0u;
+          const int ccol = in ? col : 0;
 #pragma unroll
-          for (int c8 = 0; c8 < 8; ++c8) {
-            const int col = ks * 64 + c8 * 8;
-            const bool in = col < r;
-            cp_async16(st + row_off + (((uint32_t)c8 ^ sw) << 4), src + (in ? col : 0), in ? 16u : 0u);
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t R = (uint32_t)(i * 16 + (pt >> 3));
+            cp_async16(st + R * 128u + ((c8 ^ (R & 7u)) << 4), A + rowidx[i] * r + ccol, nbytes);
           }
           cp_async_commit();
           if (gs >= kLag) { cp_async_wait<kLag>(); fence_proxy_async(); mbar_arrive(BAR(bl.full + (int)((gs - kLag) % S))); }
@@ -260,7 +363,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         tot[h] = v;
       }
-      group_sync();                           // red_s[0] is free (last tile's readers are done)
+      group_sync();                                     // red_s[0] is free (last tile's readers are done)
       if (lane == 0) {
 #pragma unroll
         for (int h = 0; h < NR; ++h) red_s[warp * NR + h] = tot[h];
@@ -295,49 +398,24 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       const uint32_t par = (uint32_t)((it >> 1) & 1);
       if (!wait_bar(ctx, BAR(bl.kfull + buf), par)) { ok = false; break; }
       tc_fence_after();
-      const int pos = pos_s[(it & (kPosBufs - 1)) * kTile + j];
+      const int pos = pos_s[buf * kTile + j];
       const int pp = pos < 0 ? 0 : pos;
-      const float2* hi = dev.rope_hi + (pp >> dev.rope_shift);
-      const float2* lo = dev.rope_lo + (pp & rmask);
       float z[NR];
 #pragma unroll
       for (int h = 0; h < NR; ++h) z[h] = 0.0f;
       const uint32_t acc = tmem + lane_base + (uint32_t)(buf * 128);
-#pragma unroll 1
-      for (int pass = 0; pass < HALF / 32; ++pass) {
-        float x1[32], x2[32];
-        tmem_ld32(acc + (uint32_t)(pass * 32), x1);
-        tmem_ld32(acc + (uint32_t)(HALF + pass * 32), x2);
-        tc_wait_ld();
-#pragma unroll
-        for (int i4 = 0; i4 < 8; ++i4) {
-          float r1[4], r2[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int ii = pass * 32 + i4 * 4 + e;
-            float cs = 1.0f, sn = 0.0f;
-            if (dev.use_rope) {
-              const float2 a = __ldg(hi + (size_t)ii * dev.n_hi), c2 = __ldg(lo + ((size_t)ii << dev.rope_shift));
-              cs = a.x * c2.x - a.y * c2.y;
-              sn = a.y * c2.x + a.x * c2.y;
-            }
-            const float u = x1[i4 * 4 + e], v = x2[i4 * 4 + e];
-            r1[e] = u * cs - v * sn;
-            r2[e] = v * cs + u * sn;
-          }
-#pragma unroll
-          for (int h = 0; h < NR; ++h) {
-            const float4 qa = *reinterpret_cast<const float4*>(q_s + h * DH + pass * 32 + i4 * 4);
-            const float4 qb = *reinterpret_cast<const float4*>(q_s + h * DH + HALF + pass * 32 + i4 * 4);
-            z[h] = fmaf(qa.x, r1[0], z[h]); z[h] = fmaf(qb.x, r2[0], z[h]);
-            z[h] = fmaf(qa.y, r1[1], z[h]); z[h] = fmaf(qb.y, r2[1], z[h]);
-            z[h] = fmaf(qa.z, r1[2], z[h]); z[h] = fmaf(qb.z, r2[2], z[h]);
-            z[h] = fmaf(qa.w, r1[3], z[h]); z[h] = fmaf(qb.w, r2[3], z[h]);
-          }
-        }
+      if (!dev.use_rope) {
+        key_logits<DH, NR, false, false>(acc, nullptr, nullptr, q_s, z);
+      } else if (rope_smem && algn_s[buf * 4 + warp]) {
+        key_logits<DH, NR, true, true>(acc, hi_s + (size_t)(buf * 16 + (j >> 3)) * kRopeStride,
+                                       lo_s + (size_t)(pp & 7) * kRopeStride, q_s, z);
+      } else {
+        key_logits<DH, NR, true, false>(acc, dev.rope_hi + (size_t)(pp >> dev.rope_shift) * HALF,
+                                        dev.rope_lo + (size_t)(pp & rmask) * HALF, q_s, z);
       }
       tc_fence_before();
       mbar_arrive(BAR(bl.kempty + buf));                // accumulator may be overwritten
+      mbar_arrive(BAR(bl.rfree + buf));                 // positions and rotary rows of this tile are consumed
       // tile max per head over the 128 rows
       float tmax[NR];
 #pragma unroll
@@ -354,6 +432,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
         for (int h = 0; h < NR; ++h) red[warp * NR + h] = tmax[h];
       }
       group_sync();
+      if (!ok) break;
       if (!wait_bar(ctx, BAR(bl.pempty + buf), par ^ 1u)) { ok = false; break; }
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
@@ -475,8 +554,9 @@ merge_segments_kernel(GroupDev dev, Sched sc, const int32_t* __restrict__ sel_cn
 template <int NR>
 size_t fused_smem_bytes(int stages, int DH) {
   const Bars bl = bar_layout(stages);
-  return 1024 + (size_t)stages * kStageBytes + sizeof(float) * ((size_t)NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) +
-         sizeof(int) * kPosBufs * kTile + 8 * (size_t)bl.total + 16;
+  return 1024 + (size_t)stages * kStageBytes + sizeof(float2) * (size_t)(2 * 16 + 8) * kRopeStride +
+         sizeof(float) * ((size_t)NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) + sizeof(int) * (2 * kTile + 8) +
+         8 * (size_t)bl.total + 16;
 }
 
 template <int DH, int NR>

@@ -27,8 +27,8 @@ struct GroupDev {
   const __nv_bfloat16* landmarks;   // [batch][G][H_kv][n_c][d_h]
   const __nv_bfloat16* Bt_k;        // [batch][G][H_kv][kDP][r_k]  transposed head blocks, zero padded
   const __nv_bfloat16* Bt_v;        // [batch][G][H_kv][kDP][r_v]
-  const float2* rope_hi;            // [d_h/2][n_hi]          (cos, sin) of (p_hi << rope_shift) * theta_i
-  const float2* rope_lo;            // [d_h/2][2^rope_shift]  (cos, sin) of p_lo * theta_i
+  const float2* rope_hi;            // [n_hi][d_h/2]          (cos, sin) of (p_hi << rope_shift) * theta_i
+  const float2* rope_lo;            // [2^rope_shift][d_h/2]  (cos, sin) of p_lo * theta_i
   float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
   float* part;                      // attention partials, see xkv_attend.cu
   unsigned int* flags;              // device flag word

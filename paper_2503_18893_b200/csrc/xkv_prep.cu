@@ -34,23 +34,22 @@ cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch
   return cudaGetLastError();
 }
 
-// theta_i = base^(-2i/d_h); position p = (p_hi << shift) + p_lo.  hi[i][p_hi] = (cos, sin)((p_hi << shift) * theta_i),
-// lo[i][p_lo] = (cos, sin)(p_lo * theta_i), evaluated in fp64 so that combining the two by the angle-addition
-// formulas carries fp32 rounding only.  Frequency-major layout: threads that hold consecutive token rows read
-// consecutive table entries.
+// theta_i = base^(-2i/d_h); position p = (p_hi << shift) + p_lo.  hi[p_hi][i] = (cos, sin)((p_hi << shift) * theta_i),
+// lo[p_lo][i] = (cos, sin)(p_lo * theta_i), evaluated in fp64 so that combining the two by the angle-addition
+// formulas carries fp32 rounding only.  Position-major layout: the d_h/2 entries of one position are contiguous.
 __global__ void rope_tables_kernel(float2* hi, float2* lo, int n_hi, int shift, int half, double base) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int n_lo = 1 << shift;
   const long long total = (long long)(n_hi + n_lo) * half;
   if (idx >= total) return;
-  const int i = (int)(idx / (n_hi + n_lo));
-  const int col = (int)(idx % (n_hi + n_lo));
+  const int col = (int)(idx / half);
+  const int i = (int)(idx % half);
   const double theta = pow(base, -(double)i / (double)half);
   const double p = col < n_hi ? (double)((long long)col << shift) : (double)(col - n_hi);
   double sn, cs;
   sincos(p * theta, &sn, &cs);
   const float2 v = make_float2((float)cs, (float)sn);
-  if (col < n_hi) hi[(size_t)i * n_hi + col] = v; else lo[(size_t)i * n_lo + (col - n_hi)] = v;
+  if (col < n_hi) hi[(size_t)col * half + i] = v; else lo[(size_t)(col - n_hi) * half + i] = v;
 }
 
 cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift, int d_h, double base,
