@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--T", type=int, default=None)
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--r", type=int, default=None)
+    ap.add_argument("--r-k", type=int, default=None)
+    ap.add_argument("--r-v", type=int, default=None)
+    ap.add_argument("--rope-base", type=float, default=None)
     ap.add_argument("--groups", type=int, default=None, help="number of windows (default: the config's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-problems", type=int, default=None, help="oracle sample size in (layer,head) problems")
@@ -55,6 +58,9 @@ def make_shape(args):
     if args.T is not None: over["T"] = args.T
     if args.k is not None: over["k"] = args.k
     if args.r is not None: over["r_k"] = over["r_v"] = args.r
+    if args.r_k is not None: over["r_k"] = args.r_k
+    if args.r_v is not None: over["r_v"] = args.r_v
+    if args.rope_base is not None: over["rope_base"] = args.rope_base
     if args.groups is not None: over["n_groups"] = args.groups
     return synth.config(args.config, **over)
 

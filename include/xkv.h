@@ -161,6 +161,15 @@ XKV_API int xkv_last_cuda_error(void);
 /* Number of kernels the library has launched since load (all handles); for launch accounting. */
 XKV_API uint64_t xkv_kernel_launch_count(void);
 
+/*
+ * Diagnostic.  If the environment variable XKV_FUSED_PROF=1 was set when the handle was created, the
+ * reconstruct+attend kernel adds, per CTA, the cycles each warp role spent waiting on each of its
+ * hand-offs (64 counters per CTA; the layout is documented beside the kernel).  Synchronises the device,
+ * copies up to max_words counters to `out` (host) and clears them.  Returns the number of words copied,
+ * XKV_ERR_UNSUPPORTED if profiling was not requested, or another negative status.
+ */
+XKV_API int xkv_debug_read_profile(xkv_group* grp, uint64_t* out, int max_words);
+
 #ifdef __cplusplus
 }
 #endif

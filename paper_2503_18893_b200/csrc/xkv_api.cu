@@ -195,6 +195,13 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     {
       const char* e = getenv("XKV_ATTEND_IMPL");
       g->attend_impl = (e && e[0] == 't') ? 1 : 0;
+      const char* pe = getenv("XKV_FUSED_PROF");
+      if (pe && pe[0] == '1') {
+        XKV_TRY_CUDA(cudaMalloc(&p, (size_t)g->sm_count * 64 * sizeof(unsigned long long)));
+        g->owned[g->n_owned++] = p;
+        g->prof = (unsigned long long*)p;
+        XKV_TRY_CUDA(cudaMemset(p, 0, (size_t)g->sm_count * 64 * sizeof(unsigned long long)));
+      }
     }
   }
   *out = g;
@@ -233,6 +240,18 @@ int xkv_group_status(xkv_group* g, uint32_t* device_flags, void* stream) {
   if (f & XKV_FLAG_TIMEOUT) return XKV_ERR_TIMEOUT;
   if (f & XKV_FLAG_INDEX_RANGE) return XKV_ERR_INDEX_RANGE;
   return XKV_OK;
+}
+
+int xkv_debug_read_profile(xkv_group* g, uint64_t* out, int max_words) {
+  if (!g || !out || max_words < 0) return XKV_ERR_INVALID_ARG;
+  if (!g->prof) return XKV_ERR_UNSUPPORTED;
+  size_t n = (size_t)g->sm_count * 64;
+  if ((size_t)max_words < n) n = (size_t)max_words;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(out, g->prof, n * sizeof(uint64_t), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemset(g->prof, 0, (size_t)g->sm_count * 64 * sizeof(uint64_t));
+  if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+  return (int)n;
 }
 
 int xkv_sr_select(xkv_group* g, int layer_begin, int layer_end, const void* q, int32_t k, int32_t* sel_idx,

@@ -8,7 +8,8 @@
 //   V_hat^T [d][j] = sum_m B_v[m][d] * A_v[S_t[j]][m]     tcgen05.mma, M = d_h, N = rows
 //   o[h][d] += sum_j p[h][j] * V_hat^T[d][j]                thread d owns TMEM lane d; online softmax
 // Rebuilt K/V never leave the SM.  Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-11 gather
-// producers (cp.async of the selected rows, TMA of the B slabs), 12 MMA issue.
+// producers (cp.async of the selected rows into a deep ring), 12 MMA issue, 13 TMA loader of the B slabs
+// (a short ring of its own: those come from L2 and need little lead).
 // Every wait is bounded; a wait that runs out raises XKV_FLAG_TIMEOUT and the CTA winds down.
 #include <cuda.h>
 
@@ -23,9 +24,9 @@ using namespace ptx;
 
 constexpr int kTile = 128;                       // selected rows per tile
 constexpr int kSlabBytes = kTile * 128;          // 128 rows x 64 bf16 (one 128-byte swizzle row each)
-constexpr int kStageBytes = 2 * kSlabBytes;      // gathered rows + B slab
-constexpr int kLag = 3;                          // cp.async groups a producer thread keeps in flight
-constexpr int kThreads = 13 * 32;
+constexpr int kNB = 4;                           // slots of the B-slab ring
+constexpr int kThreads = 14 * 32;
+constexpr int kSmemLimit = 227 * 1024;
 constexpr int kRopeStride = 66;                  // float2 per staged rotary row (64 + pad against bank conflicts)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kLog2e = 1.4426950408889634f;
@@ -38,17 +39,18 @@ struct Sched {
   int n_ctas;
   int n_slots;       // partial slots per problem
   int k_cap;
-  int stages;
+  unsigned long long* prof;   // diagnostic counters [n_ctas][64] or nullptr
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, empty, kfull, kempty, vfull, vempty, pfull, pempty, rfree, grp, pgrp, total;
+  int full, empty, bfull, kfull, kempty, vfull, vempty, pfull, pempty, rfree, posfull, grp, total;
 };
-__host__ __device__ inline Bars bar_layout(int stages) {
-  Bars b;
-  b.full = 0; b.empty = stages; b.kfull = 2 * stages; b.kempty = b.kfull + 2; b.vfull = b.kempty + 2;
+__host__ __device__ constexpr Bars bar_layout(int na) {
+  Bars b{};
+  b.full = 0; b.empty = na; b.bfull = na + na / 2; b.kfull = b.bfull + kNB;   // `empty` holds one barrier per slot pair
+  b.kempty = b.kfull + 2; b.vfull = b.kempty + 2;
   b.vempty = b.vfull + 2; b.pfull = b.vempty + 2; b.pempty = b.pfull + 2; b.rfree = b.pempty + 2;
-  b.grp = b.rfree + 2; b.pgrp = b.grp + 1; b.total = b.pgrp + 1;
+  b.posfull = b.rfree + 2; b.grp = b.posfull + 2; b.total = b.grp + 1;
   return b;
 }
 
@@ -58,6 +60,7 @@ __device__ __forceinline__ int cta_of_tile(long long t, int C, int N) { return (
 struct Ctx {
   volatile int* abort;
   unsigned int* flags;
+  unsigned long long* prof;   // per-CTA diagnostic counters (cycles), nullptr unless profiling was requested
 };
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -66,7 +69,16 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait on an mbarrier phase.  Returns false if another thread of the CTA has given up, or if the
 // phase does not complete within kWaitLimitNs (then this thread raises the flag and makes the others give up).
-__device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity);
+// `slot` >= 0 (passed warp-uniformly by one warp per role when diagnostics are on) adds the cycles waited.
+__device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity, int slot = -1) {
+  if (c.prof == nullptr || slot < 0) return wait_bar_raw(c, bar, parity);
+  const long long c0 = clock64();
+  const bool r = wait_bar_raw(c, bar, parity);
+  if ((threadIdx.x & 31) == 0) atomicAdd(c.prof + slot, (unsigned long long)(clock64() - c0));
+  return r;
+}
+__device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t i = 1;; ++i) {
@@ -135,6 +147,18 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
   }
 }
 
+// Shared memory besides the two rings: rotary rows, queries, softmax weights, positions, barriers.
+template <int DH, int NR>
+__host__ __device__ constexpr int misc_smem_bytes() {
+  return (int)(sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) +
+               sizeof(int) * (2 * kTile + 8) + 8 * (2 * 16 + 2 * kNB + 20) + 16);
+}
+// Slots of the gathered-row ring: whatever fits beside the B ring.
+template <int DH, int NR>
+__host__ __device__ constexpr int ring_slots() {
+  return ((kSmemLimit - 1024 - misc_smem_bytes<DH, NR>() - kNB * kSlabBytes) / kSlabBytes) & ~1;   // even: released in pairs
+}
+
 template <int DH, int NR>
 __global__ void __launch_bounds__(kThreads, 1)
 sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constant__ CUtensorMap bv_map, GroupDev dev,
@@ -145,9 +169,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  const int S = sc.stages;
-  // carve-up after the stage ring
-  float2* hi_s = reinterpret_cast<float2*>(gen + (size_t)S * kStageBytes);       // [2][16][kRopeStride] coarse rotary rows
+  constexpr int S = ring_slots<DH, NR>();          // gathered-row slots, all of which may be in flight
+  static_assert(S >= 4 && S <= 16, "ring size");
+  const uint32_t bring = base + (uint32_t)S * kSlabBytes;                         // B-slab ring
+  // carve-up after the two rings
+  float2* hi_s = reinterpret_cast<float2*>(gen + (size_t)(S + kNB) * kSlabBytes); // [2][16][kRopeStride] coarse rotary rows
   float2* lo_s = hi_s + 2 * 16 * kRopeStride;                                    // [8][kRopeStride]     fine rotary rows
   float* q_s = reinterpret_cast<float*>(lo_s + 8 * kRopeStride);                 // [NR][DH]
   float* P_s = q_s + NR * DH;                                                    // [2][NR][128]
@@ -156,25 +182,26 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [2][128]
   int* algn_s = pos_s + 2 * kTile;                                               // [2][4]
   uint64_t* bars = reinterpret_cast<uint64_t*>(algn_s + 8);
-  const Bars bl = bar_layout(S);
+  constexpr Bars bl = bar_layout(S);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + bl.total);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int word) { return bar0 + 8u * (uint32_t)word; };
-  Ctx ctx{abort_flag, dev.flags};
+  Ctx ctx{abort_flag, dev.flags, sc.prof ? sc.prof + (size_t)blockIdx.x * 64 : nullptr};
   // the staged rotary path needs the fine table to cover exactly 8 positions
   const bool rope_smem = dev.use_rope && dev.rope_shift == 3;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 129); mbar_init(BAR(bl.empty + s), 1); }
+    for (int s = 0; s < S; ++s) mbar_init(BAR(bl.full + s), 128);
+    for (int s = 0; s < S / 2; ++s) mbar_init(BAR(bl.empty + s), 1);
+    for (int s = 0; s < kNB; ++s) mbar_init(BAR(bl.bfull + s), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(BAR(bl.kfull + b), 1); mbar_init(BAR(bl.kempty + b), 128);
       mbar_init(BAR(bl.vfull + b), 1); mbar_init(BAR(bl.vempty + b), 128);
       mbar_init(BAR(bl.pfull + b), 128); mbar_init(BAR(bl.pempty + b), 128);
-      mbar_init(BAR(bl.rfree + b), 128);
+      mbar_init(BAR(bl.rfree + b), 128); mbar_init(BAR(bl.posfull + b), 128);
     }
     mbar_init(BAR(bl.grp), 128);
-    mbar_init(BAR(bl.pgrp), 128);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -201,30 +228,64 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
     return ((long long)l * dev.batch + b) * dev.H_kv + g;
   };
 
+  // Walks this CTA's tiles, skipping tiles that start at or beyond the problem's row count.
+  struct TileIter {
+    long long t; int py, ti, cnt, l, b, g; long long prob; bool fresh;   // fresh: first visited tile of its problem
+  };
+  auto iter_begin = [&](TileIter& it_) { it_.t = t_begin - 1; it_.py = -1; it_.cnt = 0; it_.fresh = false; };
+  // advance to the next non-empty tile; returns false at the end of the range.  `on_problem(py)` runs whenever
+  // the walk enters a new problem (also for problems whose tiles are all empty), before its tiles.
+  auto iter_next = [&](TileIter& it_, auto&& on_problem) -> bool {
+    for (;;) {
+      ++it_.t;
+      if (it_.t >= t_end) return false;
+      const int py = (int)(it_.t / sc.tpp);
+      it_.ti = (int)(it_.t % sc.tpp);
+      if (py != it_.py) {
+        on_problem(py);
+        it_.py = py;
+        it_.prob = prob_of(py, it_.l, it_.b, it_.g);
+        it_.cnt = min(sel_cnt[it_.prob], sc.k_cap);
+      }
+      if (it_.ti * kTile < it_.cnt) return true;
+    }
+  };
+  auto no_op = [](int) {};
+
   if (warp >= 8 && warp < 12) {
     // =============================== producers: gather rows of A, TMA the B slabs ===============================
     // Eight consecutive lanes copy the eight 16-byte pieces of one 128-byte row slab, so that every
     // request of a warp covers whole 128-byte lines; thread pt serves rows (pt>>3) + 16*i, i = 0..7.
     const int pt = tid - 256, pw = warp - 8;
     const uint32_t c8 = (uint32_t)(pt & 7);
-    long long gs = 0;                 // stages issued so far (ring position)
-    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
-    long long prob = 0;
+    int slot = 0;                     // ring position and the parity of its current round
+    uint32_t ring_par = 0;
+    // rows (pt>>3) + 16*i share the swizzle phase (pt>>3)&7; slot-relative destination of the i = 0 piece
+    const uint32_t dst0 = (uint32_t)(pt >> 3) * 128u + ((c8 ^ ((uint32_t)(pt >> 3) & 7u)) << 4);
+    const int ps = pw == 0 ? 0 : -1000;
+    const long long role_t0 = clock64();
+    int it = 0;
     bool ok = true;
-    uint32_t pg_par = 0;
-    for (long long t = t_begin; t < t_end && ok; ++t) {
-      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
-      if (py != cur_py) { cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
-      const int row0 = ti * kTile;
-      if (row0 >= cnt) continue;
-      const int buf = it & 1;
-      // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
-      if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1))) { ok = false; break; }
+    TileIter cur, nxt;
+    iter_begin(nxt);
+    bool have = iter_next(nxt, no_op);
+    auto load_pos = [&](const TileIter& x) {
       int p = -1;
-      if (row0 + pt < cnt) {
-        p = sel_idx[prob * sc.k_cap + row0 + pt];
+      if (x.ti * kTile + pt < x.cnt) {
+        p = sel_idx[x.prob * sc.k_cap + x.ti * kTile + pt];
         if (p < 0 || p >= dev.T) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
       }
+      return p;
+    };
+    int p_next = have ? load_pos(nxt) : -1;   // row index of the next tile, fetched one tile ahead
+    while (have && ok) {
+      cur = nxt;
+      const int p = p_next;
+      have = iter_next(nxt, no_op);
+      if (have) p_next = load_pos(nxt);
+      const int buf = it & 1;
+      // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
+      if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
       pos_s[buf * kTile + pt] = p;
       if (rope_smem) {
         // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
@@ -246,59 +307,55 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
           }
         }
       }
-      // make every row position of the tile visible to all producer threads
-      mbar_arrive(BAR(bl.pgrp));
-      if (!wait_bar(ctx, BAR(bl.pgrp), pg_par)) { ok = false; break; }
-      pg_par ^= 1u;
+      // publish the row positions of the tile (to the other producer threads and to the key epilogue)
+      mbar_arrive(BAR(bl.posfull + buf));
+      if (!wait_bar(ctx, BAR(bl.posfull + buf), (uint32_t)((it >> 1) & 1), ps + 2)) { ok = false; break; }
       long long rowidx[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int pr = pos_s[buf * kTile + i * 16 + (pt >> 3)];
-        rowidx[i] = (long long)b * dev.T + (pr < 0 ? 0 : pr);
+        rowidx[i] = (long long)cur.b * dev.T + (pr < 0 ? 0 : pr);
       }
-      const int head_row = (int)((((size_t)b * dev.G + l) * dev.H_kv + g) * kDP);
 #pragma unroll 1
       for (int phase = 0; phase < 2 && ok; ++phase) {
         const int r = phase ? dev.r_v : dev.r_k;
         const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
-        const CUtensorMap* map = phase ? &bv_map : &bk_map;
         const int nks = (r + 63) >> 6;
-#pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks, ++gs) {
-          const int s = (int)(gs % S);
-          if (!wait_bar(ctx, BAR(bl.empty + s), (uint32_t)(((gs / S) & 1) ^ 1))) { ok = false; break; }
-          const uint32_t st = base + (uint32_t)s * kStageBytes;
-          if (pt == 0) {
-            mbar_expect_tx(BAR(bl.full + s), kSlabBytes);
-            tma_load_2d(st + kSlabBytes, map, ks * 64, head_row, BAR(bl.full + s));
-          }
-          const int col = ks * 64 + (int)c8 * 8;
-          const bool in = col < r;
-          const uint32_t nbytes = in ? 16u : 0u;
-          const int ccol = in ? col : 0;
+        const __nv_bfloat16* rp[8];                    // this thread's piece of each of its eight rows
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint32_t R = (uint32_t)(i * 16 + (pt >> 3));
-            cp_async16(st + R * 128u + ((c8 ^ (R & 7u)) << 4), A + rowidx[i] * r + ccol, nbytes);
-          }
-          cp_async_commit();
-          if (gs >= kLag) { cp_async_wait<kLag>(); fence_proxy_async(); mbar_arrive(BAR(bl.full + (int)((gs - kLag) % S))); }
+        for (int i = 0; i < 8; ++i) rp[i] = A + rowidx[i] * r + (int)c8 * 8;
+#pragma unroll 1
+        for (int ks = 0; ks < nks; ++ks) {
+          // slots are released in pairs (one tcgen05.commit per two slabs): wait when entering a pair
+          if ((slot & 1) == 0 && !wait_bar(ctx, BAR(bl.empty + (slot >> 1)), ring_par ^ 1u, ps + 3)) { ok = false; break; }
+          const uint32_t st = base + (uint32_t)slot * kSlabBytes + dst0;
+          const bool in = ks * 64 + (int)c8 * 8 < r;   // false only in a ragged last slab: zero-fill
+          const uint32_t nbytes = in ? 16u : 0u;
+          const int adv = in ? ks * 64 : 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
+          cp_async_arrive_noinc(BAR(bl.full + slot));  // arrives when this thread's copies have landed
+          if (++slot == S) { slot = 0; ring_par ^= 1u; }
         }
       }
       ++it;
     }
-    // drain: the last kLag stages (fewer if less were issued)
-    cp_async_wait<0>();
-    fence_proxy_async();
-    if (ok) {
-      for (long long x = (gs > kLag ? gs - kLag : 0); x < gs; ++x) mbar_arrive(BAR(bl.full + (int)(x % S)));
-    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (ctx.prof && pt == 0) { ctx.prof[0] = (unsigned long long)(clock64() - role_t0); ctx.prof[4] = (unsigned long long)it; }
   } else if (warp == 12) {
     // =============================== MMA issue ===============================
     constexpr uint32_t idesc = idesc_bf16_f32(128, 128);
-    long long gs = 0;
+    const int ps = 8;
+    const long long role_t0 = clock64();
+    int slot = 0, bslot = 0;                          // positions in the two rings and their round parities
+    uint32_t ring_par = 0, bring_par = 0;
+    // descriptors differ between slots only in the start-address field (units of 16 bytes)
+    const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
+    const uint32_t rows_lo0 = (uint32_t)(smem_desc_sw128(base, 0) & 0xFFFFFFFFull);
+    const uint32_t b_lo0 = (uint32_t)(smem_desc_sw128(bring, 0) & 0xFFFFFFFFull);
     int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
     bool ok = true;
+    // the whole warp walks the loop (all values are warp-uniform); one lane issues the tensor-core instructions
     for (long long t = t_begin; t < t_end && ok; ++t) {
       const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
       if (py != cur_py) { cur_py = py; const long long prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
@@ -309,33 +366,70 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       for (int phase = 0; phase < 2 && ok; ++phase) {
         const int r = phase ? dev.r_v : dev.r_k;
         const int nks = (r + 63) >> 6;
+        const int last_kk = (((r - 1) & 63) >> 4) + 1;          // 16-column steps in the last slab
         const uint32_t acc = tmem + (uint32_t)(phase * 256 + buf * 128);
-        if (!wait_bar(ctx, BAR((phase ? bl.vempty : bl.kempty) + buf), par ^ 1u)) { ok = false; break; }
+        if (!wait_bar(ctx, BAR((phase ? bl.vempty : bl.kempty) + buf), par ^ 1u, ps + 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks, ++gs) {
-          const int s = (int)(gs % S);
-          if (!wait_bar(ctx, BAR(bl.full + s), (uint32_t)((gs / S) & 1))) { ok = false; break; }
+        for (int ks = 0; ks < nks; ++ks) {
+          if (!wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
+          if (!wait_bar(ctx, BAR(bl.full + slot), ring_par, ps + 3)) { ok = false; break; }
           tc_fence_after();
+          const long long i0 = ctx.prof ? clock64() : 0;
           if (lane == 0) {
-            const uint32_t rows_tile = base + (uint32_t)s * kStageBytes;       // gathered rows of A
-            const uint32_t b_tile = rows_tile + kSlabBytes;                    // slab of the transposed B block
-            const uint32_t a_addr = phase ? b_tile : rows_tile;                // keys: M = rows; values: M = d
-            const uint32_t b_addr = phase ? rows_tile : b_tile;
+            const uint32_t rows_lo = rows_lo0 + (uint32_t)slot * (kSlabBytes >> 4);   // gathered rows of A
+            const uint32_t b_lo = b_lo0 + (uint32_t)bslot * (kSlabBytes >> 4);        // slab of the transposed B block
+            const uint64_t a_desc = desc_hi | (phase ? b_lo : rows_lo);               // keys: M = rows; values: M = d
+            const uint64_t b_desc = desc_hi | (phase ? rows_lo : b_lo);
+            const int nkk = (ks == nks - 1) ? last_kk : 4;
+            tc_mma_bf16(acc, a_desc, b_desc, idesc, ks ? 1u : 0u);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              if (ks * 64 + kk * 16 < r) {
-                tc_mma_bf16(acc, smem_desc_sw128(a_addr, kk * 32), smem_desc_sw128(b_addr, kk * 32), idesc,
-                            (ks | kk) ? 1u : 0u);
-              }
+            for (int kk = 1; kk < 4; ++kk) {
+              if (kk < nkk) tc_mma_bf16(acc, a_desc + 2u * kk, b_desc + 2u * kk, idesc, 1u);   // +32 bytes per step
             }
-            tc_commit(BAR(bl.empty + s));
+            if (slot & 1) tc_commit(BAR(bl.empty + (slot >> 1)));   // releases both slabs of the pair (and their B slabs)
             if (ks == nks - 1) tc_commit(BAR((phase ? bl.vfull : bl.kfull) + buf));
           }
           __syncwarp();
+          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + 12, (unsigned long long)(clock64() - i0));
+          if (++slot == S) { slot = 0; ring_par ^= 1u; }
+          if (++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
       }
       ++it;
+    }
+    if (ctx.prof && lane == 0) ctx.prof[8] = (unsigned long long)(clock64() - role_t0);
+    __syncwarp();
+  } else if (warp == 13) {
+    // =============================== B-slab loader (TMA) ===============================
+    // B slab of stage n goes to slot n % kNB.  That slot held stage n - kNB, whose MMAs are known to be complete
+    // when the row-ring pair of stage n - kNB has been released; the loader follows that stage's ring position.
+    int bslot = 0, n_issued = 0, xslot = 0;
+    uint32_t xpar = 0;
+    int cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    bool ok = true;
+    for (long long t = t_begin; t < t_end && ok && lane == 0; ++t) {
+      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
+      if (py != cur_py) { cur_py = py; const long long prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
+      if (ti * kTile >= cnt) continue;
+      const int head_row = (int)((((size_t)b * dev.G + l) * dev.H_kv + g) * kDP);
+#pragma unroll 1
+      for (int phase = 0; phase < 2 && ok; ++phase) {
+        const int r = phase ? dev.r_v : dev.r_k;
+        const CUtensorMap* map = phase ? &bv_map : &bk_map;
+        const int nks = (r + 63) >> 6;
+#pragma unroll 1
+        for (int ks = 0; ks < nks; ++ks) {
+          if (n_issued >= kNB) {
+            if (!wait_bar(ctx, BAR(bl.empty + (xslot >> 1)), xpar, 17)) { ok = false; break; }
+            if (++xslot == S) { xslot = 0; xpar ^= 1u; }
+          }
+          ++n_issued;
+          mbar_expect_tx(BAR(bl.bfull + bslot), kSlabBytes);
+          tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, map, ks * 64, head_row, BAR(bl.bfull + bslot));
+          if (++bslot == kNB) bslot = 0;
+        }
+      }
     }
   } else if (warp < 4) {
     // =============================== key epilogue: rope, logits, softmax statistics ===============================
@@ -348,10 +442,12 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
     long long prob = 0;
     bool ok = true;
     uint32_t grp_par = 0;
+    const int ps = warp == 0 ? 24 : -1000;
+    const long long role_t0 = clock64();
     // barrier among the 128 threads of this role, with the same bounded wait as every other wait
     auto group_sync = [&]() {
       mbar_arrive(BAR(bl.grp));
-      if (!wait_bar(ctx, BAR(bl.grp), grp_par)) ok = false;
+      if (!wait_bar(ctx, BAR(bl.grp), grp_par, ps + 3)) ok = false;
       grp_par ^= 1u;
     };
     auto flush = [&]() {   // end of a segment: write (m, l) of every head to the problem's partial slot
@@ -396,7 +492,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       if (ti * kTile >= cnt) continue;
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
-      if (!wait_bar(ctx, BAR(bl.kfull + buf), par)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.posfull + buf), par, ps + 1)) { ok = false; break; }   // positions published
+      if (!wait_bar(ctx, BAR(bl.kfull + buf), par, ps + 2)) { ok = false; break; }
       tc_fence_after();
       const int pos = pos_s[buf * kTile + j];
       const int pp = pos < 0 ? 0 : pos;
@@ -433,7 +530,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       }
       group_sync();
       if (!ok) break;
-      if (!wait_bar(ctx, BAR(bl.pempty + buf), par ^ 1u)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.pempty + buf), par ^ 1u, ps + 4)) { ok = false; break; }
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
         const float tm = fmaxf(fmaxf(red[h], red[NR + h]), fmaxf(red[2 * NR + h], red[3 * NR + h]));
@@ -449,11 +546,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       ++it;
     }
     if (ok && cur_py >= 0) flush();
+    if (ctx.prof && j == 0) ctx.prof[24] = (unsigned long long)(clock64() - role_t0);
   } else {
     // =============================== value epilogue: o += p * V_hat ===============================
     const int dd = tid - 128;                           // output column = TMEM lane
     const uint32_t lane_base = (uint32_t)((warp - 4) * 32) << 16;
     float o[NR];
+    const int ps = warp == 4 ? 32 : -1000;
+    const long long role_t0 = clock64();
     int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
     long long prob = 0;
     bool ok = true;
@@ -477,8 +577,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       if (ti * kTile >= cnt) continue;
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
-      if (!wait_bar(ctx, BAR(bl.pfull + buf), par)) { ok = false; break; }
-      if (!wait_bar(ctx, BAR(bl.vfull + buf), par)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.pfull + buf), par, ps + 1)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.vfull + buf), par, ps + 2)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll
       for (int h = 0; h < NR; ++h) o[h] *= alpha_s[buf * NR + h];
@@ -507,10 +607,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       ++it;
     }
     if (ok && cur_py >= 0) flush();
+    if (ctx.prof && dd == 0) ctx.prof[32] = (unsigned long long)(clock64() - role_t0);
   }
 
   // wind down: nothing of this CTA may still touch shared or tensor memory
-  cp_async_wait<0>();
+  asm volatile("cp.async.wait_all;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   if (warp == 12) {
@@ -551,12 +652,9 @@ merge_segments_kernel(GroupDev dev, Sched sc, const int32_t* __restrict__ sel_cn
   if (lse && threadIdx.x == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
 }
 
-template <int NR>
-size_t fused_smem_bytes(int stages, int DH) {
-  const Bars bl = bar_layout(stages);
-  return 1024 + (size_t)stages * kStageBytes + sizeof(float2) * (size_t)(2 * 16 + 8) * kRopeStride +
-         sizeof(float) * ((size_t)NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) + sizeof(int) * (2 * kTile + 8) +
-         8 * (size_t)bl.total + 16;
+template <int DH, int NR>
+constexpr size_t fused_smem_bytes() {
+  return 1024 + (size_t)(ring_slots<DH, NR>() + kNB) * kSlabBytes + misc_smem_bytes<DH, NR>();
 }
 
 template <int DH, int NR>
@@ -571,10 +669,10 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   sc.n_ctas = sc.n_tiles < grp->sm_count ? sc.n_tiles : grp->sm_count;
   sc.n_slots = fused_slots(grp);
   sc.k_cap = k_cap;
-  int stages = 6;
-  while (stages > 3 && fused_smem_bytes<NR>(stages, DH) > 227 * 1024) --stages;
-  sc.stages = stages;
-  const size_t smem = fused_smem_bytes<NR>(stages, DH);
+  sc.prof = grp->prof;
+  static_assert(bar_layout(ring_slots<DH, NR>()).total <= 2 * 16 + 2 * kNB + 20, "barrier space");
+  static_assert(kNB >= 2 && kNB < ring_slots<DH, NR>(), "B ring must be shorter than the row ring");
+  const size_t smem = fused_smem_bytes<DH, NR>();
   cudaError_t e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   CUtensorMap mk, mv;

@@ -43,13 +43,14 @@ struct xkv_group {
   int sm_count;
   int k_cap_max;                    // ceil(k_max/c)*c
   size_t workspace_bytes;
-  void* owned[8];
+  void* owned[12];
   int n_owned;
   alignas(64) unsigned char lm_tmap[128];   // CUtensorMap for the landmark scan
   int has_lm_tmap;
   alignas(64) unsigned char bk_tmap[128];   // CUtensorMap over Bt_k rows
   alignas(64) unsigned char bv_tmap[128];   // CUtensorMap over Bt_v rows
   int has_b_tmap;
+  unsigned long long* prof;         // diagnostic cycle counters of the fused kernel, or nullptr
   int attend_impl;                  // 0: tensor-core fused kernel, 1: plain tile kernel
 };
 

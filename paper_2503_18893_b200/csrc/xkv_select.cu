@@ -144,7 +144,8 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
 // ---------------------------------------------------------------------------------------------
 
 constexpr int kTopkThreads = 1024;
-constexpr int kTopkItems = 16;   // consecutive chunks per thread in the compaction
+constexpr int kTopkItems = 16;    // consecutive chunks per thread and super-block
+constexpr int kTopkBins = 2048;   // histogram bins per radix pass
 
 // Order-preserving map float -> uint32 (larger float = larger key), with -0 folded onto +0.
 __device__ __forceinline__ uint32_t score_key(float f) {
@@ -153,14 +154,34 @@ __device__ __forceinline__ uint32_t score_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Keys of this thread's 16 consecutive chunks of one super-block (0 beyond n_c; callers mask by index).
+__device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, uint32_t (&key)[kTopkItems]) {
+  if (j0 + kTopkItems <= n_c && ((n_c & 3) == 0)) {
+    const float4* p = reinterpret_cast<const float4*>(S + j0);
+#pragma unroll
+    for (int i = 0; i < kTopkItems / 4; ++i) {
+      const float4 v = p[i];
+      key[4 * i] = score_key(v.x); key[4 * i + 1] = score_key(v.y);
+      key[4 * i + 2] = score_key(v.z); key[4 * i + 3] = score_key(v.w);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) key[i] = (j0 + i < n_c) ? score_key(S[j0 + i]) : 0u;
+  }
+}
+
 // One CTA per (layer, sequence, KV head).  grid.x = problems of the call.
+// Exact k_ch-th largest key by a radix select whose bins subdivide the range that still contains it
+// (first the [min, max] range of all keys, then the chosen bin, ...: at most three 11-bit passes), followed
+// by an ordered compaction.  CACHED: n_c fits one super-block and the keys stay in registers.
+template <bool CACHED>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel_idx,
             int32_t* __restrict__ sel_cnt) {
-  __shared__ uint32_t whist[kTopkThreads / 32][256];
-  __shared__ uint32_t hist[256];
+  __shared__ uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_tot[kTopkThreads / 32];
-  __shared__ uint32_t sh_prefix, sh_need;
+  __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
+  __shared__ uint32_t sh_a, sh_b;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_layer = dev.batch * dev.H_kv;
@@ -168,66 +189,110 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
   const float* __restrict__ S = dev.pooled + prob * dev.n_c;
   int32_t* __restrict__ out = sel_idx + prob * k_cap;
   const int n_c = dev.n_c, c = dev.c, T = dev.T;
+  const int super = kTopkThreads * kTopkItems;
+  const bool out_vec = (reinterpret_cast<uintptr_t>(out) & 15u) == 0;   // 16-byte stores of the row ids
+
+  uint32_t creg[kTopkItems];
+  if (CACHED) load_keys(S, tid * kTopkItems, n_c, creg);
 
   uint32_t thr = 0, need_eq = 0;
   const bool all = (k_ch >= n_c);
   if (!all) {
-    uint32_t prefix = 0, mask = 0, need = (uint32_t)k_ch;
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      for (int i = tid; i < (kTopkThreads / 32) * 256; i += kTopkThreads) (&whist[0][0])[i] = 0;
+    // ---- range of the keys
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    for (int base = 0; base < n_c; base += super) {
+      uint32_t key[kTopkItems];
+      const int j0 = base + tid * kTopkItems;
+      if (CACHED) {
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
+      } else {
+        load_keys(S, j0, n_c, key);
+      }
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) {
+        if (j0 + i < n_c) { kmin = min(kmin, key[i]); kmax = max(kmax, key[i]); }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    if (lane == 0) { warp_min[warp] = kmin; warp_max[warp] = kmax; }
+    __syncthreads();
+    kmin = warp_min[lane]; kmax = warp_max[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    // ---- radix passes over the window [lo, lo + span]
+    uint32_t lo = kmin, span = kmax - kmin, need = (uint32_t)k_ch;
+    for (;;) {
+      const int bits = 32 - __clz(span);                      // span < 2^bits
+      const int sh = bits > 11 ? bits - 11 : 0;
+      for (int i = tid; i < kTopkBins; i += kTopkThreads) hist[i] = 0;
       __syncthreads();
-      for (int j = tid; j < n_c; j += kTopkThreads) {
-        const uint32_t key = score_key(S[j]);
-        if ((key & mask) == prefix) atomicAdd(&whist[warp][(key >> shift) & 255u], 1u);
+      for (int base = 0; base < n_c; base += super) {
+        uint32_t key[kTopkItems];
+        const int j0 = base + tid * kTopkItems;
+        if (CACHED) {
+#pragma unroll
+          for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
+        } else {
+          load_keys(S, j0, n_c, key);
+        }
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) {
+          const uint32_t rel = key[i] - lo;
+          if (j0 + i < n_c && key[i] >= lo && rel <= span) atomicAdd(&hist[rel >> sh], 1u);
+        }
       }
       __syncthreads();
-      if (tid < 256) {
-        uint32_t s = 0;
-#pragma unroll 8
-        for (int w = 0; w < kTopkThreads / 32; ++w) s += whist[w][tid];
-        hist[tid] = s;
+      // suffix counts from the top bin down: thread t owns bins 2t, 2t+1
+      const uint32_t h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+      const uint32_t mine = h0 + h1;
+      uint32_t suf = mine;                                     // inclusive over higher lanes of the warp
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += v;
       }
+      if (lane == 0) warp_tot[warp] = suf;
       __syncthreads();
       if (warp == 0) {
-        // lane owns bins 8*lane .. 8*lane+7; suffix sums from the top bin downwards
-        uint32_t loc[8], tot = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { loc[i] = hist[lane * 8 + i]; tot += loc[i]; }
-        uint32_t above = tot;                       // inclusive suffix over lanes >= lane
+        const uint32_t t = warp_tot[lane];
+        uint32_t ws = t;                                       // inclusive over higher warps
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
-          if (lane + o < 32) above += v;
+          const uint32_t v = __shfl_down_sync(0xffffffffu, ws, o);
+          if (lane + o < 32) ws += v;
         }
-        above -= tot;                               // elements in bins of higher lanes
-        // exactly one lane holds the bin where the running count crosses `need`
-        if (above < need && above + tot >= need) {
-          uint32_t run = above;
-          int bsel = 0;
-#pragma unroll
-          for (int i = 7; i >= 0; --i) {
-            if (run < need && run + loc[i] >= need) { bsel = i; break; }
-            run += loc[i];
-          }
-          sh_prefix = prefix | ((uint32_t)(lane * 8 + bsel) << shift);
-          sh_need = need - run;
-        }
+        warp_tot[lane] = ws - t;                               // keys in bins of higher warps
       }
       __syncthreads();
-      prefix = sh_prefix;
-      need = sh_need;
-      mask |= 255u << shift;
+      const uint32_t above = warp_tot[warp] + (suf - mine);    // keys in bins above 2t+1
+      if (above < need && above + mine >= need) {              // exactly one thread
+        if (above + h1 >= need) { sh_a = 2 * tid + 1; sh_b = need - above; }
+        else { sh_a = 2 * tid; sh_b = need - above - h1; }
+      }
       __syncthreads();
+      const uint32_t bsel = sh_a;
+      need = sh_b;
+      lo += bsel << sh;
+      span = min(span - (bsel << sh), (sh ? (1u << sh) : 1u) - 1u);
+      __syncthreads();
+      if (sh == 0) break;
     }
-    thr = prefix;
+    thr = lo;
     need_eq = need;
   }
 
   // Ordered compaction: chunk j is taken if key > thr, or key == thr and fewer than need_eq equal
   // keys precede it.  Positions follow ascending j.
   uint32_t run_gt = 0, run_eq = 0;                  // totals of the super-blocks already done
-  const int super = kTopkThreads * kTopkItems;
+  uint32_t last_key = 0;
   for (int base = 0; base < n_c; base += super) {
     const int j0 = base + tid * kTopkItems;
     uint32_t gtm = 0, eqm = 0;                      // bit i set: item i is > / == thr
@@ -235,12 +300,19 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
 #pragma unroll
       for (int i = 0; i < kTopkItems; ++i) if (j0 + i < n_c) gtm |= 1u << i;
     } else {
+      uint32_t key[kTopkItems];
+      if (CACHED) {
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
+      } else {
+        load_keys(S, j0, n_c, key);
+      }
 #pragma unroll
       for (int i = 0; i < kTopkItems; ++i) {
         if (j0 + i < n_c) {
-          const uint32_t key = score_key(S[j0 + i]);
-          gtm |= (key > thr ? 1u : 0u) << i;
-          eqm |= (key == thr ? 1u : 0u) << i;
+          gtm |= (key[i] > thr ? 1u : 0u) << i;
+          eqm |= (key[i] == thr ? 1u : 0u) << i;
+          if (j0 + i == n_c - 1) last_key = key[i];
         }
       }
     }
@@ -262,7 +334,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
         if (lane >= o) ti += v;
       }
       warp_tot[lane] = ti - t;                      // exclusive prefix of warp totals
-      if (lane == 31) { sh_prefix = ti; }           // super-block total
+      if (lane == 31) sh_a = ti;                    // super-block total
     }
     __syncthreads();
     const uint32_t excl = inc - mine + warp_tot[warp];
@@ -276,25 +348,34 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
         const uint32_t pos = gt_before + min(eq_before, need_eq);
         const int j = j0 + i;
         const int rows = min(c, T - j * c);
-        for (int t = 0; t < rows; ++t) out[(size_t)pos * c + t] = j * c + t;
+        if (c == 8 && rows == 8 && out_vec) {
+          int4* o4 = reinterpret_cast<int4*>(out + (size_t)pos * 8);
+          o4[0] = make_int4(j * 8, j * 8 + 1, j * 8 + 2, j * 8 + 3);
+          o4[1] = make_int4(j * 8 + 4, j * 8 + 5, j * 8 + 6, j * 8 + 7);
+        } else {
+          for (int t = 0; t < rows; ++t) out[(size_t)pos * c + t] = j * c + t;
+        }
       }
       gt_before += is_gt ? 1u : 0u;
       eq_before += is_eq ? 1u : 0u;
     }
-    run_gt += sh_prefix & 0xffffu;
-    run_eq += sh_prefix >> 16;
+    run_gt += sh_a & 0xffffu;
+    run_eq += sh_a >> 16;
     __syncthreads();
   }
   // Row count: k_ch whole chunks unless the ragged last chunk was taken (it is then the last one).
   const int taken = all ? n_c : k_ch;
+  // the last chunk has the highest index, so it wins a tie only if every equal key fits
+  __shared__ uint32_t sh_last;                    // key of chunk n_c-1, published by the thread that owns it
+  {
+    const int owner = ((n_c - 1) % super) / kTopkItems;
+    if (tid == owner) sh_last = last_key;
+    __syncthreads();
+  }
   int cnt = taken * c;
   {
     bool last_in = all;
-    if (!all) {
-      const uint32_t key = score_key(S[n_c - 1]);
-      // the last chunk has the highest index, so it wins a tie only if every equal key fits
-      last_in = key > thr || (key == thr && run_eq <= need_eq);
-    }
+    if (!all) last_in = sh_last > thr || (sh_last == thr && run_eq <= need_eq);
     if (last_in) cnt -= (n_c * c - T);
   }
   for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
@@ -329,7 +410,10 @@ cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloa
   count_launch();
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  topk_kernel<<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+  if (dev.n_c <= kTopkThreads * kTopkItems)
+    topk_kernel<true><<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+  else
+    topk_kernel<false><<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
   count_launch();
   return cudaGetLastError();
 }

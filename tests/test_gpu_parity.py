@@ -195,3 +195,31 @@ def test_model_shapes_reduced_context(cfg_id, over):
         np.testing.assert_allclose(glse[l, b, hs], olse[l, b, hs], atol=2e-2)
     assert g.status() == (0, 0)
     g.close()
+
+
+def test_small_ranks_and_many_tiles_do_not_stall():
+    """One 64-column slab per phase and many tiles per CTA: exercises the ring hand-offs with almost no work
+    per tile (a regression test for a stall that the bounded waits turned into a TIMEOUT flag)."""
+    s = synth.config(1, T=20000, k=6000, H_kv=1, H_q=4, d_h=128, r_k=64, r_v=8)
+    inp = C.case_from_factors(s)
+    oidx, ocnt, oout, olse = C.oracle_step(s, inp, 0)
+    g = C.GpuCase(s, inp)
+    gidx, gcnt = g.select(0)
+    _check_select(gidx, gcnt, oidx, ocnt)
+    gout, glse = g.attend(gidx, gcnt, 0)
+    assert g.status() == (0, 0)
+    assert C.rel_err(gout, oout) <= TOL
+    g.close()
+
+
+def test_more_chunks_than_one_topk_superblock():
+    """n_c = 17501 > 16384: the top-k kernel re-reads the pooled scores instead of caching them in registers."""
+    s = synth.config(1, T=140001, k=3000, r_k=8, r_v=8)
+    inp = C.case_from_factors(s)
+    oidx, ocnt, _, _ = C.oracle_step(s, inp, 0, problems=[(0, 0, 0), (1, 0, 1)])
+    g = C.GpuCase(s, inp)
+    gidx, gcnt = g.select(0)
+    for (l, hk) in ((0, 0), (1, 1)):
+        np.testing.assert_array_equal(gidx[l, 0, hk], oidx[l, 0, hk])
+        assert gcnt[l, 0, hk] == ocnt[l, 0, hk]
+    g.close()
