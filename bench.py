@@ -239,6 +239,10 @@ def main():
     stream = torch.cuda.current_stream()
     for i in range(args.warmup):
         wl.step(i)
+        if i == 0:
+            st0, fl0 = xkv.xkv_group_status(wl.groups[0])
+            if st0 != 0:   # a kernel gave up on a bounded wait or saw a bad index: do not time a broken run
+                raise SystemExit(f"device status {st0} (flags {fl0}) after the first step: {xkv.xkv_strerror(st0)}")
     barrier()
 
     # ---- timed region 1: inputs resident in HBM; per-call events for the kernel roofline

@@ -166,16 +166,19 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
       dst = (type)p;                                       \
       g->workspace_bytes += (bytes);                       \
     } while (0)
-    __nv_bfloat16 *Bt_k, *Bt_v; float2 *rhi, *rlo;
+    __nv_bfloat16 *Bt_k, *Bt_v, *Bv_copy; float2 *rhi, *rlo;
     XKV_ALLOC(Bt_k, __nv_bfloat16*, btk);
     XKV_ALLOC(Bt_v, __nv_bfloat16*, btv);
+    XKV_ALLOC(Bv_copy, __nv_bfloat16*, (size_t)c.batch * c.G * c.r_v * c.H_kv * c.d_h * sizeof(__nv_bfloat16));
     XKV_ALLOC(d.pooled, float*, pooled);
     XKV_ALLOC(rhi, float2*, hi);
     XKV_ALLOC(rlo, float2*, lo);
     XKV_ALLOC(d.part, float*, part);
     XKV_ALLOC(d.flags, unsigned int*, 256);
 #undef XKV_ALLOC
-    d.Bt_k = Bt_k; d.Bt_v = Bt_v; d.rope_hi = rhi; d.rope_lo = rlo;
+    d.Bt_k = Bt_k; d.Bt_v = Bt_v; d.B_v = Bv_copy; d.rope_hi = rhi; d.rope_lo = rlo;
+    XKV_TRY_CUDA(cudaMemcpyAsync(Bv_copy, c.B_v, (size_t)c.batch * c.G * c.r_v * c.H_kv * c.d_h * sizeof(__nv_bfloat16),
+                                 cudaMemcpyDeviceToDevice, s));
     XKV_TRY_CUDA(cudaMemsetAsync(d.flags, 0, 256, s));
     XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_k, Bt_k, c.batch, c.G, c.r_k, c.H_kv, c.d_h, s));
     XKV_TRY_CUDA(launch_repack_b((const __nv_bfloat16*)c.B_v, Bt_v, c.batch, c.G, c.r_v, c.H_kv, c.d_h, s));
@@ -276,7 +279,7 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) ||
       ((uintptr_t)sel_cnt & 3u) || ((uintptr_t)lse & 3u))
     return XKV_ERR_INVALID_ARG;
-  cudaError_t e = g->attend_impl
+  cudaError_t e = (g->attend_impl || !fused_supported(g))
                       ? launch_reconstruct_attend(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt,
                                                   k_cap, (__nv_bfloat16*)out, lse, (cudaStream_t)stream)
                       : launch_fused(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt, k_cap,

@@ -2,15 +2,24 @@
 // tensor-core path.  One persistent CTA per SM walks a contiguous range of 128-row tiles of the selected
 // sets; a problem is one (layer, sequence, KV head).
 //
-// Per tile (128 selected rows S_t of one problem):
-//   K_hat   [j][d] = sum_m A_k[S_t[j]][m] * B_k[m][d]     tcgen05.mma, M = rows, N = d_h, accumulator in TMEM
-//   logits  z[h][j] = scale * <q_h, rope(K_hat[j])>         thread j owns TMEM lane j (one rebuilt key row)
-//   V_hat^T [d][j] = sum_m B_v[m][d] * A_v[S_t[j]][m]     tcgen05.mma, M = d_h, N = rows
-//   o[h][d] += sum_j p[h][j] * V_hat^T[d][j]                thread d owns TMEM lane d; online softmax
-// Rebuilt K/V never leave the SM.  Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-11 gather
-// producers (cp.async of the selected rows into a deep ring), 12 MMA issue, 13 TMA loader of the B slabs
-// (a short ring of its own: those come from L2 and need little lead).
+// Per tile (128 selected rows S_t of one problem, j indexes the tile's rows, m the rank dimension):
+//   keys    K_hat[j][d] = sum_m A_k[S_t[j]][m] B_k[m][d]       tcgen05.mma, M = rows, N = d_h, fp32 in TMEM
+//           z[h][j]     = scale * <q_h, rope(K_hat[j])>          thread j owns TMEM lane j (one rebuilt key row)
+//           p[h][j]     = exp(z - running max)                   online softmax; p is handed on as bf16
+//   values  W[m][h]    += sum_j A_v[S_t[j]][m] p[h][j]           tcgen05.mma, M = 128 rank columns, N = heads
+// and once per problem, after the segments have been merged,  out_h = (W[:, h] / l_h)^T B_v.
+// This is Eq. 3 for the values with the product re-associated: sum_j p_j (A_v[S_j] B_v) = (sum_j p_j A_v[S_j]) B_v,
+// so the rebuilt value rows are consumed in factored form and never materialised.  Rebuilt key rows live in
+// TMEM only.  Every gathered byte is written to shared memory once and read by the tensor core once.
+//
+// Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-11 gather producers (cp.async of the selected rows into
+// a deep ring), 12 MMA issue, 13 TMA loader of the B_k slabs (a short ring: they come from L2).
 // Every wait is bounded; a wait that runs out raises XKV_FLAG_TIMEOUT and the CTA winds down.
+//
+// Diagnostic counters (cycles, per CTA, 64 words; see xkv_debug_read_profile): 0 producer total, 1-3 producer
+// waits (rotary buffer, positions, ring), 4 tiles; 8 MMA total, 9 accumulator waits, 10 B ring, 11 row ring,
+// 12 issue; 13 weights; 17 loader wait; 24 key epilogue total, 25 positions, 26 accumulator, 27 group barrier,
+// 28 weights buffer; 32 value epilogue total, 33 accumulator.
 #include <cuda.h>
 
 #include "xkv_internal.cuh"
@@ -28,7 +37,9 @@ constexpr int kNB = 4;                           // slots of the B-slab ring
 constexpr int kThreads = 14 * 32;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kRopeStride = 66;                  // float2 per staged rotary row (64 + pad against bank conflicts)
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
+constexpr int kPBytes = 2 * 16 * 128;            // softmax weights of a tile as a bf16 MMA operand: [2][16 heads][64 rows]
+constexpr int kMaxBlocks = 8;                    // 128-column blocks of r_v that fit the TMEM accumulators
+constexpr unsigned long long kWaitLimitNs = 250000000ull;    // a wait that lasts a quarter of a second has failed
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -43,19 +54,20 @@ struct Sched {
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, empty, bfull, kfull, kempty, vfull, vempty, pfull, pempty, rfree, posfull, grp, total;
+  int full, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, grp, total;
 };
 __host__ __device__ constexpr Bars bar_layout(int na) {
   Bars b{};
-  b.full = 0; b.empty = na; b.bfull = na + na / 2; b.kfull = b.bfull + kNB;   // `empty` holds one barrier per slot pair
-  b.kempty = b.kfull + 2; b.vfull = b.kempty + 2;
-  b.vempty = b.vfull + 2; b.pfull = b.vempty + 2; b.pempty = b.pfull + 2; b.rfree = b.pempty + 2;
-  b.posfull = b.rfree + 2; b.grp = b.posfull + 2; b.total = b.grp + 1;
+  // one release barrier per slot pair and kind of occupant (key-phase or value-phase slabs): a waiter that knows
+  // the kind it waits for is never confused by the other kind's completions
+  b.full = 0; b.emptyk = na; b.emptyv = na + na / 2; b.bfull = 2 * na; b.kfull = b.bfull + kNB;
+  b.kempty = b.kfull + 2; b.wfull = b.kempty + 2; b.wempty = b.wfull + 2; b.pfull = b.wempty + 2;
+  b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.grp = b.posfull + 2; b.total = b.grp + 1;
   return b;
 }
 
 // cta that owns global tile t when cta i owns tiles [i*N/C, (i+1)*N/C)
-__device__ __forceinline__ int cta_of_tile(long long t, int C, int N) { return (int)(((t + 1) * C - 1) / N); }
+__host__ __device__ __forceinline__ int cta_of_tile(long long t, int C, int N) { return (int)(((t + 1) * C - 1) / N); }
 
 struct Ctx {
   volatile int* abort;
@@ -69,15 +81,6 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait on an mbarrier phase.  Returns false if another thread of the CTA has given up, or if the
 // phase does not complete within kWaitLimitNs (then this thread raises the flag and makes the others give up).
-__device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity);
-// `slot` >= 0 (passed warp-uniformly by one warp per role when diagnostics are on) adds the cycles waited.
-__device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity, int slot = -1) {
-  if (c.prof == nullptr || slot < 0) return wait_bar_raw(c, bar, parity);
-  const long long c0 = clock64();
-  const bool r = wait_bar_raw(c, bar, parity);
-  if ((threadIdx.x & 31) == 0) atomicAdd(c.prof + slot, (unsigned long long)(clock64() - c0));
-  return r;
-}
 __device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
@@ -91,6 +94,14 @@ __device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_
   *c.abort = 1;
   atomicOr(c.flags, XKV_FLAG_TIMEOUT);
   return false;
+}
+// `slot` >= 0 (passed warp-uniformly by one warp per role when diagnostics are on) adds the cycles waited.
+__device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity, int slot = -1) {
+  if (c.prof == nullptr || slot < 0) return wait_bar_raw(c, bar, parity);
+  const long long c0 = clock64();
+  const bool r = wait_bar_raw(c, bar, parity);
+  if ((threadIdx.x & 31) == 0) atomicAdd(c.prof + slot, (unsigned long long)(clock64() - c0));
+  return r;
 }
 
 // Logits of one rebuilt key row against NR query heads: rotate the (i, i+HALF) pairs, accumulate q . k.
@@ -147,11 +158,11 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
   }
 }
 
-// Shared memory besides the two rings: rotary rows, queries, softmax weights, positions, barriers.
+// Shared memory besides the two rings: weights, rotary rows, queries, positions, barriers.
 template <int DH, int NR>
 __host__ __device__ constexpr int misc_smem_bytes() {
-  return (int)(sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR * kTile + 2 * NR + 8 * NR) +
-               sizeof(int) * (2 * kTile + 8) + 8 * (2 * 16 + 2 * kNB + 20) + 16);
+  return (int)(2 * kPBytes + sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR + 8 * NR) +
+               sizeof(int) * (2 * kTile + 8) + 8 * (2 * 16 + kNB + 24) + 16);
 }
 // Slots of the gathered-row ring: whatever fits beside the B ring.
 template <int DH, int NR>
@@ -159,25 +170,28 @@ __host__ __device__ constexpr int ring_slots() {
   return ((kSmemLimit - 1024 - misc_smem_bytes<DH, NR>() - kNB * kSlabBytes) / kSlabBytes) & ~1;   // even: released in pairs
 }
 
-template <int DH, int NR>
+// NR: query heads per KV head rounded up to 4, 8 or 16.  WB: most 128-column blocks of r_v (registers of the
+// value epilogue): NR * WB <= 64.
+template <int DH, int NR, int WB>
 __global__ void __launch_bounds__(kThreads, 1)
-sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constant__ CUtensorMap bv_map, GroupDev dev,
-                Sched sc, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ sel_idx,
-                const int32_t* __restrict__ sel_cnt) {
+sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched sc, const __nv_bfloat16* __restrict__ q,
+                const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int HALF = DH / 2;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   constexpr int S = ring_slots<DH, NR>();          // gathered-row slots, all of which may be in flight
-  static_assert(S >= 4 && S <= 16, "ring size");
+  static_assert(S >= 4 && S <= 16, "ring size");   // slot pairs are tracked in 3 bits by the loader
+  static_assert(kNB <= 8, "loader fifo");
   const uint32_t bring = base + (uint32_t)S * kSlabBytes;                         // B-slab ring
   // carve-up after the two rings
-  float2* hi_s = reinterpret_cast<float2*>(gen + (size_t)(S + kNB) * kSlabBytes); // [2][16][kRopeStride] coarse rotary rows
+  uint8_t* P_gen = gen + (size_t)(S + kNB) * kSlabBytes;                         // [2][kPBytes] bf16 weights (MMA operand)
+  const uint32_t P_addr = base + (uint32_t)(S + kNB) * kSlabBytes;
+  float2* hi_s = reinterpret_cast<float2*>(P_gen + 2 * kPBytes);                 // [2][16][kRopeStride] coarse rotary rows
   float2* lo_s = hi_s + 2 * 16 * kRopeStride;                                    // [8][kRopeStride]     fine rotary rows
   float* q_s = reinterpret_cast<float*>(lo_s + 8 * kRopeStride);                 // [NR][DH]
-  float* P_s = q_s + NR * DH;                                                    // [2][NR][128]
-  float* alpha_s = P_s + 2 * NR * kTile;                                         // [2][NR]
+  float* alpha_s = q_s + NR * DH;                                                // [2][NR]
   float* red_s = alpha_s + 2 * NR;                                               // [2][4][NR]
   int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [2][128]
   int* algn_s = pos_s + 2 * kTile;                                               // [2][4]
@@ -190,15 +204,18 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   Ctx ctx{abort_flag, dev.flags, sc.prof ? sc.prof + (size_t)blockIdx.x * 64 : nullptr};
   // the staged rotary path needs the fine table to cover exactly 8 positions
   const bool rope_smem = dev.use_rope && dev.rope_shift == 3;
+  // both phases are padded to an even number of 64-column slabs so that slabs pair up inside ring-slot pairs
+  const int nks_k = (dev.r_k + 63) >> 6, nks_v = (dev.r_v + 63) >> 6;
+  const int nst_k = (nks_k + 1) & ~1, nst_v = (nks_v + 1) & ~1;
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) mbar_init(BAR(bl.full + s), 128);
-    for (int s = 0; s < S / 2; ++s) mbar_init(BAR(bl.empty + s), 1);
+    for (int s = 0; s < S / 2; ++s) { mbar_init(BAR(bl.emptyk + s), 1); mbar_init(BAR(bl.emptyv + s), 1); }
     for (int s = 0; s < kNB; ++s) mbar_init(BAR(bl.bfull + s), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(BAR(bl.kfull + b), 1); mbar_init(BAR(bl.kempty + b), 128);
-      mbar_init(BAR(bl.vfull + b), 1); mbar_init(BAR(bl.vempty + b), 128);
-      mbar_init(BAR(bl.pfull + b), 128); mbar_init(BAR(bl.pempty + b), 128);
+      mbar_init(BAR(bl.wfull + b), 1); mbar_init(BAR(bl.wempty + b), 128);
+      mbar_init(BAR(bl.pfull + b), 128);
       mbar_init(BAR(bl.rfree + b), 128); mbar_init(BAR(bl.posfull + b), 128);
     }
     mbar_init(BAR(bl.grp), 128);
@@ -208,6 +225,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   if (rope_smem) {
     for (int i = tid; i < 8 * HALF; i += kThreads) lo_s[(i / HALF) * kRopeStride + (i % HALF)] = dev.rope_lo[i];
   }
+  // weights of heads that do not exist stay zero for the whole kernel
+  for (int i = tid; i < 2 * kPBytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(P_gen)[i] = 0u;
+  fence_proxy_async();
   if (warp == 12) {
     tmem_alloc(smem_u32(tmem_slot), 512);
     tmem_relinquish();
@@ -227,12 +247,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
     g = py % dev.H_kv; b = (py / dev.H_kv) % dev.batch; l = sc.l0 + py / per_layer;
     return ((long long)l * dev.batch + b) * dev.H_kv + g;
   };
-
   // Walks this CTA's tiles, skipping tiles that start at or beyond the problem's row count.
   struct TileIter {
-    long long t; int py, ti, cnt, l, b, g; long long prob; bool fresh;   // fresh: first visited tile of its problem
+    long long t; int py, ti, cnt, l, b, g; long long prob;
   };
-  auto iter_begin = [&](TileIter& it_) { it_.t = t_begin - 1; it_.py = -1; it_.cnt = 0; it_.fresh = false; };
+  auto iter_begin = [&](TileIter& it_) { it_.t = t_begin - 1; it_.py = -1; it_.cnt = 0; it_.prob = 0; };
   // advance to the next non-empty tile; returns false at the end of the range.  `on_problem(py)` runs whenever
   // the walk enters a new problem (also for problems whose tiles are all empty), before its tiles.
   auto iter_next = [&](TileIter& it_, auto&& on_problem) -> bool {
@@ -251,15 +270,22 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
     }
   };
   auto no_op = [](int) {};
+  // partial slot of the segment (this CTA's share) of problem ordinal py
+  auto part_of = [&](int py, long long prob) {
+    const int seg = (int)blockIdx.x - cta_of_tile((long long)py * sc.tpp, C, N);
+    return dev.part + ((size_t)prob * sc.n_slots + seg) * (size_t)n_rep * (dev.r_v + 2);
+  };
 
   if (warp >= 8 && warp < 12) {
-    // =============================== producers: gather rows of A, TMA the B slabs ===============================
+    // =============================== producers: gather rows of A ===============================
     // Eight consecutive lanes copy the eight 16-byte pieces of one 128-byte row slab, so that every
     // request of a warp covers whole 128-byte lines; thread pt serves rows (pt>>3) + 16*i, i = 0..7.
     const int pt = tid - 256, pw = warp - 8;
     const uint32_t c8 = (uint32_t)(pt & 7);
-    int slot = 0;                     // ring position and the parity of its current round
-    uint32_t ring_par = 0;
+    int slot = 0;                     // ring position
+    // per slot pair (bit p): has it been used, was its last occupant a value-phase pair, and the parity of the
+    // number of key-phase / value-phase pairs issued into it so far
+    uint32_t occ_any = 0, occ_v = 0, cnt_k = 0, cnt_v = 0;
     // rows (pt>>3) + 16*i share the swizzle phase (pt>>3)&7; slot-relative destination of the i = 0 piece
     const uint32_t dst0 = (uint32_t)(pt >> 3) * 128u + ((c8 ^ ((uint32_t)(pt >> 3) & 7u)) << 4);
     const int ps = pw == 0 ? 0 : -1000;
@@ -278,73 +304,99 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       return p;
     };
     int p_next = have ? load_pos(nxt) : -1;   // row index of the next tile, fetched one tile ahead
-    while (have && ok) {
-      cur = nxt;
-      const int p = p_next;
-      have = iter_next(nxt, no_op);
-      if (have) p_next = load_pos(nxt);
-      const int buf = it & 1;
-      // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
-      if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
-      pos_s[buf * kTile + pt] = p;
-      if (rope_smem) {
-        // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
-        const int hidx = p < 0 ? -1 : (p >> 3);
-        int gmax = hidx;
-        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
-        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
-        gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 4));
-        const bool aligned = __all_sync(0xffffffffu, p < 0 || hidx == gmax);
-        if (lane == 0) algn_s[buf * 4 + pw] = aligned ? 1 : 0;
-        if (aligned) {
-#pragma unroll
-          for (int a = 0; a < 4; ++a) {
-            const int gm = __shfl_sync(0xffffffffu, gmax, a * 8);
-            if (lane * 2 < HALF) {
-              cp_async16(smem_u32(hi_s + (size_t)(buf * 16 + pw * 4 + a) * kRopeStride + lane * 2),
-                         dev.rope_hi + (size_t)(gm < 0 ? 0 : gm) * HALF + lane * 2, 16u);
-            }
-          }
-        }
-      }
-      // publish the row positions of the tile (to the other producer threads and to the key epilogue)
-      mbar_arrive(BAR(bl.posfull + buf));
-      if (!wait_bar(ctx, BAR(bl.posfull + buf), (uint32_t)((it >> 1) & 1), ps + 2)) { ok = false; break; }
-      long long rowidx[8];
+    // one phase of one tile: the 64-column slabs of its gathered rows, in ring order
+    auto issue_phase = [&](int phase, int buf, int b) {
+      const int r = phase ? dev.r_v : dev.r_k;
+      const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
+      const int nst = phase ? nst_v : nst_k;
+      const __nv_bfloat16* rp[8];                      // this thread's piece of each of its eight rows
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int pr = pos_s[buf * kTile + i * 16 + (pt >> 3)];
-        rowidx[i] = (long long)cur.b * dev.T + (pr < 0 ? 0 : pr);
+        rp[i] = A + ((long long)b * dev.T + (pr < 0 ? 0 : pr)) * r + (int)c8 * 8;
       }
 #pragma unroll 1
-      for (int phase = 0; phase < 2 && ok; ++phase) {
-        const int r = phase ? dev.r_v : dev.r_k;
-        const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
-        const int nks = (r + 63) >> 6;
-        const __nv_bfloat16* rp[8];                    // this thread's piece of each of its eight rows
-#pragma unroll
-        for (int i = 0; i < 8; ++i) rp[i] = A + rowidx[i] * r + (int)c8 * 8;
-#pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks) {
-          // slots are released in pairs (one tcgen05.commit per two slabs): wait when entering a pair
-          if ((slot & 1) == 0 && !wait_bar(ctx, BAR(bl.empty + (slot >> 1)), ring_par ^ 1u, ps + 3)) { ok = false; break; }
-          const uint32_t st = base + (uint32_t)slot * kSlabBytes + dst0;
-          const bool in = ks * 64 + (int)c8 * 8 < r;   // false only in a ragged last slab: zero-fill
-          const uint32_t nbytes = in ? 16u : 0u;
-          const int adv = in ? ks * 64 : 0;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
-          cp_async_arrive_noinc(BAR(bl.full + slot));  // arrives when this thread's copies have landed
-          if (++slot == S) { slot = 0; ring_par ^= 1u; }
+      for (int ks = 0; ks < nst; ++ks) {
+        // slots are released in pairs (one tcgen05.commit per two slabs): when entering a pair, wait for the
+        // release of its previous occupant (occupant number c of its kind completes phase c of that barrier)
+        if ((slot & 1) == 0) {
+          const int pr = slot >> 1;
+          const uint32_t bit = 1u << pr;
+          if (occ_any & bit) {
+            const bool was_v = (occ_v & bit) != 0;
+            const uint32_t par = (((was_v ? cnt_v : cnt_k) >> pr) & 1u) ^ 1u;
+            if (!wait_bar(ctx, BAR((was_v ? bl.emptyv : bl.emptyk) + pr), par, ps + 3)) { ok = false; return; }
+          }
+          occ_any |= bit;
+          if (phase) { occ_v |= bit; cnt_v ^= bit; } else { occ_v &= ~bit; cnt_k ^= bit; }
         }
+        const uint32_t st = base + (uint32_t)slot * kSlabBytes + dst0;
+        const bool in = ks * 64 + (int)c8 * 8 < r;     // false in a ragged last slab or a padding slab: zero-fill
+        const uint32_t nbytes = in ? 16u : 0u;
+        const int adv = in ? ks * 64 : 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
+        cp_async_arrive_noinc(BAR(bl.full + slot));    // arrives when this thread's copies have landed
+        if (++slot == S) slot = 0;
       }
-      ++it;
+    };
+    // Ring order: K(0), K(1), V(0), K(2), V(1), ...  The value phase of a tile needs the softmax weights that
+    // the key epilogue derives from its key phase, so the next tile's key phase is put in between.
+    int nv = 0, b_pend = 0;           // value phases issued; `it` counts key phases issued
+    while (ok) {
+      const bool do_k = have;
+      if (do_k) {
+        cur = nxt;
+        const int p = p_next;
+        have = iter_next(nxt, no_op);
+        if (have) p_next = load_pos(nxt);
+        const int buf = it & 1;
+        // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
+        if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
+        pos_s[buf * kTile + pt] = p;
+        if (rope_smem) {
+          // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
+          const int hidx = p < 0 ? -1 : (p >> 3);
+          int gmax = hidx;
+          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 4));
+          const bool aligned = __all_sync(0xffffffffu, p < 0 || hidx == gmax);
+          if (lane == 0) algn_s[buf * 4 + pw] = aligned ? 1 : 0;
+          if (aligned) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+              const int gm = __shfl_sync(0xffffffffu, gmax, a * 8);
+              if (lane * 2 < HALF) {
+                cp_async16(smem_u32(hi_s + (size_t)(buf * 16 + pw * 4 + a) * kRopeStride + lane * 2),
+                           dev.rope_hi + (size_t)(gm < 0 ? 0 : gm) * HALF + lane * 2, 16u);
+              }
+            }
+          }
+        }
+        // publish the row positions of the tile (to the other producer threads and to the key epilogue)
+        mbar_arrive(BAR(bl.posfull + buf));
+        if (!wait_bar(ctx, BAR(bl.posfull + buf), (uint32_t)((it >> 1) & 1), ps + 2)) { ok = false; break; }
+        issue_phase(0, buf, cur.b);
+        if (!ok) break;
+      }
+      const int k_issued = it + (do_k ? 1 : 0);
+      if (nv < k_issued - (do_k ? 1 : 0)) {
+        // positions of tile nv are still in its buffer: that buffer is next written for tile nv + 2
+        issue_phase(1, nv & 1, b_pend);
+        ++nv;
+      } else if (!do_k) {
+        break;
+      }
+      if (do_k) { b_pend = cur.b; ++it; }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     if (ctx.prof && pt == 0) { ctx.prof[0] = (unsigned long long)(clock64() - role_t0); ctx.prof[4] = (unsigned long long)it; }
   } else if (warp == 12) {
     // =============================== MMA issue ===============================
-    constexpr uint32_t idesc = idesc_bf16_f32(128, 128);
+    // the whole warp walks the loop (all values are warp-uniform); one lane issues the tensor-core instructions
+    constexpr uint32_t idesc_k = idesc_bf16_f32(128, 128);                     // keys: both operands K-major
+    constexpr uint32_t idesc_v = idesc_bf16_f32(128, 16) | (1u << 15);         // values: A is read along its rows (MN-major)
     const int ps = 8;
     const long long role_t0 = clock64();
     int slot = 0, bslot = 0;                          // positions in the two rings and their round parities
@@ -353,104 +405,163 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
     const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
     const uint32_t rows_lo0 = (uint32_t)(smem_desc_sw128(base, 0) & 0xFFFFFFFFull);
     const uint32_t b_lo0 = (uint32_t)(smem_desc_sw128(bring, 0) & 0xFFFFFFFFull);
-    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
-    bool ok = true;
-    // the whole warp walks the loop (all values are warp-uniform); one lane issues the tensor-core instructions
-    for (long long t = t_begin; t < t_end && ok; ++t) {
-      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
-      if (py != cur_py) { cur_py = py; const long long prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
-      if (ti * kTile >= cnt) continue;
-      const int buf = it & 1;
-      const uint32_t par = (uint32_t)((it >> 1) & 1);
-#pragma unroll 1
-      for (int phase = 0; phase < 2 && ok; ++phase) {
-        const int r = phase ? dev.r_v : dev.r_k;
-        const int nks = (r + 63) >> 6;
-        const int last_kk = (((r - 1) & 63) >> 4) + 1;          // 16-column steps in the last slab
-        const uint32_t acc = tmem + (uint32_t)(phase * 256 + buf * 128);
-        if (!wait_bar(ctx, BAR((phase ? bl.vempty : bl.kempty) + buf), par ^ 1u, ps + 1)) { ok = false; break; }
+    // value phase: A = two adjacent row slabs read transposed (64 rank columns each, 16384 bytes apart),
+    // rows advance in 8-row groups of 1024 bytes; B = the weights of 16 heads x 16 rows
+    const uint32_t rows_t_lo0 = (rows_lo0 & 0xFFFFu) | ((uint32_t)(kSlabBytes >> 4) << 16);
+    const uint32_t p_lo0 = (uint32_t)(smem_desc_sw128(P_addr, 0) & 0xFFFFFFFFull);
+    int it = 0, nv = 0;               // key phases and value phases issued
+    bool ok = true, more = true;
+    TileIter cur;
+    iter_begin(cur);
+    // same order as the producers: K(0), K(1), V(0), K(2), V(1), ...
+    while (ok) {
+      const bool do_k = more && iter_next(cur, no_op);
+      if (!do_k) more = false;
+      // ---- keys: K_hat = A_k[S] B_k
+      const long long ph0 = ctx.prof ? clock64() : 0;
+      if (do_k) {
+        const int buf = it & 1;
+        const uint32_t par = (uint32_t)((it >> 1) & 1);
+        const int last_kk = (((dev.r_k - 1) & 63) >> 4) + 1;    // 16-column steps in the last real slab
+        const uint32_t acc = tmem + (uint32_t)(buf * 128);
+        if (!wait_bar(ctx, BAR(bl.kempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks) {
-          if (!wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
+        for (int ks = 0; ks < nst_k && ok; ++ks) {
+          const bool real = ks < nks_k;
+          if (real && !wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
           if (!wait_bar(ctx, BAR(bl.full + slot), ring_par, ps + 3)) { ok = false; break; }
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
           if (lane == 0) {
-            const uint32_t rows_lo = rows_lo0 + (uint32_t)slot * (kSlabBytes >> 4);   // gathered rows of A
-            const uint32_t b_lo = b_lo0 + (uint32_t)bslot * (kSlabBytes >> 4);        // slab of the transposed B block
-            const uint64_t a_desc = desc_hi | (phase ? b_lo : rows_lo);               // keys: M = rows; values: M = d
-            const uint64_t b_desc = desc_hi | (phase ? rows_lo : b_lo);
-            const int nkk = (ks == nks - 1) ? last_kk : 4;
-            tc_mma_bf16(acc, a_desc, b_desc, idesc, ks ? 1u : 0u);
+            if (real) {
+              const uint64_t a_desc = desc_hi | (rows_lo0 + (uint32_t)slot * (kSlabBytes >> 4));
+              const uint64_t b_desc = desc_hi | (b_lo0 + (uint32_t)bslot * (kSlabBytes >> 4));
+              const int nkk = (ks == nks_k - 1) ? last_kk : 4;
+              tc_mma_bf16(acc, a_desc, b_desc, idesc_k, ks ? 1u : 0u);
 #pragma unroll
-            for (int kk = 1; kk < 4; ++kk) {
-              if (kk < nkk) tc_mma_bf16(acc, a_desc + 2u * kk, b_desc + 2u * kk, idesc, 1u);   // +32 bytes per step
+              for (int kk = 1; kk < 4; ++kk) {
+                if (kk < nkk) tc_mma_bf16(acc, a_desc + 2u * kk, b_desc + 2u * kk, idesc_k, 1u);   // +32 bytes per step
+              }
             }
-            if (slot & 1) tc_commit(BAR(bl.empty + (slot >> 1)));   // releases both slabs of the pair (and their B slabs)
-            if (ks == nks - 1) tc_commit(BAR((phase ? bl.vfull : bl.kfull) + buf));
+            if (slot & 1) tc_commit(BAR(bl.emptyk + (slot >> 1)));   // releases both slabs of the pair (and their B slabs)
+            if (ks == nst_k - 1) tc_commit(BAR(bl.kfull + buf));
           }
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + 12, (unsigned long long)(clock64() - i0));
           if (++slot == S) { slot = 0; ring_par ^= 1u; }
-          if (++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
+          if (real && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
+        if (!ok) break;
+        ++it;
       }
-      ++it;
+      const long long ph1 = ctx.prof ? clock64() : 0;
+      if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + 14, (unsigned long long)(ph1 - ph0)); }
+      // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
+      if (nv < it - (do_k ? 1 : 0)) {
+        const int buf = nv & 1;
+        const uint32_t par = (uint32_t)((nv >> 1) & 1);
+        if (!wait_bar(ctx, BAR(bl.wempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
+        if (!wait_bar(ctx, BAR(bl.pfull + buf), par, ps + 5)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t accw = tmem + 256u + (uint32_t)(buf * 128);
+        const uint32_t p_lo = p_lo0 + (uint32_t)buf * (kPBytes >> 4);
+#pragma unroll 1
+        for (int ks = 0; ks < nst_v && ok; ks += 2) {
+          if (!wait_bar(ctx, BAR(bl.full + slot), ring_par, ps + 3)) { ok = false; break; }
+          if (!wait_bar(ctx, BAR(bl.full + slot + 1), ring_par, ps + 3)) { ok = false; break; }
+          tc_fence_after();
+          const long long i0 = ctx.prof ? clock64() : 0;
+          if (lane == 0) {
+            const uint64_t a_desc = desc_hi | (rows_t_lo0 + (uint32_t)slot * (kSlabBytes >> 4));
+            const uint32_t acc = accw + (uint32_t)(ks >> 1) * 16u;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {   // 16 tile rows per step: 2048 bytes down the slab, 32 bytes along P
+              const uint64_t b_desc = desc_hi | (p_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u);
+              tc_mma_bf16(acc, a_desc + (uint32_t)kk * (2048u >> 4), b_desc, idesc_v, kk ? 1u : 0u);
+            }
+            tc_commit(BAR(bl.emptyv + (slot >> 1)));
+            if (ks + 2 >= nst_v) tc_commit(BAR(bl.wfull + buf));
+          }
+          __syncwarp();
+          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + 12, (unsigned long long)(clock64() - i0));
+          slot += 2;
+          if (slot == S) { slot = 0; ring_par ^= 1u; }
+        }
+        if (!ok) break;
+        ++nv;
+        if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + 15, (unsigned long long)(clock64() - ph1)); }
+      } else if (!do_k) {
+        break;
+      }
     }
     if (ctx.prof && lane == 0) ctx.prof[8] = (unsigned long long)(clock64() - role_t0);
     __syncwarp();
   } else if (warp == 13) {
-    // =============================== B-slab loader (TMA) ===============================
-    // B slab of stage n goes to slot n % kNB.  That slot held stage n - kNB, whose MMAs are known to be complete
-    // when the row-ring pair of stage n - kNB has been released; the loader follows that stage's ring position.
-    int bslot = 0, n_issued = 0, xslot = 0;
-    uint32_t xpar = 0;
-    int cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
+    // =============================== B_k slab loader (TMA) ===============================
+    // B slab n goes to slot n % kNB, which held slab n - kNB.  That slab's MMAs are known to be complete
+    //   - if it belongs to an earlier tile: when the previous tile's key accumulator was committed (kfull);
+    //   - if it belongs to this tile: when the row-ring pair of its stage was released (key-kind barrier).
+    // In both cases the barrier's previous phase is already known to be complete and its next phase cannot
+    // complete before the slab being loaded is consumed, so the parity test is unambiguous.
+    int bslot = 0, it = 0, slot = 0;
+    uint32_t cnt_k = 0;                  // per slot pair: parity of the number of key-phase pairs that used it
+    uint32_t fifo = 0;                   // per B slot, 4 bits: slot pair (3) and phase parity (1) of the slab it holds
     bool ok = true;
-    for (long long t = t_begin; t < t_end && ok && lane == 0; ++t) {
-      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
-      if (py != cur_py) { cur_py = py; const long long prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap); }
-      if (ti * kTile >= cnt) continue;
-      const int head_row = (int)((((size_t)b * dev.G + l) * dev.H_kv + g) * kDP);
+    TileIter cur;
+    iter_begin(cur);
+    while (ok && lane == 0 && iter_next(cur, no_op)) {
+      const int head_row = (int)((((size_t)cur.b * dev.G + cur.l) * dev.H_kv + cur.g) * kDP);
+      uint32_t my = 0;
 #pragma unroll 1
-      for (int phase = 0; phase < 2 && ok; ++phase) {
-        const int r = phase ? dev.r_v : dev.r_k;
-        const CUtensorMap* map = phase ? &bv_map : &bk_map;
-        const int nks = (r + 63) >> 6;
-#pragma unroll 1
-        for (int ks = 0; ks < nks; ++ks) {
-          if (n_issued >= kNB) {
-            if (!wait_bar(ctx, BAR(bl.empty + (xslot >> 1)), xpar, 17)) { ok = false; break; }
-            if (++xslot == S) { xslot = 0; xpar ^= 1u; }
-          }
-          ++n_issued;
-          mbar_expect_tx(BAR(bl.bfull + bslot), kSlabBytes);
-          tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, map, ks * 64, head_row, BAR(bl.bfull + bslot));
-          if (++bslot == kNB) bslot = 0;
+      for (int ks = 0; ks < nks_k; ++ks) {
+        int sl = slot + ks;
+        while (sl >= S) sl -= S;
+        if ((ks & 1) == 0) {             // key stages start on even slots: entering a slot pair
+          const int pr = sl >> 1;
+          my = (uint32_t)pr | (((cnt_k >> pr) & 1u) << 3);
+          cnt_k ^= 1u << pr;
         }
+        if (ks >= kNB) {
+          const uint32_t e = (fifo >> (4 * bslot)) & 15u;
+          if (!wait_bar(ctx, BAR(bl.emptyk + (int)(e & 7u)), e >> 3, 17)) { ok = false; break; }
+        } else if (it > 0 && it * nks_k + ks >= kNB) {
+          if (!wait_bar(ctx, BAR(bl.kfull + ((it - 1) & 1)), (uint32_t)(((it - 1) >> 1) & 1), 18)) { ok = false; break; }
+        }
+        fifo = (fifo & ~(15u << (4 * bslot))) | (my << (4 * bslot));
+        mbar_expect_tx(BAR(bl.bfull + bslot), kSlabBytes);
+        tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, &bk_map, ks * 64, head_row, BAR(bl.bfull + bslot));
+        if (++bslot == kNB) bslot = 0;
       }
+      // ring order is K(0), K(1), V(0), K(2), V(1), ...: every key phase but the first is followed by a value phase
+      slot += nst_k + (it > 0 ? nst_v : 0);
+      while (slot >= S) slot -= S;
+      ++it;
     }
   } else if (warp < 4) {
-    // =============================== key epilogue: rope, logits, softmax statistics ===============================
+    // =============================== key epilogue: rope, logits, softmax statistics, weights ===============================
     const int j = tid;                                  // tile row = TMEM lane
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     const float scale2 = dev.att_scale * kLog2e;
     const int rmask = (1 << dev.rope_shift) - 1;
     float m_run[NR], l_thr[NR];
-    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
-    long long prob = 0;
+    int it = 0;
     bool ok = true;
     uint32_t grp_par = 0;
     const int ps = warp == 0 ? 24 : -1000;
     const long long role_t0 = clock64();
+    // where this row's weights go in the bf16 operand tile: [row block j/64][head][64 rows], 128-byte swizzle
+    const uint32_t p_off = (uint32_t)(j >> 6) * 2048u + (uint32_t)(j & 7) * 2u;
+    const uint32_t p_unit = (uint32_t)((j & 63) >> 3);
     // barrier among the 128 threads of this role, with the same bounded wait as every other wait
     auto group_sync = [&]() {
       mbar_arrive(BAR(bl.grp));
       if (!wait_bar(ctx, BAR(bl.grp), grp_par, ps + 3)) ok = false;
       grp_par ^= 1u;
     };
-    auto flush = [&]() {   // end of a segment: write (m, l) of every head to the problem's partial slot
+    TileIter cur;
+    iter_begin(cur);
+    auto flush = [&](int py) {   // end of a segment: write (m, l) of every head to the problem's partial slot
       float tot[NR];
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
@@ -466,30 +577,27 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       }
       group_sync();
       if (j < n_rep) {
-        const long long first = (long long)cur_py * sc.tpp;
-        const int seg = (int)blockIdx.x - cta_of_tile(first, C, N);
-        float* part = dev.part + (((size_t)prob * sc.n_slots + seg) * n_rep + j) * (DH + 2);
+        float* part = part_of(py, cur.prob) + (size_t)j * (dev.r_v + 2) + dev.r_v;
         float ls = 0.0f, mm = -INFINITY;
 #pragma unroll
         for (int h = 0; h < NR; ++h) {
           if (h == j) { ls = red_s[h] + red_s[NR + h] + red_s[2 * NR + h] + red_s[3 * NR + h]; mm = m_run[h]; }
         }
-        part[DH] = mm;
-        part[DH + 1] = ls;
+        part[0] = mm;
+        part[1] = ls;
       }
     };
-    for (long long t = t_begin; t < t_end && ok; ++t) {
-      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
-      if (py != cur_py) {
-        if (cur_py >= 0) flush();
-        cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap);
+    auto on_problem = [&](int py) {
+      if (cur.py >= 0) flush(cur.py);
+      int l, b, g;
+      prob_of(py, l, b, g);
 #pragma unroll
-        for (int h = 0; h < NR; ++h) { m_run[h] = -INFINITY; l_thr[h] = 0.0f; }
-        const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
-        for (int i = j; i < NR * DH; i += 128) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
-        group_sync();
-      }
-      if (ti * kTile >= cnt) continue;
+      for (int h = 0; h < NR; ++h) { m_run[h] = -INFINITY; l_thr[h] = 0.0f; }
+      const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
+      for (int i = j; i < NR * DH; i += 128) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
+      group_sync();
+    };
+    while (ok && iter_next(cur, on_problem)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
       if (!wait_bar(ctx, BAR(bl.posfull + buf), par, ps + 1)) { ok = false; break; }   // positions published
@@ -530,84 +638,82 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
       }
       group_sync();
       if (!ok) break;
-      if (!wait_bar(ctx, BAR(bl.pempty + buf), par ^ 1u, ps + 4)) { ok = false; break; }
+      // the weights buffer and the rescale factors of tile it-2 must have been consumed
+      if (!wait_bar(ctx, BAR(bl.wempty + buf), par ^ 1u, ps + 4)) { ok = false; break; }
+      uint8_t* Pw = P_gen + buf * kPBytes + p_off;
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
         const float tm = fmaxf(fmaxf(red[h], red[NR + h]), fmaxf(red[2 * NR + h], red[3 * NR + h]));
         const float m_new = fmaxf(m_run[h], tm);
         const float alpha = (m_run[h] == -INFINITY) ? 0.0f : exp2f(m_run[h] - m_new);
         const float p = (m_new == -INFINITY) ? 0.0f : exp2f(z[h] - m_new);
-        l_thr[h] = l_thr[h] * alpha + p;
+        const __nv_bfloat16 pb = __float2bfloat16(p);
+        l_thr[h] = l_thr[h] * alpha + __bfloat162float(pb);   // the denominator sums the weights as they are used
         m_run[h] = m_new;
-        P_s[(buf * NR + h) * kTile + j] = p;
+        if (h < n_rep) *reinterpret_cast<__nv_bfloat16*>(Pw + h * 128 + ((p_unit ^ (uint32_t)(h & 7)) << 4)) = pb;
         if (j == h) alpha_s[buf * NR + h] = alpha;
       }
+      fence_proxy_async();                              // the weights are read by the tensor core
       mbar_arrive(BAR(bl.pfull + buf));
       ++it;
     }
-    if (ok && cur_py >= 0) flush();
+    if (ok && cur.py >= 0) flush(cur.py);
     if (ctx.prof && j == 0) ctx.prof[24] = (unsigned long long)(clock64() - role_t0);
   } else {
-    // =============================== value epilogue: o += p * V_hat ===============================
-    const int dd = tid - 128;                           // output column = TMEM lane
+    // =============================== value epilogue: running W = W * alpha + W_tile ===============================
+    const int mm = tid - 128;                           // rank column inside a 128-column block = TMEM lane
     const uint32_t lane_base = (uint32_t)((warp - 4) * 32) << 16;
-    float o[NR];
+    const int nblk = (dev.r_v + 127) >> 7;
+    float w[WB][NR];
     const int ps = warp == 4 ? 32 : -1000;
     const long long role_t0 = clock64();
-    int it = 0, cur_py = -1, cnt = 0, l = 0, b = 0, g = 0;
-    long long prob = 0;
+    int it = 0;
     bool ok = true;
-    auto flush = [&]() {
-      if (dd < DH) {
-        const long long first = (long long)cur_py * sc.tpp;
-        const int seg = (int)blockIdx.x - cta_of_tile(first, C, N);
-        float* part = dev.part + ((size_t)prob * sc.n_slots + seg) * n_rep * (DH + 2);
+    TileIter cur;
+    iter_begin(cur);
+    auto flush = [&](int py) {
+      float* part = part_of(py, cur.prob);
 #pragma unroll
-        for (int h = 0; h < NR; ++h) if (h < n_rep) part[h * (DH + 2) + dd] = o[h];
+      for (int bk = 0; bk < WB; ++bk) {
+        const int col = bk * 128 + mm;
+        if (bk < nblk && col < dev.r_v) {
+#pragma unroll
+          for (int h = 0; h < NR; ++h) if (h < n_rep) part[(size_t)h * (dev.r_v + 2) + col] = w[bk][h];
+        }
       }
     };
-    for (long long t = t_begin; t < t_end && ok; ++t) {
-      const int py = (int)(t / sc.tpp), ti = (int)(t % sc.tpp);
-      if (py != cur_py) {
-        if (cur_py >= 0) flush();
-        cur_py = py; prob = prob_of(py, l, b, g); cnt = min(sel_cnt[prob], sc.k_cap);
+    auto on_problem = [&](int) {
+      if (cur.py >= 0) flush(cur.py);
 #pragma unroll
-        for (int h = 0; h < NR; ++h) o[h] = 0.0f;
-      }
-      if (ti * kTile >= cnt) continue;
+      for (int bk = 0; bk < WB; ++bk)
+#pragma unroll
+        for (int h = 0; h < NR; ++h) w[bk][h] = 0.0f;
+    };
+    while (ok && iter_next(cur, on_problem)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
-      if (!wait_bar(ctx, BAR(bl.pfull + buf), par, ps + 1)) { ok = false; break; }
-      if (!wait_bar(ctx, BAR(bl.vfull + buf), par, ps + 2)) { ok = false; break; }
+      if (!wait_bar(ctx, BAR(bl.wfull + buf), par, ps + 1)) { ok = false; break; }
       tc_fence_after();
+      float al[NR];
 #pragma unroll
-      for (int h = 0; h < NR; ++h) o[h] *= alpha_s[buf * NR + h];
-      const uint32_t acc = tmem + lane_base + (uint32_t)(256 + buf * 128);
-      const float* P = P_s + buf * NR * kTile;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        float v[32];
-        tmem_ld32(acc + (uint32_t)(ch * 32), v);
-        tc_wait_ld();
+      for (int h = 0; h < NR; ++h) al[h] = alpha_s[buf * NR + h];
+      const uint32_t acc = tmem + lane_base + 256u + (uint32_t)(buf * 128);
 #pragma unroll
-        for (int j4 = 0; j4 < 8; ++j4) {
+      for (int bk = 0; bk < WB; ++bk) {
+        if (bk < nblk) {
+          float v[NR];
+          tmem_ld<NR>(acc + (uint32_t)(bk * 16), v);
+          tc_wait_ld();
 #pragma unroll
-          for (int h = 0; h < NR; ++h) {
-            const float4 p4 = *reinterpret_cast<const float4*>(P + h * kTile + ch * 32 + j4 * 4);
-            o[h] = fmaf(p4.x, v[j4 * 4 + 0], o[h]);
-            o[h] = fmaf(p4.y, v[j4 * 4 + 1], o[h]);
-            o[h] = fmaf(p4.z, v[j4 * 4 + 2], o[h]);
-            o[h] = fmaf(p4.w, v[j4 * 4 + 3], o[h]);
-          }
+          for (int h = 0; h < NR; ++h) w[bk][h] = fmaf(w[bk][h], al[h], v[h]);
         }
       }
       tc_fence_before();
-      mbar_arrive(BAR(bl.vempty + buf));
-      mbar_arrive(BAR(bl.pempty + buf));
+      mbar_arrive(BAR(bl.wempty + buf));
       ++it;
     }
-    if (ok && cur_py >= 0) flush();
-    if (ctx.prof && dd == 0) ctx.prof[32] = (unsigned long long)(clock64() - role_t0);
+    if (ok && cur.py >= 0) flush(cur.py);
+    if (ctx.prof && mm == 0) ctx.prof[32] = (unsigned long long)(clock64() - role_t0);
   }
 
   // wind down: nothing of this CTA may still touch shared or tensor memory
@@ -620,12 +726,20 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, const __grid_constan
   }
 }
 
-// Partials of a problem -> out, lse.  grid.x = problems * n_rep, blockDim = DH.  m is in log2 units.
+// Partials of a problem -> out, lse.  grid.x = problems * n_rep, 1024 threads.  m is in log2 units.
+// W_h = sum_seg 2^(m_seg - M) W_seg[h], L = sum_seg 2^(m_seg - M) l_seg, then
+// out_h[d] = (1/L) sum_m W_h[m] B_v[m][g*d_h + d]   (Eq. 3 applied once to the weighted sum of basis rows).
+// DH/8 threads read one 16-byte piece each of a B_v row; 1024/(DH/8) rows are in flight per pass.
+constexpr int kMergeThreads = 1024;
 template <int DH>
-__global__ void __launch_bounds__(DH)
-merge_segments_kernel(GroupDev dev, Sched sc, const int32_t* __restrict__ sel_cnt, __nv_bfloat16* __restrict__ out,
-                      float* __restrict__ lse) {
-  const int n_rep = dev.n_rep;
+__global__ void __launch_bounds__(kMergeThreads)
+merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+  extern __shared__ float m_s[];                      // [r_v] weights-times-basis, then [rows per pass][DH] partial sums
+  constexpr int TPR = DH / 8, RPP = kMergeThreads / TPR;
+  const int n_rep = dev.n_rep, r = dev.r_v;
+  float* w_s = m_s;
+  float* red = m_s + ((r + 3) & ~3);
+  const int tid = threadIdx.x;
   const int h = blockIdx.x % n_rep, py = blockIdx.x / n_rep;
   const int per_layer = dev.batch * dev.H_kv;
   const int g = py % dev.H_kv, b = (py / dev.H_kv) % dev.batch, l = sc.l0 + py / per_layer;
@@ -633,23 +747,56 @@ merge_segments_kernel(GroupDev dev, Sched sc, const int32_t* __restrict__ sel_cn
   const long long first = (long long)py * sc.tpp;
   const int c0 = cta_of_tile(first, sc.n_ctas, sc.n_tiles), c1 = cta_of_tile(first + sc.tpp - 1, sc.n_ctas, sc.n_tiles);
   const int nseg = c1 - c0 + 1;
-  const float* part = dev.part + ((size_t)prob * sc.n_slots) * n_rep * (DH + 2) + (size_t)h * (DH + 2);
-  const size_t stride = (size_t)n_rep * (DH + 2);
+  const size_t stride = (size_t)n_rep * (r + 2);
+  const float* part = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h * (r + 2);
   float M = -INFINITY;
-  for (int s = 0; s < nseg; ++s) M = fmaxf(M, part[s * stride + DH]);
-  float L = 0.0f, o = 0.0f;
+  for (int s = 0; s < nseg; ++s) M = fmaxf(M, part[s * stride + r]);
+  float L = 0.0f;
+  for (int m = tid; m < r; m += kMergeThreads) {
+    float acc = 0.0f;
+    if (M != -INFINITY) {
+      for (int s = 0; s < nseg; ++s) {
+        const float ms = part[s * stride + r];
+        if (ms != -INFINITY) acc += exp2f(ms - M) * part[s * stride + m];
+      }
+    }
+    w_s[m] = acc;
+  }
   if (M != -INFINITY) {
     for (int s = 0; s < nseg; ++s) {
-      const float ms = part[s * stride + DH];
-      if (ms == -INFINITY) continue;
-      const float w = exp2f(ms - M);
-      L += w * part[s * stride + DH + 1];
-      o += w * part[s * stride + threadIdx.x];
+      const float ms = part[s * stride + r];
+      if (ms != -INFINITY) L += exp2f(ms - M) * part[s * stride + r + 1];
     }
   }
-  const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
-  out[qh * DH + threadIdx.x] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
-  if (lse && threadIdx.x == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  __syncthreads();
+  const int rg = tid / TPR, dg = tid % TPR;
+  const size_t ld = (size_t)dev.H_kv * DH;
+  const __nv_bfloat16* Bv = dev.B_v + (((size_t)b * dev.G + l) * r) * ld + (size_t)g * DH + dg * 8;
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+#pragma unroll 4
+  for (int m = rg; m < r; m += RPP) {
+    const uint4 v = *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld);
+    const float w = w_s[m];
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      acc[2 * e] = fmaf(w, __uint_as_float(u[e] << 16), acc[2 * e]);
+      acc[2 * e + 1] = fmaf(w, __uint_as_float(u[e] & 0xffff0000u), acc[2 * e + 1]);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[rg * DH + dg * 8 + e] = acc[e];
+  __syncthreads();
+  if (tid < DH) {
+    float o = 0.0f;
+#pragma unroll 8
+    for (int i = 0; i < RPP; ++i) o += red[i * DH + tid];
+    const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
+    out[qh * DH + tid] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+    if (lse && tid == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
 }
 
 template <int DH, int NR>
@@ -657,7 +804,7 @@ constexpr size_t fused_smem_bytes() {
   return 1024 + (size_t)(ring_slots<DH, NR>() + kNB) * kSlabBytes + misc_smem_bytes<DH, NR>();
 }
 
-template <int DH, int NR>
+template <int DH, int NR, int WB>
 cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
                            const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
   const GroupDev& dev = grp->dev;
@@ -670,19 +817,22 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   sc.n_slots = fused_slots(grp);
   sc.k_cap = k_cap;
   sc.prof = grp->prof;
-  static_assert(bar_layout(ring_slots<DH, NR>()).total <= 2 * 16 + 2 * kNB + 20, "barrier space");
+  static_assert(bar_layout(ring_slots<DH, NR>()).total <= 2 * 16 + kNB + 24, "barrier space");
   static_assert(kNB >= 2 && kNB < ring_slots<DH, NR>(), "B ring must be shorter than the row ring");
+  static_assert(NR * WB <= 64 && WB <= kMaxBlocks, "value epilogue registers");
   const size_t smem = fused_smem_bytes<DH, NR>();
-  cudaError_t e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  CUtensorMap mk, mv;
+  CUtensorMap mk;
   memcpy(&mk, grp->bk_tmap, sizeof(mk));
-  memcpy(&mv, grp->bv_tmap, sizeof(mv));
-  sr_fused_kernel<DH, NR><<<sc.n_ctas, kThreads, smem, s>>>(mk, mv, dev, sc, q, sel_idx, sel_cnt);
+  sr_fused_kernel<DH, NR, WB><<<sc.n_ctas, kThreads, smem, s>>>(mk, dev, sc, q, sel_idx, sel_cnt);
   count_launch();
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  merge_segments_kernel<DH><<<problems * dev.n_rep, DH, 0, s>>>(dev, sc, sel_cnt, out, lse);
+  const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
+  e = cudaFuncSetAttribute(merge_segments_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
+  if (e != cudaSuccess) return e;
+  merge_segments_kernel<DH><<<problems * dev.n_rep, kMergeThreads, msmem, s>>>(dev, sc, out, lse);
   count_launch();
   return cudaGetLastError();
 }
@@ -696,16 +846,22 @@ int fused_slots(const xkv_group* grp) {
 
 size_t fused_part_floats(const xkv_group* grp) {
   const xkv_group_config& c = grp->cfg;
-  return (size_t)c.G * c.batch * c.H_kv * fused_slots(grp) * (size_t)(c.H_q / c.H_kv) * (c.d_h + 2);
+  return (size_t)c.G * c.batch * c.H_kv * fused_slots(grp) * (size_t)(c.H_q / c.H_kv) * (c.r_v + 2);
+}
+
+// The tensor-core path covers r_v up to 1024 (512 with more than 8 query heads per KV head).
+bool fused_supported(const xkv_group* grp) {
+  const int n_rep = grp->dev.n_rep, blocks = (grp->dev.r_v + 127) / 128;
+  return blocks <= (n_rep <= 8 ? 8 : 4);
 }
 
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
                          const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
   const int n_rep = grp->dev.n_rep;
-#define XKV_DISPATCH(DH)                                                                              \
-  if (n_rep <= 4) return launch_fused_t<DH, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
-  if (n_rep <= 8) return launch_fused_t<DH, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
-  return launch_fused_t<DH, 16>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);
+#define XKV_DISPATCH(DH)                                                                                 \
+  if (n_rep <= 4) return launch_fused_t<DH, 4, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
+  if (n_rep <= 8) return launch_fused_t<DH, 8, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
+  return launch_fused_t<DH, 16, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);
   if (grp->dev.d_h == 128) { XKV_DISPATCH(128) }
   XKV_DISPATCH(64)
 #undef XKV_DISPATCH

@@ -27,6 +27,7 @@ struct GroupDev {
   const __nv_bfloat16* landmarks;   // [batch][G][H_kv][n_c][d_h]
   const __nv_bfloat16* Bt_k;        // [batch][G][H_kv][kDP][r_k]  transposed head blocks, zero padded
   const __nv_bfloat16* Bt_v;        // [batch][G][H_kv][kDP][r_v]
+  const __nv_bfloat16* B_v;         // [batch][G][r_v][H_kv*d_h]   owned copy in the caller's layout
   const float2* rope_hi;            // [n_hi][d_h/2]          (cos, sin) of (p_hi << rope_shift) * theta_i
   const float2* rope_lo;            // [2^rope_shift][d_h/2]  (cos, sin) of p_lo * theta_i
   float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
@@ -78,6 +79,7 @@ cudaError_t launch_reconstruct_attend(const xkv_group* grp, int l0, int l1, cons
 // xkv_fused.cu
 int fused_slots(const xkv_group* grp);
 size_t fused_part_floats(const xkv_group* grp);
+bool fused_supported(const xkv_group* grp);
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
                          const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s);
 
