@@ -52,7 +52,8 @@ typedef enum {
   XKV_ERR_CUDA = -4,        /* a CUDA runtime call failed; see xkv_last_cuda_error */
   XKV_ERR_OOM = -5,         /* device allocation for the handle failed */
   XKV_ERR_INDEX_RANGE = -6, /* device flag: a selected row was outside [0,T) and was skipped */
-  XKV_ERR_TIMEOUT = -7      /* device flag: a bounded wait inside a kernel ran out */
+  XKV_ERR_TIMEOUT = -7,     /* device flag: a bounded wait inside a kernel ran out */
+  XKV_ERR_TOO_LARGE = -8    /* xkv_sr_select_static: the call needs more than its fixed scratch */
 } xkv_status;
 
 /* Bits of the device flag word returned by xkv_group_status. */
@@ -160,6 +161,42 @@ XKV_API int xkv_last_cuda_error(void);
 
 /* Number of kernels the library has launched since load (all handles); for launch accounting. */
 XKV_API uint64_t xkv_kernel_launch_count(void);
+
+/*
+ * Chunk selection for callers that must not allocate device memory.  (The paper has no counterpart: this is a
+ * packaging variant of xkv_sr_select, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving loop whose memory pool owns
+ * every byte of the device, under an allocator that forbids side allocations, or in a process that may only
+ * use memory handed to it.  xkv_group_create allocates (pooled scores, repacked matrices, tables); this entry
+ * point takes no handle and allocates nothing, neither with cudaMalloc/cudaFree nor through any library.
+ *
+ * Where the scratch lives: the pooled landmark scores go to a fixed array inside the library image
+ * (XKV_STATIC_SELECT_MAX_SCORES floats, 4 MiB, plus 256 bytes of flag words).  Every GPU that loads the library
+ * carries that array until the process exits.  A call needs G*batch*H_kv*ceil(T/c) scores; if that is more than
+ * the array holds, the call does nothing and returns XKV_ERR_TOO_LARGE.
+ *
+ * First call on a device: the library looks up the array's device address (once per device, for the device
+ * that is current at the call) before it launches anything.  Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, which keeps the previous call's scores; the flag words are
+ * cleared at the start of each call.  Two calls whose kernels overlap on the GPU (different streams, or
+ * different host threads) race on it: serialise them.  Device-side give-ups (a bounded wait that ran out) are
+ * not reported by this entry point.
+ *
+ * cfg       host struct; landmarks as in xkv_group_config (bf16 [batch][G][H_kv][n_c][d_h], device, 16-byte aligned).
+ * other arguments, outputs and tie rules: exactly those of xkv_sr_select (k_cap = ceil(k/c)*c is the row stride).
+ * Errors: INVALID_ARG, TOO_LARGE, ARCH, CUDA.
+ */
+#define XKV_STATIC_SELECT_MAX_SCORES (1u << 20)
+typedef struct {
+  uint32_t struct_size; /* sizeof(xkv_select_static_config) */
+  int32_t G, batch, T, H_kv, H_q, d_h;
+  int32_t chunk;        /* 0 means 8 */
+  const void* landmarks;
+} xkv_select_static_config;
+XKV_API int xkv_sr_select_static(const xkv_select_static_config* cfg, int layer_begin, int layer_end, const void* q,
+                                 int32_t k, int32_t* sel_idx, int32_t* sel_cnt, void* stream);
 
 /*
  * Diagnostic.  If the environment variable XKV_FUSED_PROF=1 was set when the handle was created, the

@@ -70,6 +70,10 @@ static bool encode_rows64(void* out, const void* base, uint64_t rows, uint64_t c
   return r == CUDA_SUCCESS;
 }
 
+bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols) {
+  return encode_rows64(out, base, rows, cols, 256);
+}
+
 }  // namespace xkv
 
 using namespace xkv;
@@ -97,6 +101,7 @@ const char* xkv_strerror(int s) {
     case XKV_ERR_OOM: return "out of device memory";
     case XKV_ERR_INDEX_RANGE: return "a selected row index was outside [0,T) and was skipped";
     case XKV_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case XKV_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the allocation-free entry point";
     default: return "unknown status";
   }
 }
@@ -243,6 +248,11 @@ int xkv_group_status(xkv_group* g, uint32_t* device_flags, void* stream) {
   if (f & XKV_FLAG_TIMEOUT) return XKV_ERR_TIMEOUT;
   if (f & XKV_FLAG_INDEX_RANGE) return XKV_ERR_INDEX_RANGE;
   return XKV_OK;
+}
+
+int xkv_sr_select_static(const xkv_select_static_config* cfg, int layer_begin, int layer_end, const void* q,
+                         int32_t k, int32_t* sel_idx, int32_t* sel_cnt, void* stream) {
+  return select_static(cfg, layer_begin, layer_end, q, k, sel_idx, sel_cnt, (cudaStream_t)stream);
 }
 
 int xkv_debug_read_profile(xkv_group* g, uint64_t* out, int max_words) {

@@ -70,6 +70,11 @@ cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift,
 cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
                           int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
 
+int select_static(const xkv_select_static_config* c, int l0, int l1, const void* q, int32_t k, int32_t* sel_idx,
+                  int32_t* sel_cnt, cudaStream_t s);
+// xkv_api.cu: tensor map over [rows][cols] bf16 landmarks, 256-row boxes of 64 columns, 128-byte swizzle
+bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols);
+
 // xkv_attend.cu
 size_t attend_part_floats(const xkv_group* grp);
 cudaError_t launch_reconstruct_attend(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q,

@@ -5,6 +5,9 @@
 //                      compaction (ties to the lowest chunk index, output ascending) and expansion of
 //                      chunk ids to token rows.
 #include <cuda.h>
+#include <math.h>
+
+#include <mutex>
 
 #include "xkv_internal.cuh"
 
@@ -384,17 +387,15 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
 
 }  // namespace
 
-cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
-                          int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
-  const GroupDev& dev = grp->dev;
+// Both kernels of the selection for the problems of layers [l0, l1); `tmap` describes dev.landmarks.
+static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tmap, int l0, int l1,
+                                     const __nv_bfloat16* q, int k, int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
   const int problems = (l1 - l0) * dev.batch * dev.H_kv;
   const int tiles = (dev.n_c + kScoreRows - 1) / kScoreRows;
   const int c = dev.c;
   const int k_ch_raw = (k + c - 1) / c;
   const int k_ch = k_ch_raw < dev.n_c ? k_ch_raw : dev.n_c;
   const int k_cap = k_ch_raw * c;
-  CUtensorMap tmap;
-  memcpy(&tmap, grp->lm_tmap, sizeof(tmap));
   const size_t smem = 1024 + (size_t)(dev.d_h / 64) * kScoreRows * 128 + (size_t)dev.n_rep * dev.d_h * 4;
   dim3 grid(tiles, problems);
   cudaError_t e;
@@ -416,6 +417,77 @@ cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloa
     topk_kernel<false><<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
   count_launch();
   return cudaGetLastError();
+}
+
+cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
+                          int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
+  CUtensorMap tmap;
+  memcpy(&tmap, grp->lm_tmap, sizeof(tmap));
+  return launch_select_dev(grp->dev, tmap, l0, l1, q, k, sel_idx, sel_cnt, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Selection without a handle and without any allocation: the pooled scores live in a file-scope device array.
+
+// 64 flag words followed by the pooled scores of every problem of the call.
+static __device__ __align__(256) float g_static_scratch[64 + XKV_STATIC_SELECT_MAX_SCORES];
+
+// The array's name is only a host-side stand-in; its device address is looked up once per device.
+static float* static_scratch_ptr(int device, cudaError_t* err) {
+  static std::mutex mu;
+  static float* ptrs[64] = {};
+  std::lock_guard<std::mutex> lock(mu);
+  *err = cudaSuccess;
+  if (device < 0 || device >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
+  if (!ptrs[device]) {
+    float* p = nullptr;
+    *err = cudaGetSymbolAddress((void**)&p, g_static_scratch);   // the current device is `device`
+    if (*err != cudaSuccess) return nullptr;
+    ptrs[device] = p;
+  }
+  return ptrs[device];
+}
+
+int select_static(const xkv_select_static_config* c, int l0, int l1, const void* q, int32_t k, int32_t* sel_idx,
+                  int32_t* sel_cnt, cudaStream_t s) {
+  if (!c || !q || !sel_idx || !sel_cnt || c->struct_size != sizeof(xkv_select_static_config)) return XKV_ERR_INVALID_ARG;
+  if (c->G < 1 || c->batch < 1 || c->T < 1 || c->T >= (1 << 24) || c->H_kv < 1 || c->H_q < 1 ||
+      c->H_q % c->H_kv != 0 || c->H_q / c->H_kv > kMaxRep || (c->d_h != 64 && c->d_h != 128) || c->chunk < 0 ||
+      c->chunk > 4096 || !c->landmarks || ((uintptr_t)c->landmarks & 15u) || ((uintptr_t)q & 15u) ||
+      ((uintptr_t)sel_idx & 3u) || ((uintptr_t)sel_cnt & 3u))
+    return XKV_ERR_INVALID_ARG;
+  if (l0 < 0 || l1 > c->G || l0 >= l1 || k < 1) return XKV_ERR_INVALID_ARG;
+  GroupDev dev{};
+  dev.G = c->G; dev.batch = c->batch; dev.T = c->T; dev.H_kv = c->H_kv; dev.H_q = c->H_q; dev.d_h = c->d_h;
+  dev.c = c->chunk ? c->chunk : 8;
+  dev.n_c = (c->T + dev.c - 1) / dev.c;
+  dev.n_rep = c->H_q / c->H_kv;
+  dev.sel_scale = 1.0f / sqrtf((float)c->d_h);
+  dev.landmarks = (const __nv_bfloat16*)c->landmarks;
+  const size_t scores = (size_t)c->G * c->batch * c->H_kv * dev.n_c;   // indexed by absolute layer, like the handle's
+  if (scores > (size_t)XKV_STATIC_SELECT_MAX_SCORES) return XKV_ERR_TOO_LARGE;
+  int device = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+  cudaDeviceProp prop;
+  static int cc_major[64] = {};
+  if (device >= 0 && device < 64 && cc_major[device] == 0) {
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+    cc_major[device] = prop.major;
+  }
+  if (device < 0 || device >= 64 || cc_major[device] != 10) return XKV_ERR_ARCH;
+  float* scratch = static_scratch_ptr(device, &e);
+  if (!scratch) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  dev.flags = reinterpret_cast<unsigned int*>(scratch);
+  dev.pooled = scratch + 64;
+  CUtensorMap tmap;
+  if (!encode_landmark_map(&tmap, c->landmarks, (uint64_t)c->batch * c->G * c->H_kv * dev.n_c, (uint64_t)c->d_h))
+    return XKV_ERR_CUDA;
+  e = cudaMemsetAsync(scratch, 0, 64 * sizeof(float), s);              // the flag words start at zero
+  if (e == cudaSuccess) e = launch_select_dev(dev, tmap, l0, l1, (const __nv_bfloat16*)q, k, sel_idx, sel_cnt, s);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
 }
 
 }  // namespace xkv

@@ -30,6 +30,7 @@ XKV_ERR_CUDA = -4
 XKV_ERR_OOM = -5
 XKV_ERR_INDEX_RANGE = -6
 XKV_ERR_TIMEOUT = -7
+XKV_ERR_TOO_LARGE = -8
 XKV_FLAG_INDEX_RANGE = 1
 XKV_FLAG_TIMEOUT = 2
 
@@ -48,6 +49,17 @@ class xkv_group_config(ctypes.Structure):
     ]
 
 
+class xkv_select_static_config(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("G", ctypes.c_int32), ("batch", ctypes.c_int32), ("T", ctypes.c_int32),
+        ("H_kv", ctypes.c_int32), ("H_q", ctypes.c_int32), ("d_h", ctypes.c_int32),
+        ("chunk", ctypes.c_int32),
+        ("landmarks", ctypes.c_void_p),
+    ]
+
+
+XKV_STATIC_SELECT_MAX_SCORES = 1 << 20
 _P = ctypes.c_void_p
 _lib.xkv_group_create.argtypes = [ctypes.POINTER(xkv_group_config), _P, ctypes.POINTER(_P)]
 _lib.xkv_group_create.restype = ctypes.c_int
@@ -55,6 +67,9 @@ _lib.xkv_sr_select.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, ctypes.c_int3
 _lib.xkv_sr_select.restype = ctypes.c_int
 _lib.xkv_sr_reconstruct_attend.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, ctypes.c_int32, _P, _P, _P]
 _lib.xkv_sr_reconstruct_attend.restype = ctypes.c_int
+_lib.xkv_sr_select_static.argtypes = [ctypes.POINTER(xkv_select_static_config), ctypes.c_int, ctypes.c_int, _P,
+                                      ctypes.c_int32, _P, _P, _P]
+_lib.xkv_sr_select_static.restype = ctypes.c_int
 _lib.xkv_group_destroy.argtypes = [_P]
 _lib.xkv_group_destroy.restype = ctypes.c_int
 _lib.xkv_group_status.argtypes = [_P, ctypes.POINTER(ctypes.c_uint32), _P]
@@ -158,6 +173,20 @@ def xkv_sr_select(grp: Group, layer_begin: int, layer_end: int, q, k: int, sel_i
                             _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_sr_select")
+
+
+def xkv_sr_select_static(*, G, batch, T, H_kv, H_q, d_h, landmarks, layer_begin, layer_end, q, k, sel_idx, sel_cnt,
+                         chunk=8, stream=None) -> None:
+    """Selection without a handle and without any device allocation (fixed scratch inside the library, see
+    include/xkv.h).  Same outputs as xkv_sr_select.  Raises XKVError(XKV_ERR_TOO_LARGE) beyond the fixed size."""
+    cfg = xkv_select_static_config()
+    cfg.struct_size = ctypes.sizeof(xkv_select_static_config)
+    cfg.G, cfg.batch, cfg.T, cfg.H_kv, cfg.H_q, cfg.d_h, cfg.chunk = G, batch, T, H_kv, H_q, d_h, chunk
+    cfg.landmarks = _ptr(landmarks)
+    st = _lib.xkv_sr_select_static(ctypes.byref(cfg), layer_begin, layer_end, _ptr(q), k, _ptr(sel_idx), _ptr(sel_cnt),
+                                   _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_sr_select_static")
 
 
 def xkv_sr_reconstruct_attend(grp: Group, layer_begin: int, layer_end: int, q, sel_idx, sel_cnt, k_cap: int,
