@@ -236,6 +236,10 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // everything above is independent of the inputs; the selection (or whatever wrote q and the index sets) comes
+  // from earlier kernels of the stream
+  grid_dependency_wait();
+  grid_dependency_launch();
 
   const int C = sc.n_ctas, N = sc.n_tiles;
   const long long t_begin = ((long long)blockIdx.x * N) / C, t_end = ((long long)(blockIdx.x + 1) * N) / C;
@@ -731,10 +735,13 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 // out_h[d] = (1/L) sum_m W_h[m] B_v[m][g*d_h + d]   (Eq. 3 applied once to the weighted sum of basis rows).
 // DH/8 threads read one 16-byte piece each of a B_v row; 1024/(DH/8) rows are in flight per pass.
 constexpr int kMergeThreads = 1024;
+constexpr int kMergeMaxSeg = 160;                     // a problem never has more segments than there are CTAs + 1
 template <int DH>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
   extern __shared__ float m_s[];                      // [r_v] weights-times-basis, then [rows per pass][DH] partial sums
+  __shared__ float wgt_s[kMergeMaxSeg];
+  __shared__ float ML_s[2];
   constexpr int TPR = DH / 8, RPP = kMergeThreads / TPR;
   const int n_rep = dev.n_rep, r = dev.r_v;
   float* w_s = m_s;
@@ -746,53 +753,81 @@ merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, f
   const long long prob = ((long long)l * dev.batch + b) * dev.H_kv + g;
   const long long first = (long long)py * sc.tpp;
   const int c0 = cta_of_tile(first, sc.n_ctas, sc.n_tiles), c1 = cta_of_tile(first + sc.tpp - 1, sc.n_ctas, sc.n_tiles);
-  const int nseg = c1 - c0 + 1;
+  const int nseg = min(c1 - c0 + 1, kMergeMaxSeg);
   const size_t stride = (size_t)n_rep * (r + 2);
-  const float* part = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h * (r + 2);
-  float M = -INFINITY;
-  for (int s = 0; s < nseg; ++s) M = fmaxf(M, part[s * stride + r]);
-  float L = 0.0f;
-  for (int m = tid; m < r; m += kMergeThreads) {
-    float acc = 0.0f;
-    if (M != -INFINITY) {
-      for (int s = 0; s < nseg; ++s) {
-        const float ms = part[s * stride + r];
-        if (ms != -INFINITY) acc += exp2f(ms - M) * part[s * stride + m];
-      }
-    }
-    w_s[m] = acc;
-  }
-  if (M != -INFINITY) {
-    for (int s = 0; s < nseg; ++s) {
-      const float ms = part[s * stride + r];
-      if (ms != -INFINITY) L += exp2f(ms - M) * part[s * stride + r + 1];
-    }
-  }
-  __syncthreads();
+  // the B_v pieces do not depend on the partials: start those loads before anything else
   const int rg = tid / TPR, dg = tid % TPR;
   const size_t ld = (size_t)dev.H_kv * DH;
   const __nv_bfloat16* Bv = dev.B_v + (((size_t)b * dev.G + l) * r) * ld + (size_t)g * DH + dg * 8;
+  constexpr int kPre = 8;                             // rows of B_v held in registers per thread
+  uint4 pre[kPre];
+#pragma unroll
+  for (int i = 0; i < kPre; ++i) {
+    const int m = rg + i * RPP;
+    pre[i] = m < r ? *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld) : make_uint4(0, 0, 0, 0);
+  }
+  grid_dependency_wait();                             // the partials come from the kernel launched before this one
+  const float* part = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h * (r + 2);
+  if (tid < 32) {                                     // one warp: maxima, weights of the segments, denominator
+    float mx = -INFINITY;
+    for (int s = tid; s < nseg; s += 32) mx = fmaxf(mx, part[s * stride + r]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float Ls = 0.0f;
+    for (int s = tid; s < nseg; s += 32) {
+      const float ms = part[s * stride + r];
+      const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
+      wgt_s[s] = w;
+      Ls += w * part[s * stride + r + 1];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
+    if (tid == 0) { ML_s[0] = mx; ML_s[1] = Ls; }
+  }
+  __syncthreads();
+  for (int m = tid; m < r; m += kMergeThreads) {
+    float acc = 0.0f;
+    for (int s = 0; s < nseg; ++s) acc = fmaf(wgt_s[s], part[s * stride + m], acc);
+    w_s[m] = acc;
+  }
+  __syncthreads();
   float acc[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
-#pragma unroll 4
-  for (int m = rg; m < r; m += RPP) {
-    const uint4 v = *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld);
-    const float w = w_s[m];
+  auto add_row = [&](const uint4& v, float w) {
     const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       acc[2 * e] = fmaf(w, __uint_as_float(u[e] << 16), acc[2 * e]);
       acc[2 * e + 1] = fmaf(w, __uint_as_float(u[e] & 0xffff0000u), acc[2 * e + 1]);
     }
+  };
+#pragma unroll
+  for (int i = 0; i < kPre; ++i) {
+    const int m = rg + i * RPP;
+    if (m < r) add_row(pre[i], w_s[m]);
   }
+#pragma unroll 4
+  for (int m = rg + kPre * RPP; m < r; m += RPP) add_row(*reinterpret_cast<const uint4*>(Bv + (size_t)m * ld), w_s[m]);
 #pragma unroll
   for (int e = 0; e < 8; ++e) red[rg * DH + dg * 8 + e] = acc[e];
   __syncthreads();
+  // two-level sum over the row groups: 1024 threads fold RPP partials to 8 per column, then DH threads finish
+  constexpr int FOLD = kMergeThreads / DH;            // 8 (d_h = 128) or 16 (d_h = 64) threads per column
+  {
+    const int d = tid % DH, f = tid / DH;
+    float o = 0.0f;
+#pragma unroll 4
+    for (int i = f; i < RPP; i += FOLD) o += red[i * DH + d];
+    __syncthreads();
+    red[f * DH + d] = o;
+  }
+  __syncthreads();
   if (tid < DH) {
     float o = 0.0f;
-#pragma unroll 8
-    for (int i = 0; i < RPP; ++i) o += red[i * DH + tid];
+#pragma unroll
+    for (int f = 0; f < FOLD; ++f) o += red[f * DH + tid];
+    const float M = ML_s[0], L = ML_s[1];
     const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
     out[qh * DH + tid] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
     if (lse && tid == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
@@ -825,14 +860,14 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   if (e != cudaSuccess) return e;
   CUtensorMap mk;
   memcpy(&mk, grp->bk_tmap, sizeof(mk));
-  sr_fused_kernel<DH, NR, WB><<<sc.n_ctas, kThreads, smem, s>>>(mk, dev, sc, q, sel_idx, sel_cnt);
+  e = launch_pdl(sr_fused_kernel<DH, NR, WB>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   count_launch();
-  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
   e = cudaFuncSetAttribute(merge_segments_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
   if (e != cudaSuccess) return e;
-  merge_segments_kernel<DH><<<problems * dev.n_rep, kMergeThreads, msmem, s>>>(dev, sc, out, lse);
+  e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, out, lse);
+  if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
 }

@@ -58,6 +58,23 @@ struct xkv_group {
 namespace xkv {
 
 void set_cuda_error(cudaError_t e);
+
+// Launch with programmatic stream serialization: the kernel may begin while the previous kernel of the stream
+// drains; it must execute griddepcontrol.wait before it reads anything an earlier kernel may have written.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 void count_launch(int n = 1);
 
 // xkv_prep.cu

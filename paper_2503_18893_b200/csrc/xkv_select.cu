@@ -10,6 +10,7 @@
 #include <mutex>
 
 #include "xkv_internal.cuh"
+#include "xkv_ptx.cuh"
 
 namespace xkv {
 
@@ -19,32 +20,14 @@ constexpr int kScoreRows = 256;      // landmark rows (chunks) per CTA
 constexpr int kScoreThreads = 128;   // two rows per thread
 constexpr uint32_t kWaitLimit = 1u << 22;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+using namespace ptx;
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
 // Bounded wait: returns false if the phase did not complete within the limit.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
   for (uint32_t i = 0; i < kWaitLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -111,7 +94,7 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
 
   if (threadIdx.x == 0) {
     mbar_init(bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_mbar_init();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -120,6 +103,7 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
 #pragma unroll
     for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar);
   }
+  grid_dependency_launch();
   // queries of this KV head, widened to fp32 while the landmarks are in flight
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * dev.n_rep) * DH;
   for (int i = threadIdx.x; i < dev.n_rep * DH; i += kScoreThreads) qs[i] = __bfloat162float(qg[i]);
@@ -195,6 +179,8 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
   const int super = kTopkThreads * kTopkItems;
   const bool out_vec = (reinterpret_cast<uintptr_t>(out) & 15u) == 0;   // 16-byte stores of the row ids
 
+  grid_dependency_wait();                      // the pooled scores come from the kernel launched before
+  grid_dependency_launch();
   uint32_t creg[kTopkItems];
   if (CACHED) load_keys(S, tid * kTopkItems, n_c, creg);
 
@@ -412,11 +398,11 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (dev.n_c <= kTopkThreads * kTopkItems)
-    topk_kernel<true><<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
   else
-    topk_kernel<false><<<problems, kTopkThreads, 0, s>>>(dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
