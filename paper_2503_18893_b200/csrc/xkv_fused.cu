@@ -34,7 +34,7 @@ using namespace ptx;
 constexpr int kTile = 128;                       // selected rows per tile
 constexpr int kSlabBytes = kTile * 128;          // 128 rows x 64 bf16 (one 128-byte swizzle row each)
 constexpr int kNB = 4;                           // slots of the B-slab ring
-constexpr int kThreads = 14 * 32;
+constexpr int kThreads = 15 * 32;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kRopeStride = 66;                  // float2 per staged rotary row (64 + pad against bank conflicts)
 constexpr int kPBytes = 2 * 16 * 128;            // softmax weights of a tile as a bf16 MMA operand: [2][16 heads][64 rows]
@@ -396,12 +396,15 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     if (ctx.prof && pt == 0) { ctx.prof[0] = (unsigned long long)(clock64() - role_t0); ctx.prof[4] = (unsigned long long)it; }
-  } else if (warp == 12) {
-    // =============================== MMA issue ===============================
+  } else if (warp == 12 || warp == 14) {
+    // =============================== MMA issue: warp 12 the key phases, warp 14 the value phases ===============
+    // Both walk the same ring order; each steps over the other's stages.  Two issuing threads, because one thread
+    // spends 70-130 cycles per tcgen05.mma and about 235 per tcgen05.commit.
+    const bool kside = warp == 12;
     // the whole warp walks the loop (all values are warp-uniform); one lane issues the tensor-core instructions
     constexpr uint32_t idesc_k = idesc_bf16_f32(128, 128);                     // keys: both operands K-major
     constexpr uint32_t idesc_v = idesc_bf16_f32(128, 16) | (1u << 15);         // values: A is read along its rows (MN-major)
-    const int ps = 8;
+    const int ps = kside ? 8 : 40;
     const long long role_t0 = clock64();
     int slot = 0, bslot = 0;                          // positions in the two rings and their round parities
     uint32_t ring_par = 0, bring_par = 0;
@@ -423,7 +426,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       if (!do_k) more = false;
       // ---- keys: K_hat = A_k[S] B_k
       const long long ph0 = ctx.prof ? clock64() : 0;
-      if (do_k) {
+      if (do_k && !kside) {
+        slot += nst_k;
+        while (slot >= S) { slot -= S; ring_par ^= 1u; }
+        ++it;
+      } else if (do_k) {
         const int buf = it & 1;
         const uint32_t par = (uint32_t)((it >> 1) & 1);
         const int last_kk = (((dev.r_k - 1) & 63) >> 4) + 1;    // 16-column steps in the last real slab
@@ -452,7 +459,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
             if (ks == nst_k - 1) tc_commit(BAR(bl.kfull + buf));
           }
           __syncwarp();
-          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + 12, (unsigned long long)(clock64() - i0));
+          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
           if (++slot == S) { slot = 0; ring_par ^= 1u; }
           if (real && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
@@ -460,9 +467,13 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         ++it;
       }
       const long long ph1 = ctx.prof ? clock64() : 0;
-      if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + 14, (unsigned long long)(ph1 - ph0)); }
+      if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + ps + 6, (unsigned long long)(ph1 - ph0)); }
       // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
-      if (nv < it - (do_k ? 1 : 0)) {
+      if (nv < it - (do_k ? 1 : 0) && kside) {
+        slot += nst_v;
+        while (slot >= S) { slot -= S; ring_par ^= 1u; }
+        ++nv;
+      } else if (nv < it - (do_k ? 1 : 0)) {
         const int buf = nv & 1;
         const uint32_t par = (uint32_t)((nv >> 1) & 1);
         if (!wait_bar(ctx, BAR(bl.wempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
@@ -488,18 +499,18 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
             if (ks + 2 >= nst_v) tc_commit(BAR(bl.wfull + buf));
           }
           __syncwarp();
-          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + 12, (unsigned long long)(clock64() - i0));
+          if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
           slot += 2;
           if (slot == S) { slot = 0; ring_par ^= 1u; }
         }
         if (!ok) break;
         ++nv;
-        if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + 15, (unsigned long long)(clock64() - ph1)); }
+        if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + ps + 7, (unsigned long long)(clock64() - ph1)); }
       } else if (!do_k) {
         break;
       }
     }
-    if (ctx.prof && lane == 0) ctx.prof[8] = (unsigned long long)(clock64() - role_t0);
+    if (ctx.prof && lane == 0) ctx.prof[ps] = (unsigned long long)(clock64() - role_t0);
     __syncwarp();
   } else if (warp == 13) {
     // =============================== B_k slab loader (TMA) ===============================
