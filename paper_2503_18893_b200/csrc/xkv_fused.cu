@@ -54,13 +54,13 @@ struct Sched {
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, grp, total;
+  int full, fullv, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, grp, total;
 };
 __host__ __device__ constexpr Bars bar_layout(int na) {
   Bars b{};
   // one release barrier per slot pair and kind of occupant (key-phase or value-phase slabs): a waiter that knows
   // the kind it waits for is never confused by the other kind's completions
-  b.full = 0; b.emptyk = na; b.emptyv = na + na / 2; b.bfull = 2 * na; b.kfull = b.bfull + kNB;
+  b.full = 0; b.fullv = na; b.emptyk = 2 * na; b.emptyv = 2 * na + na / 2; b.bfull = 3 * na; b.kfull = b.bfull + kNB;
   b.kempty = b.kfull + 2; b.wfull = b.kempty + 2; b.wempty = b.wfull + 2; b.pfull = b.wempty + 2;
   b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.grp = b.posfull + 2; b.total = b.grp + 1;
   return b;
@@ -162,7 +162,7 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
 template <int DH, int NR>
 __host__ __device__ constexpr int misc_smem_bytes() {
   return (int)(2 * kPBytes + sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR + 8 * NR) +
-               sizeof(int) * (2 * kTile + 8) + 8 * (2 * 16 + kNB + 24) + 16);
+               sizeof(int) * (2 * kTile + 8) + 8 * (3 * 16 + kNB + 24) + 16);
 }
 // Slots of the gathered-row ring: whatever fits beside the B ring.
 template <int DH, int NR>
@@ -209,7 +209,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   const int nst_k = (nks_k + 1) & ~1, nst_v = (nks_v + 1) & ~1;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) mbar_init(BAR(bl.full + s), 128);
+    for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 128); mbar_init(BAR(bl.fullv + s), 128); }
     for (int s = 0; s < S / 2; ++s) { mbar_init(BAR(bl.emptyk + s), 1); mbar_init(BAR(bl.emptyv + s), 1); }
     for (int s = 0; s < kNB; ++s) mbar_init(BAR(bl.bfull + s), 1);
     for (int b = 0; b < 2; ++b) {
@@ -340,7 +340,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         const int adv = in ? ks * 64 : 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
-        cp_async_arrive_noinc(BAR(bl.full + slot));    // arrives when this thread's copies have landed
+        cp_async_arrive_noinc(BAR((phase ? bl.fullv : bl.full) + slot));   // arrives when this thread's copies have landed
         if (++slot == S) slot = 0;
       }
     };
@@ -407,7 +407,12 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     const int ps = kside ? 8 : 40;
     const long long role_t0 = clock64();
     int slot = 0, bslot = 0;                          // positions in the two rings and their round parities
-    uint32_t ring_par = 0, bring_par = 0;
+    uint32_t bring_par = 0;
+    // The `full` barriers are per slot and per kind of occupant (key-phase or value-phase slab), and this warp is
+    // the only one that releases its kind: it sees every phase of its barriers in order, so one parity bit per
+    // slot is enough.  With one barrier per slot for both kinds, the warp that steps over the other kind's stage
+    // could be lapped by it or test it too early, and a one-bit parity cannot tell those cases apart.
+    uint32_t seen = 0;
     // descriptors differ between slots only in the start-address field (units of 16 bytes)
     const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
     const uint32_t rows_lo0 = (uint32_t)(smem_desc_sw128(base, 0) & 0xFFFFFFFFull);
@@ -428,7 +433,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       const long long ph0 = ctx.prof ? clock64() : 0;
       if (do_k && !kside) {
         slot += nst_k;
-        while (slot >= S) { slot -= S; ring_par ^= 1u; }
+        while (slot >= S) slot -= S;
         ++it;
       } else if (do_k) {
         const int buf = it & 1;
@@ -441,7 +446,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         for (int ks = 0; ks < nst_k && ok; ++ks) {
           const bool real = ks < nks_k;
           if (real && !wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
-          if (!wait_bar(ctx, BAR(bl.full + slot), ring_par, ps + 3)) { ok = false; break; }
+          if (!wait_bar(ctx, BAR(bl.full + slot), (seen >> slot) & 1u, ps + 3)) { ok = false; break; }
+          seen ^= 1u << slot;
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
           if (lane == 0) {
@@ -460,7 +466,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           }
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
-          if (++slot == S) { slot = 0; ring_par ^= 1u; }
+          if (++slot == S) slot = 0;
           if (real && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
         if (!ok) break;
@@ -471,7 +477,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
       if (nv < it - (do_k ? 1 : 0) && kside) {
         slot += nst_v;
-        while (slot >= S) { slot -= S; ring_par ^= 1u; }
+        while (slot >= S) slot -= S;
         ++nv;
       } else if (nv < it - (do_k ? 1 : 0)) {
         const int buf = nv & 1;
@@ -483,8 +489,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         const uint32_t p_lo = p_lo0 + (uint32_t)buf * (kPBytes >> 4);
 #pragma unroll 1
         for (int ks = 0; ks < nst_v && ok; ks += 2) {
-          if (!wait_bar(ctx, BAR(bl.full + slot), ring_par, ps + 3)) { ok = false; break; }
-          if (!wait_bar(ctx, BAR(bl.full + slot + 1), ring_par, ps + 3)) { ok = false; break; }
+          if (!wait_bar(ctx, BAR(bl.fullv + slot), (seen >> slot) & 1u, ps + 3)) { ok = false; break; }
+          if (!wait_bar(ctx, BAR(bl.fullv + slot + 1), (seen >> (slot + 1)) & 1u, ps + 3)) { ok = false; break; }
+          seen ^= 3u << slot;
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
           if (lane == 0) {
@@ -501,7 +508,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
           slot += 2;
-          if (slot == S) { slot = 0; ring_par ^= 1u; }
+          if (slot == S) slot = 0;
         }
         if (!ok) break;
         ++nv;
@@ -863,7 +870,7 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   sc.n_slots = fused_slots(grp);
   sc.k_cap = k_cap;
   sc.prof = grp->prof;
-  static_assert(bar_layout(ring_slots<DH, NR>()).total <= 2 * 16 + kNB + 24, "barrier space");
+  static_assert(bar_layout(ring_slots<DH, NR>()).total <= 3 * 16 + kNB + 24, "barrier space");
   static_assert(kNB >= 2 && kNB < ring_slots<DH, NR>(), "B ring must be shorter than the row ring");
   static_assert(NR * WB <= 64 && WB <= kMaxBlocks, "value epilogue registers");
   const size_t smem = fused_smem_bytes<DH, NR>();
