@@ -71,7 +71,7 @@ static bool encode_rows64(void* out, const void* base, uint64_t rows, uint64_t c
 }
 
 bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols) {
-  return encode_rows64(out, base, rows, cols, 256);
+  return encode_rows64(out, base, rows, cols, kLandmarkBoxRows);
 }
 
 }  // namespace xkv
@@ -192,7 +192,7 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
 
     if (c.landmarks) {
       const uint64_t rows = (uint64_t)heads * d.n_c;
-      g->has_lm_tmap = encode_rows64(g->lm_tmap, c.landmarks, rows, (uint64_t)c.d_h, 256) ? 1 : 0;
+      g->has_lm_tmap = encode_landmark_map(g->lm_tmap, c.landmarks, rows, (uint64_t)c.d_h) ? 1 : 0;
       if (!g->has_lm_tmap) { st = XKV_ERR_CUDA; goto fail; }
     }
     // Tensor maps over the repacked B blocks (row pitch r*2 bytes is a multiple of 16 because r % 8 == 0;

@@ -12,6 +12,7 @@ namespace xkv {
 constexpr int kDP = 128;          // rows of a repacked B head block (d_h padded to 128 with zeros)
 constexpr int kMaxRep = 16;       // query heads per KV head
 constexpr int kAttTile = 128;     // selected rows per attention tile
+constexpr int kLandmarkBoxRows = 256;   // landmark rows per TMA box = chunks scored per CTA of the landmark scan
 constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, head) problem
 
 // Device-side description of one window; a copy lives in the handle and is passed by value.
@@ -89,7 +90,7 @@ cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloa
 
 int select_static(const xkv_select_static_config* c, int l0, int l1, const void* q, int32_t k, int32_t* sel_idx,
                   int32_t* sel_cnt, cudaStream_t s);
-// xkv_api.cu: tensor map over [rows][cols] bf16 landmarks, 256-row boxes of 64 columns, 128-byte swizzle
+// xkv_api.cu: tensor map over [rows][cols] bf16 landmarks, kLandmarkBoxRows-row boxes of 64 columns, 128-byte swizzle
 bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols);
 
 // xkv_attend.cu

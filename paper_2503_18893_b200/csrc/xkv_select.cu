@@ -16,7 +16,7 @@ namespace xkv {
 
 namespace {
 
-constexpr int kScoreRows = 256;      // landmark rows (chunks) per CTA
+constexpr int kScoreRows = kLandmarkBoxRows;   // landmark rows (chunks) per CTA
 constexpr int kScoreThreads = 128;   // two rows per thread
 constexpr uint32_t kWaitLimit = 1u << 22;
 
