@@ -27,6 +27,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, sr_fused_kernel (95.77 + 4.32 MB) + merge_segments_kernel
+# (6.17 MB), one window of config 3
+NCU_ATTEND_DRAM_BYTES = 106.2e6
 METRIC = "SR decode steps/sec per layer group at 128K ctx"
 UNIT = "group-steps/s"
 
@@ -319,7 +322,12 @@ def main():
         roof = {"bound": "tensor", "achieved": flops / att_s / 1e12, "peak": pk["bf16_tflops_sustained"],
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update({"traffic": None, "kernel": "xkv_sr_reconstruct_attend (gather + reconstruct + attention)",
+    # DRAM bytes of one reconstruct_attend call (fused kernel + segment merge) from the ncu capture of one window of
+    # this workload (profiles/kernels_one_window_cfg3.md); it only applies to the unmodified headline shape.
+    traffic = None
+    if shape.name == "cfg3_llama_128k" and (s.T, s.r_k, s.r_v, s.k, s.batch) == (131072, 512, 512, 4096, 1):
+        traffic = NCU_ATTEND_DRAM_BYTES
+    roof.update({"traffic": traffic, "kernel": "xkv_sr_reconstruct_attend (gather + reconstruct + attention)",
                  "peak_source": pk["source"], "us_per_launch": att_s * 1e6,
                  "algorithmic_bytes_per_launch": att_bytes, "algorithmic_flops_per_launch": flops})
     step_t = max(bytes_model["bytes_min"] / (pk["hbm_gbs"] * 1e9), tc_t)
