@@ -300,6 +300,52 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
 
 
 # --------------------------------------------------------------------------
+# Uncompressed tail  (Sec. 4 "Implementation details", Sec. 7 "Long Generation Scenario":
+# tokens generated during decoding are not compressed; they are attended to densely)
+# --------------------------------------------------------------------------
+
+
+def sr_attend_with_tail(q_heads, K_hat, V_hat, K_tail, V_tail, scale: float):
+    """Attention of the query heads of one KV head over the union of the reconstructed selected rows
+    (K_hat already rotated) and the uncompressed tail rows (K_tail as the model stores it: post-RoPE).
+
+    The definition written out: one softmax over the concatenated logits.  Returns (o, lse) in fp64.
+    """
+    K = np.concatenate([np.asarray(K_hat, dtype=np.float64), np.asarray(K_tail, dtype=np.float64)], axis=0)
+    V = np.concatenate([np.asarray(V_hat, dtype=np.float64), np.asarray(V_tail, dtype=np.float64)], axis=0)
+    return attend(q_heads, K, V, scale)
+
+
+def sr_decode_step_with_tail(A_k, A_v, B_k, B_v, q, sel_idx, sel_cnt, tail_k, tail_v, tail_len, H_kv,
+                             rope_base, scale=None, problems=None):
+    """`sr_decode_step` with given selections plus an uncompressed tail.
+
+    tail_k, tail_v (G,B,H_kv,tail_cap,d_h); tail_len (B,) rows of the tail that are valid for each sequence.
+    Returns out (G,B,H_q,d_h) fp64, lse (G,B,H_q) fp64.
+    """
+    Bsz, T, _ = A_k.shape
+    G = B_k.shape[1]
+    H_q, d_h = q.shape[2], q.shape[3]
+    n_rep = H_q // H_kv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d_h)
+    out = np.zeros((G, Bsz, H_q, d_h))
+    lse = np.zeros((G, Bsz, H_q))
+    if problems is None:
+        problems = [(l, b, g) for l in range(G) for b in range(Bsz) for g in range(H_kv)]
+    for (l, b, g) in problems:
+        qh = q[l, b, g * n_rep:(g + 1) * n_rep]
+        rows = np.asarray(sel_idx[l, b, g, :int(sel_cnt[l, b, g])], dtype=np.int32)
+        K_hat = sr_reconstruct_keys(A_k[b], B_k[b, l][:, g * d_h:(g + 1) * d_h], rows, rope_base)
+        V_hat = sr_reconstruct(A_v[b], B_v[b, l][:, g * d_h:(g + 1) * d_h], rows)
+        n_t = int(tail_len[b])
+        o, ls = sr_attend_with_tail(qh, K_hat, V_hat, tail_k[l, b, g, :n_t], tail_v[l, b, g, :n_t], scale)
+        out[l, b, g * n_rep:(g + 1) * n_rep] = o
+        lse[l, b, g * n_rep:(g + 1) * n_rep] = ls
+    return out, lse
+
+
+# --------------------------------------------------------------------------
 # Cost and memory accounting  (App. C, "FLOPs & Memory Cost")
 # --------------------------------------------------------------------------
 

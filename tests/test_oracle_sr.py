@@ -295,3 +295,66 @@ def test_step_with_given_index_set_skips_selection():
     ref, _ = O.attend(q[0, 0], A_k[0][rows] @ B_k[0, 0], A_v[0][rows] @ B_v[0, 0], 1 / math.sqrt(d_h))
     np.testing.assert_allclose(out[0, 0], ref, atol=1e-12)
     assert c2[0, 0, 0] == 4
+
+
+# ------------------------------------------------------------------ uncompressed tail (Sec. 4, Sec. 7)
+
+def test_tail_union_equals_dense_and_merge_of_the_two_parts():
+    """Attention over selected rows + tail is one softmax over the union: it must equal the row-by-row dense
+    routine on the concatenation, the library SDPA, and the log-sum-exp merge of the two separate results."""
+    rng = np.random.default_rng(40)
+    q = rng.standard_normal((3, 8))
+    Ks, Vs = 2 * rng.standard_normal((21, 8)), rng.standard_normal((21, 8))
+    Kt, Vt = 2 * rng.standard_normal((6, 8)), rng.standard_normal((6, 8))
+    o, lse = O.sr_attend_with_tail(q, Ks, Vs, Kt, Vt, 0.4)
+    Kc, Vc = np.concatenate([Ks, Kt]), np.concatenate([Vs, Vt])
+    np.testing.assert_allclose(o, O.dense_attend(q, Kc, Vc, 0.4), atol=1e-12)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q)[None], torch.from_numpy(Kc)[None], torch.from_numpy(Vc)[None], scale=0.4)[0].numpy()
+    np.testing.assert_allclose(o, ref, atol=1e-12)
+    om, lm = O.merge_partials([O.attend(q, Ks, Vs, 0.4), O.attend(q, Kt, Vt, 0.4)])
+    np.testing.assert_allclose(o, om, atol=1e-12)
+    np.testing.assert_allclose(lse, lm, atol=1e-12)
+
+
+def test_tail_special_cases():
+    rng = np.random.default_rng(41)
+    q = rng.standard_normal((2, 8))
+    Ks, Vs = rng.standard_normal((5, 8)), rng.standard_normal((5, 8))
+    Kt, Vt = rng.standard_normal((4, 8)), rng.standard_normal((4, 8))
+    # empty tail: the plain SR result
+    o, lse = O.sr_attend_with_tail(q, Ks, Vs, Kt[:0], Vt[:0], 0.3)
+    np.testing.assert_allclose(o, O.attend(q, Ks, Vs, 0.3)[0], atol=1e-15)
+    # empty selection: dense attention over the tail
+    o, lse = O.sr_attend_with_tail(q, Ks[:0], Vs[:0], Kt, Vt, 0.3)
+    np.testing.assert_allclose(o, O.dense_attend(q, Kt, Vt, 0.3), atol=1e-12)
+    # a tail row whose logit dwarfs everything takes all the weight
+    big = np.concatenate([Kt, 200.0 * q[:1]])
+    o, _ = O.sr_attend_with_tail(q[:1], Ks, Vs, big, np.concatenate([Vt, np.full((1, 8), 7.0)]), 1.0)
+    np.testing.assert_allclose(o, np.full((1, 8), 7.0), atol=1e-9)
+
+
+def test_step_with_tail_layouts_and_per_sequence_lengths():
+    """The window-level routine indexes (layer, sequence, head) and honours tail_len per sequence:
+    compare with a direct per-problem evaluation from the definitions."""
+    rng = np.random.default_rng(42)
+    G, Bsz, H_kv, n_rep, d_h, T, r = 2, 2, 2, 2, 8, 40, 6
+    A_k, A_v = _bf(rng.standard_normal((Bsz, T, r))), _bf(rng.standard_normal((Bsz, T, r)))
+    B_k, B_v = _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h))), _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h)))
+    q = _bf(rng.standard_normal((G, Bsz, H_kv * n_rep, d_h)))
+    sel_idx = np.stack([np.sort(rng.choice(T, 12, replace=False)) for _ in range(G * Bsz * H_kv)]).reshape(G, Bsz, H_kv, 12).astype(np.int32)
+    sel_cnt = rng.integers(0, 13, size=(G, Bsz, H_kv)).astype(np.int32)
+    tk, tv = _bf(rng.standard_normal((G, Bsz, H_kv, 5, d_h))), _bf(rng.standard_normal((G, Bsz, H_kv, 5, d_h)))
+    tail_len = np.array([5, 2], dtype=np.int32)
+    out, lse = O.sr_decode_step_with_tail(A_k, A_v, B_k, B_v, q, sel_idx, sel_cnt, tk, tv, tail_len, H_kv, 10000.0)
+    scale = 1 / math.sqrt(d_h)
+    for l in range(G):
+        for b in range(Bsz):
+            for g in range(H_kv):
+                rows = sel_idx[l, b, g, :sel_cnt[l, b, g]]
+                Kh = O.rope_rotate(A_k[b][rows].astype(np.float64) @ B_k[b, l][:, g * d_h:(g + 1) * d_h].astype(np.float64), rows, 10000.0)
+                Vh = A_v[b][rows].astype(np.float64) @ B_v[b, l][:, g * d_h:(g + 1) * d_h].astype(np.float64)
+                n_t = tail_len[b]
+                Kc = np.concatenate([Kh, tk[l, b, g, :n_t]]); Vc = np.concatenate([Vh, tv[l, b, g, :n_t]])
+                ref = O.dense_attend(q[l, b, g * n_rep:(g + 1) * n_rep], Kc, Vc, scale)
+                np.testing.assert_allclose(out[l, b, g * n_rep:(g + 1) * n_rep], ref, atol=1e-10)
