@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--r-v", type=int, default=None)
     ap.add_argument("--rope-base", type=float, default=None)
     ap.add_argument("--groups", type=int, default=None, help="number of windows (default: the config's)")
+    ap.add_argument("--tail", type=int, default=0,
+                    help="rows of uncompressed generated tokens attended to besides the selected rows (default none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-problems", type=int, default=None, help="oracle sample size in (layer,head) problems")
     return ap.parse_args()
@@ -228,7 +230,7 @@ def main():
     shape = make_shape(args)
     # Each rank owns one full replica of the workload (its own sequence): per-GPU work is fixed.
     n_q = 8
-    wl = workload.DeviceWorkload(shape, n_steps=n_q, device="cuda")
+    wl = workload.DeviceWorkload(shape, n_steps=n_q, device="cuda", tail_rows=args.tail)
     n_groups = len(wl.groups)
     s = shape
     q_bytes = n_groups * s.G * s.batch * s.H_q * s.d_h * 2
@@ -264,8 +266,7 @@ def main():
             a = ev(); a.record(stream)
             xkv.xkv_sr_select(grp, 0, s.G, q, s.k, wl.sel_idx[gi], wl.sel_cnt[gi])
             b = ev(); b.record(stream)
-            xkv.xkv_sr_reconstruct_attend(grp, 0, s.G, q, wl.sel_idx[gi], wl.sel_cnt[gi], s.k_cap, wl.out[gi],
-                                          wl.lse[gi])
+            wl.attend(gi, q)
             c = ev(); c.record(stream)
             marks.append((a, b, c))
     e_stop = ev(); e_stop.record(stream)
@@ -352,6 +353,10 @@ def main():
                                                   ((ms_total / args.steps / n_groups) * 1e-3)},
         "device_status": {"status": st, "flags": flags},
     }
+    if args.tail > 0:       # not the headline workload: the step also attends to uncompressed generated tokens
+        line["config"]["tail_rows"] = args.tail
+        line["config"]["workload"] += f", plus {args.tail} uncompressed tail rows per sequence"
+        line["roofline"]["traffic"] = None
     if rank == 0 and not args.no_cpu_baseline:
         n = args.cpu_problems or min(s.G * s.batch * s.H_kv, 32)
         dt, np_, threads = oracle_sample(shape, wl.inputs[0], n)

@@ -131,6 +131,30 @@ XKV_API int xkv_sr_reconstruct_attend(xkv_group* grp, int layer_begin, int layer
                               const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_cap,
                               void* out, float* lse, void* stream);
 
+/*
+ * xkv_sr_reconstruct_attend over the union of the selected reconstructed rows and an uncompressed tail:
+ * the tokens generated during decoding are kept as plain K/V rows (Sec. 4 "Implementation details",
+ * Sec. 7 "Long Generation Scenario") and every decode step attends to all of them.  One softmax over both
+ * sets, evaluated as split partial results merged by their log-sum-exp.
+ * tail_k, tail_v  bf16 [G][batch][H_kv][tail_cap][d_h], device, borrowed for the call; keys as the model
+ *                 stores them (already rotated).
+ * tail_len        int32 [batch], device, or NULL for tail_cap rows in every sequence; 0 <= tail_len <= tail_cap
+ *                 (a larger value is clamped and XKV_FLAG_INDEX_RANGE is raised).
+ * tail_cap        1 <= tail_cap <= XKV_TAIL_MAX_ROWS.
+ * workspace       device scratch of at least xkv_tail_workspace_bytes(grp, tail_cap) bytes, 16-byte aligned,
+ *                 owned by the caller, used only during the call's kernels.
+ * The other arguments and the outputs are those of xkv_sr_reconstruct_attend.  With sel_cnt = 0 and
+ * tail_len = 0 the head's output is 0 and its lse is -inf.
+ * Errors: INVALID_ARG, UNSUPPORTED (shapes the tensor-core path does not cover), CUDA.
+ */
+#define XKV_TAIL_MAX_ROWS 32768
+XKV_API int xkv_tail_workspace_bytes(const xkv_group* grp, int32_t tail_cap, uint64_t* bytes);
+XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int layer_end, const void* q,
+                                           const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_cap,
+                                           const void* tail_k, const void* tail_v, const int32_t* tail_len,
+                                           int32_t tail_cap, void* workspace, uint64_t workspace_bytes,
+                                           void* out, float* lse, void* stream);
+
 /* Free the handle and the device memory it owns (synchronises the device first). NULL is allowed. */
 XKV_API int xkv_group_destroy(xkv_group* grp);
 

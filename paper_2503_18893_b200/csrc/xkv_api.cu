@@ -298,4 +298,35 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   return XKV_OK;
 }
 
+int xkv_tail_workspace_bytes(const xkv_group* g, int32_t tail_cap, uint64_t* bytes) {
+  if (!g || !bytes || tail_cap < 1 || tail_cap > XKV_TAIL_MAX_ROWS) return XKV_ERR_INVALID_ARG;
+  *bytes = (uint64_t)tail_part_floats(g, tail_cap) * sizeof(float);
+  return XKV_OK;
+}
+
+int xkv_sr_reconstruct_attend_tail(xkv_group* g, int layer_begin, int layer_end, const void* q,
+                                   const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_cap,
+                                   const void* tail_k, const void* tail_v, const int32_t* tail_len,
+                                   int32_t tail_cap, void* workspace, uint64_t workspace_bytes, void* out,
+                                   float* lse, void* stream) {
+  if (!g || !q || !sel_idx || !sel_cnt || !out || !tail_k || !tail_v || !workspace) return XKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
+  if (k_cap < 1 || k_cap > g->k_cap_max) return XKV_ERR_INVALID_ARG;
+  if (tail_cap < 1 || tail_cap > XKV_TAIL_MAX_ROWS) return XKV_ERR_INVALID_ARG;
+  if (workspace_bytes < (uint64_t)tail_part_floats(g, tail_cap) * sizeof(float)) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) || ((uintptr_t)sel_cnt & 3u) ||
+      ((uintptr_t)lse & 3u) || ((uintptr_t)tail_k & 15u) || ((uintptr_t)tail_v & 15u) || ((uintptr_t)tail_len & 3u) ||
+      ((uintptr_t)workspace & 15u))
+    return XKV_ERR_INVALID_ARG;
+  if (g->attend_impl || !fused_supported(g)) return XKV_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = launch_tail_partials(g, layer_begin, layer_end, (const __nv_bfloat16*)q, (const __nv_bfloat16*)tail_k,
+                                       (const __nv_bfloat16*)tail_v, tail_len, tail_cap, (float*)workspace, s);
+  if (e == cudaSuccess)
+    e = launch_fused(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt, k_cap, (__nv_bfloat16*)out,
+                     lse, s, TailParts{(const float*)workspace, tail_splits(tail_cap)});
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
 }  // extern "C"

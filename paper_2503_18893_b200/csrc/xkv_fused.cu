@@ -761,9 +761,10 @@ constexpr int kMergeThreads = 1024;
 constexpr int kMergeMaxSeg = 160;                     // a problem never has more segments than there are CTAs + 1
 template <int DH>
 __global__ void __launch_bounds__(kMergeThreads)
-merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
   extern __shared__ float m_s[];                      // [r_v] weights-times-basis, then [rows per pass][DH] partial sums
   __shared__ float wgt_s[kMergeMaxSeg];
+  __shared__ float twgt_s[kTailMaxSplit];             // weights of the partial results over the uncompressed tail
   __shared__ float ML_s[2];
   constexpr int TPR = DH / 8, RPP = kMergeThreads / TPR;
   const int n_rep = dev.n_rep, r = dev.r_v;
@@ -791,9 +792,13 @@ merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, f
   }
   grid_dependency_wait();                             // the partials come from the kernel launched before this one
   const float* part = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h * (r + 2);
+  const int nts = tail.part ? min(tail.n_split, kTailMaxSplit) : 0;
+  const size_t tstride = (size_t)n_rep * (DH + 2);
+  const float* tpart = tail.part ? tail.part + ((size_t)py * tail.n_split) * tstride + (size_t)h * (DH + 2) : nullptr;
   if (tid < 32) {                                     // one warp: maxima, weights of the segments, denominator
     float mx = -INFINITY;
     for (int s = tid; s < nseg; s += 32) mx = fmaxf(mx, part[s * stride + r]);
+    for (int s = tid; s < nts; s += 32) mx = fmaxf(mx, tpart[s * tstride + DH]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     float Ls = 0.0f;
@@ -802,6 +807,12 @@ merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, f
       const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
       wgt_s[s] = w;
       Ls += w * part[s * stride + r + 1];
+    }
+    for (int s = tid; s < nts; s += 32) {
+      const float ms = tpart[s * tstride + DH];
+      const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
+      twgt_s[s] = w;
+      Ls += w * tpart[s * tstride + DH + 1];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
@@ -850,6 +861,8 @@ merge_segments_kernel(GroupDev dev, Sched sc, __nv_bfloat16* __restrict__ out, f
     float o = 0.0f;
 #pragma unroll
     for (int f = 0; f < FOLD; ++f) o += red[f * DH + tid];
+#pragma unroll 8
+    for (int s = 0; s < nts; ++s) o = fmaf(twgt_s[s], tpart[s * tstride + tid], o);   // the tail is already in output space
     const float M = ML_s[0], L = ML_s[1];
     const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
     out[qh * DH + tid] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
@@ -864,7 +877,7 @@ constexpr size_t fused_smem_bytes() {
 
 template <int DH, int NR, int WB>
 cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
-                           const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
+                           const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s, TailParts tail) {
   const GroupDev& dev = grp->dev;
   const int problems = (l1 - l0) * dev.batch * dev.H_kv;
   Sched sc;
@@ -889,7 +902,7 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
   e = cudaFuncSetAttribute(merge_segments_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, out, lse);
+  e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, tail, out, lse);
   if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
@@ -914,12 +927,12 @@ bool fused_supported(const xkv_group* grp) {
 }
 
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
-                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s) {
+                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s, TailParts tail) {
   const int n_rep = grp->dev.n_rep;
 #define XKV_DISPATCH(DH)                                                                                 \
-  if (n_rep <= 4) return launch_fused_t<DH, 4, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
-  if (n_rep <= 8) return launch_fused_t<DH, 8, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);  \
-  return launch_fused_t<DH, 16, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s);
+  if (n_rep <= 4) return launch_fused_t<DH, 4, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
+  if (n_rep <= 8) return launch_fused_t<DH, 8, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
+  return launch_fused_t<DH, 16, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);
   if (grp->dev.d_h == 128) { XKV_DISPATCH(128) }
   XKV_DISPATCH(64)
 #undef XKV_DISPATCH

@@ -13,6 +13,8 @@ constexpr int kDP = 128;          // rows of a repacked B head block (d_h padded
 constexpr int kMaxRep = 16;       // query heads per KV head
 constexpr int kAttTile = 128;     // selected rows per attention tile
 constexpr int kLandmarkBoxRows = 256;   // landmark rows per TMA box = chunks scored per CTA of the landmark scan
+constexpr int kTailSplitRows = 128;     // tail rows per partial result
+constexpr int kTailMaxSplit = XKV_TAIL_MAX_ROWS / kTailSplitRows;
 constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, head) problem
 
 // Device-side description of one window; a copy lives in the handle and is passed by value.
@@ -99,11 +101,23 @@ cudaError_t launch_reconstruct_attend(const xkv_group* grp, int l0, int l1, cons
                                       const int32_t* sel_idx, const int32_t* sel_cnt, int k_cap,
                                       __nv_bfloat16* out, float* lse, cudaStream_t s);
 
+// xkv_tail.cu: partial attention results over an uncompressed tail, [problem of the call][split][head][d_h + 2]
+struct TailParts {
+  const float* part;   // nullptr: no tail
+  int n_split;
+};
+int tail_splits(int tail_cap);
+size_t tail_part_floats(const xkv_group* grp, int tail_cap);
+cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const __nv_bfloat16* tail_k,
+                                 const __nv_bfloat16* tail_v, const int32_t* tail_len, int tail_cap, float* part,
+                                 cudaStream_t s);
+
 // xkv_fused.cu
 int fused_slots(const xkv_group* grp);
 size_t fused_part_floats(const xkv_group* grp);
 bool fused_supported(const xkv_group* grp);
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
-                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s);
+                         const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s,
+                         TailParts tail = TailParts{nullptr, 0});
 
 }  // namespace xkv

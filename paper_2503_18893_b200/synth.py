@@ -162,7 +162,7 @@ def config(i: int, **over) -> SRShape:
 # Recipes
 # --------------------------------------------------------------------------
 
-_T_K, _T_V, _T_Q, _T_IDX = 1, 2, 3, 4
+_T_K, _T_V, _T_Q, _T_IDX, _T_TAIL_K, _T_TAIL_V = 1, 2, 3, 4, 5, 6
 
 
 def make_kv(shape: SRShape, group: int = 0, seq: int = 0, device="cpu"):
@@ -235,6 +235,17 @@ def make_queries(shape: SRShape, n_steps: int = 1, group: int = 0, device="cpu")
     q = normal(stream_key(shape.seed, _T_Q, group), (n_steps, shape.G, shape.batch, shape.H_q, shape.d_h),
                device)
     return q.to(torch.bfloat16)
+
+
+def make_tail(shape: SRShape, tail_cap: int, key_rms: float = 1.0, value_rms: float = 1.0, group: int = 0,
+              device="cpu"):
+    """Uncompressed K/V rows of the tokens generated so far (keys as the model stores them, already rotated):
+    N(0, rms^2), bf16, shape (G, batch, H_kv, tail_cap, d_h) each.  The caller picks the scales so that the
+    tail's logits are comparable with those of the reconstructed rows."""
+    shp = (shape.G, shape.batch, shape.H_kv, tail_cap, shape.d_h)
+    k = normal(stream_key(shape.seed, _T_TAIL_K, group), shp, device) * key_rms
+    v = normal(stream_key(shape.seed, _T_TAIL_V, group), shp, device) * value_rms
+    return k.to(torch.bfloat16), v.to(torch.bfloat16)
 
 
 def fixed_index_set(shape: SRShape, n_rows: int = 256, seed: int = 4242) -> torch.Tensor:

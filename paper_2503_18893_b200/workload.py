@@ -115,7 +115,7 @@ def algorithmic_flops(shape: synth.SRShape) -> float:
 class DeviceWorkload:
     """All windows of a configuration resident on one GPU, with their handles and output buffers."""
 
-    def __init__(self, shape: synth.SRShape, n_steps: int = 4, device="cuda", groups=None):
+    def __init__(self, shape: synth.SRShape, n_steps: int = 4, device="cuda", groups=None, tail_rows: int = 0):
         from . import xkv  # loads the CUDA library; raises if it is not built
         self.xkv = xkv
         self.shape = shape
@@ -136,6 +136,26 @@ class DeviceWorkload:
         self.out = torch.empty((n, s.G, s.batch, s.H_q, s.d_h), dtype=torch.bfloat16, device=device)
         self.lse = torch.empty((n, s.G, s.batch, s.H_q), dtype=torch.float32, device=device)
         self.n_steps = n_steps
+        # optional uncompressed tail of generated tokens (Sec. 4): every sequence has `tail_rows` of them
+        self.tail_rows = tail_rows
+        self.tail = []
+        self.tail_ws = None
+        if tail_rows > 0:
+            for gi in ids:
+                self.tail.append(synth.make_tail(s, tail_rows, group=gi, device=device))
+            self.tail_ws = torch.empty(xkv.xkv_tail_workspace_bytes(self.groups[0], tail_rows), dtype=torch.uint8,
+                                       device=device)
+
+    def attend(self, gi: int, q) -> None:
+        """Reconstruct+attend of window gi over the rows selected last, plus the tail if there is one."""
+        s, x, grp = self.shape, self.xkv, self.groups[gi]
+        if self.tail_rows > 0:
+            tk, tv = self.tail[gi]
+            x.xkv_sr_reconstruct_attend_tail(grp, 0, s.G, q, self.sel_idx[gi], self.sel_cnt[gi], s.k_cap, tk, tv, None,
+                                             self.tail_rows, self.tail_ws, self.out[gi], self.lse[gi])
+        else:
+            x.xkv_sr_reconstruct_attend(grp, 0, s.G, q, self.sel_idx[gi], self.sel_cnt[gi], s.k_cap,
+                                        self.out[gi], self.lse[gi])
 
     def step(self, i: int, q_override=None) -> None:
         """One decode step: every window, select then reconstruct+attend, on the current stream."""
@@ -143,8 +163,7 @@ class DeviceWorkload:
         for gi, grp in enumerate(self.groups):
             q = self.inputs[gi].q[i % self.n_steps] if q_override is None else q_override[gi]
             x.xkv_sr_select(grp, 0, s.G, q, s.k, self.sel_idx[gi], self.sel_cnt[gi])
-            x.xkv_sr_reconstruct_attend(grp, 0, s.G, q, self.sel_idx[gi], self.sel_cnt[gi], s.k_cap,
-                                        self.out[gi], self.lse[gi])
+            self.attend(gi, q)
 
     def close(self):
         for g in self.groups:

@@ -70,6 +70,11 @@ _lib.xkv_sr_reconstruct_attend.restype = ctypes.c_int
 _lib.xkv_sr_select_static.argtypes = [ctypes.POINTER(xkv_select_static_config), ctypes.c_int, ctypes.c_int, _P,
                                       ctypes.c_int32, _P, _P, _P]
 _lib.xkv_sr_select_static.restype = ctypes.c_int
+_lib.xkv_tail_workspace_bytes.argtypes = [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_tail_workspace_bytes.restype = ctypes.c_int
+_lib.xkv_sr_reconstruct_attend_tail.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, ctypes.c_int32, _P, _P, _P,
+                                                ctypes.c_int32, _P, ctypes.c_uint64, _P, _P, _P]
+_lib.xkv_sr_reconstruct_attend_tail.restype = ctypes.c_int
 _lib.xkv_group_destroy.argtypes = [_P]
 _lib.xkv_group_destroy.restype = ctypes.c_int
 _lib.xkv_group_status.argtypes = [_P, ctypes.POINTER(ctypes.c_uint32), _P]
@@ -195,6 +200,26 @@ def xkv_sr_reconstruct_attend(grp: Group, layer_begin: int, layer_end: int, q, s
                                         k_cap, _ptr(out), _ptr(lse), _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_sr_reconstruct_attend")
+
+
+def xkv_tail_workspace_bytes(grp: Group, tail_cap: int) -> int:
+    b = ctypes.c_uint64()
+    st = _lib.xkv_tail_workspace_bytes(grp.handle, tail_cap, ctypes.byref(b))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_tail_workspace_bytes")
+    return b.value
+
+
+def xkv_sr_reconstruct_attend_tail(grp: Group, layer_begin: int, layer_end: int, q, sel_idx, sel_cnt, k_cap: int,
+                                   tail_k, tail_v, tail_len, tail_cap: int, workspace, out, lse=None,
+                                   stream=None) -> None:
+    """`workspace`: a device tensor of at least xkv_tail_workspace_bytes(grp, tail_cap) bytes."""
+    st = _lib.xkv_sr_reconstruct_attend_tail(grp.handle, layer_begin, layer_end, _ptr(q), _ptr(sel_idx), _ptr(sel_cnt),
+                                             k_cap, _ptr(tail_k), _ptr(tail_v), _ptr(tail_len), tail_cap,
+                                             _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                             _ptr(out), _ptr(lse), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_sr_reconstruct_attend_tail")
 
 
 def xkv_group_status(grp: Group, stream=None):

@@ -38,6 +38,12 @@ def oracle_step(shape, inp, step=0, sel_idx=None, sel_cnt=None, problems=None, k
                             rope_base=shape.rope_base, sel_idx=sel_idx, sel_cnt=sel_cnt, problems=problems)
 
 
+def oracle_step_with_tail(shape, inp, sel_idx, sel_cnt, tail_k, tail_v, tail_len, step=0, problems=None):
+    return O.sr_decode_step_with_tail(f32(inp.A_k), f32(inp.A_v), f32(inp.B_k), f32(inp.B_v), f32(inp.q[step]),
+                                      sel_idx, sel_cnt, f32(tail_k), f32(tail_v), np.asarray(tail_len),
+                                      H_kv=shape.H_kv, rope_base=shape.rope_base, problems=problems)
+
+
 def rel_err(gpu: np.ndarray, ref: np.ndarray) -> float:
     """max_i |gpu_i - ref_i| / max_i |ref_i| over the last axis, worst vector."""
     num = np.abs(gpu.astype(np.float64) - ref).max(axis=-1)
@@ -79,6 +85,22 @@ class GpuCase:
         self.xkv.xkv_sr_reconstruct_attend(self.grp, l0, l1, self.inp.q[step], idx, cnt, idx.shape[-1], out, lse)
         torch.cuda.synchronize()
         return f32(out), (lse.cpu().numpy() if want_lse else None)
+
+    def attend_tail(self, sel_idx, sel_cnt, tail_k, tail_v, tail_len, step=0, layers=None):
+        s = self.shape
+        idx = torch.as_tensor(sel_idx, dtype=torch.int32).cuda().contiguous()
+        cnt = torch.as_tensor(sel_cnt, dtype=torch.int32).cuda().contiguous()
+        tk, tv = tail_k.cuda().contiguous(), tail_v.cuda().contiguous()
+        tl = None if tail_len is None else torch.as_tensor(tail_len, dtype=torch.int32).cuda().contiguous()
+        cap = tk.shape[3]
+        ws = torch.empty(self.xkv.xkv_tail_workspace_bytes(self.grp, cap), dtype=torch.uint8, device="cuda")
+        out = torch.zeros((s.G, s.batch, s.H_q, s.d_h), dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros((s.G, s.batch, s.H_q), dtype=torch.float32, device="cuda")
+        l0, l1 = layers or (0, s.G)
+        self.xkv.xkv_sr_reconstruct_attend_tail(self.grp, l0, l1, self.inp.q[step], idx, cnt, idx.shape[-1], tk, tv, tl,
+                                                cap, ws, out, lse)
+        torch.cuda.synchronize()
+        return f32(out), lse.cpu().numpy()
 
     def status(self):
         return self.xkv.xkv_group_status(self.grp)

@@ -1,0 +1,103 @@
+"""Parity of the uncompressed-tail variant of reconstruct+attend (Sec. 4, Sec. 7: generated tokens stay
+uncompressed) against the oracle: one softmax over the selected reconstructed rows and the tail rows."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import xkv_oracle as O
+from paper_2503_18893_b200 import synth
+from tests import _cases as C
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2       # max relative error per output vector
+
+
+def _key_rms(s, inp):
+    """RMS of a few reconstructed key rows: tail keys of that size give logits comparable with the SR part."""
+    rows = np.arange(0, min(s.T, 64))
+    K = O.sr_reconstruct(C.f32(inp.A_k)[0], C.f32(inp.B_k)[0, 0][:, :s.d_h], rows)
+    return float(np.sqrt((K ** 2).mean()))
+
+
+def _fixed_selection(s, n_rows):
+    idx = synth.fixed_index_set(s, n_rows).numpy()
+    cnt = np.full((s.G, s.batch, s.H_kv), n_rows, dtype=np.int32)
+    return idx, cnt
+
+
+CASES = [
+    ("two_splits_ragged", dict(T=2048, k=256), 700, [700]),
+    ("one_row", dict(T=1024, k=128), 1, [1]),
+    ("per_sequence_lengths", dict(T=1024, k=128, batch=3), 600, [600, 0, 129]),
+    ("d64_heads_16", dict(T=1024, k=128, H_kv=1, H_q=16, d_h=64, r_k=64, r_v=72), 300, [257]),
+    ("qwen_like_rep7", dict(T=1024, k=128, H_kv=2, H_q=14, r_k=96, r_v=160), 1500, [1400]),
+]
+
+
+@pytest.mark.parametrize("name,over,cap,lens", CASES, ids=[c[0] for c in CASES])
+def test_tail_parity(name, over, cap, lens):
+    s = synth.config(1, **over)
+    inp = C.case_from_factors(s)
+    rms = _key_rms(s, inp)
+    tk, tv = synth.make_tail(s, cap, key_rms=rms, value_rms=1.0)
+    idx, cnt = _fixed_selection(s, 96)
+    cnt[0, 0, 0] = 0                                   # one problem attends to the tail only
+    g = C.GpuCase(s, inp)
+    gout, glse = g.attend_tail(idx, cnt, tk, tv, lens)
+    oout, olse = C.oracle_step_with_tail(s, inp, idx, cnt, tk, tv, lens)
+    assert g.status() == (0, 0)
+    # empty problems (no selected rows and no tail rows) give 0 and -inf on both sides
+    empty = np.isneginf(olse)
+    assert np.array_equal(np.isneginf(glse), empty)
+    assert np.all(gout[empty] == 0)
+    assert C.rel_err(gout[~empty], oout[~empty]) <= TOL, name
+    np.testing.assert_allclose(glse[~empty], olse[~empty], atol=2e-2)
+    # the case must exercise both parts: compare with the SR-only result where both are present
+    _, _, sr_out, sr_lse = C.oracle_step(s, inp, 0, sel_idx=idx, sel_cnt=cnt)
+    both = (~empty) & ~np.isneginf(sr_lse) & (np.repeat(np.asarray(lens)[None, :, None], s.G, 0) > 0)
+    if both.any() and min(l for l in lens if l > 0) >= 96:
+        share = np.exp(sr_lse[both] - olse[both])      # weight of the SR part in the union
+        assert 0.02 < np.median(share) < 0.98, (name, float(np.median(share)))
+    g.close()
+
+
+def test_empty_tail_equals_plain_call_bit_for_bit():
+    s = synth.config(1, T=1024, k=128)
+    inp = C.case_from_factors(s)
+    tk, tv = synth.make_tail(s, 64)
+    idx, cnt = _fixed_selection(s, 80)
+    g = C.GpuCase(s, inp)
+    out0, lse0 = g.attend(idx, cnt)
+    out1, lse1 = g.attend_tail(idx, cnt, tk, tv, [0])
+    assert np.array_equal(out0, out1) and np.array_equal(lse0, lse1)
+    g.close()
+
+
+def test_tail_argument_checks_and_length_clamp():
+    s = synth.config(1, T=1024, k=128)
+    inp = C.case_from_factors(s)
+    g = C.GpuCase(s, inp)
+    x = g.xkv
+    with pytest.raises(x.XKVError) as e:
+        x.xkv_tail_workspace_bytes(g.grp, 0)
+    assert e.value.status == x.XKV_ERR_INVALID_ARG
+    with pytest.raises(x.XKVError) as e:
+        x.xkv_tail_workspace_bytes(g.grp, 32768 + 1)
+    assert e.value.status == x.XKV_ERR_INVALID_ARG
+    need = x.xkv_tail_workspace_bytes(g.grp, 100)
+    assert need == s.G * s.batch * s.H_kv * 1 * s.n_rep * (s.d_h + 2) * 4
+    tk, tv = synth.make_tail(s, 100)
+    idx, cnt = _fixed_selection(s, 40)
+    i, c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda()
+    out = torch.zeros((s.G, s.batch, s.H_q, s.d_h), dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(x.XKVError) as e:
+        x.xkv_sr_reconstruct_attend_tail(g.grp, 0, s.G, g.inp.q[0], i, c, 40, tk.cuda(), tv.cuda(), None, 100, small, out)
+    assert e.value.status == x.XKV_ERR_INVALID_ARG
+    # a length beyond the capacity is clamped and reported
+    gout, glse = g.attend_tail(idx, cnt, tk, tv, [101])
+    st, flags = g.status()
+    assert st == x.XKV_ERR_INDEX_RANGE and flags & x.XKV_FLAG_INDEX_RANGE
+    oout, olse = C.oracle_step_with_tail(s, inp, idx, cnt, tk, tv, [100])
+    assert C.rel_err(gout, oout) <= TOL
+    g.close()
