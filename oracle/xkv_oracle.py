@@ -168,12 +168,50 @@ def expand_chunks(chunks: np.ndarray, c: int, T: int) -> np.ndarray:
     return np.asarray(rows, dtype=np.int32)
 
 
-def sr_select(q_heads: np.ndarray, L_g: np.ndarray, k: int, c: int, T: int) -> np.ndarray:
-    """Selected token rows for one (layer, sequence, KV head): Algorithm 2 without outliers."""
+def union_outliers(chunks: np.ndarray, outliers, n_c: int) -> np.ndarray:
+    """Algorithm 2 line 5: the selected chunks united with the head's static outlier chunks, ascending.
+
+    Ids outside [0, n_c) are ignored and a repeated id counts once (it is a set union)."""
+    if outliers is None:
+        return np.asarray(chunks, dtype=np.int64)
+    keep = set(int(j) for j in chunks)
+    for j in np.asarray(outliers).reshape(-1):
+        if 0 <= int(j) < n_c:
+            keep.add(int(j))
+    return np.asarray(sorted(keep), dtype=np.int64)
+
+
+def sr_select(q_heads: np.ndarray, L_g: np.ndarray, k: int, c: int, T: int, outliers=None) -> np.ndarray:
+    """Selected token rows for one (layer, sequence, KV head): Algorithm 2 (line 5 only if `outliers` is given)."""
     n_c = L_g.shape[0]
     k_ch = min(-(-k // c), n_c)
     S = pool_scores(landmark_scores(q_heads, L_g))
-    return expand_chunks(topk_chunks(S, k_ch), c, T)
+    return expand_chunks(union_outliers(topk_chunks(S, k_ch), outliers, n_c), c, T)
+
+
+def min_chunk_cosine(K_rope: np.ndarray, c: int) -> np.ndarray:
+    """Algorithm 1 line 4-5 (first half): r_j = min over the tokens x of chunk j of cos(K(x), landmark_j), with the
+    landmark the exact (unrounded) chunk mean.  K_rope (T, d_h) post-RoPE keys of one head; returns (n_c,) fp64.
+    A zero vector has cosine 0 with everything."""
+    K = np.asarray(K_rope, dtype=np.float64)
+    T = K.shape[0]
+    n_c = -(-T // c)
+    out = np.empty(n_c)
+    for j in range(n_c):
+        rows = K[j * c:min(T, j * c + c)]
+        lm = rows.mean(axis=0)
+        den = np.linalg.norm(rows, axis=1) * np.linalg.norm(lm)
+        cos = np.where(den > 0, (rows @ lm) / np.where(den > 0, den, 1.0), 0.0)
+        out[j] = cos.min()
+    return out
+
+
+def static_outliers(K_rope: np.ndarray, c: int, o: int) -> np.ndarray:
+    """Algorithm 1 line 5: the o chunks with the smallest minimum within-chunk cosine (ties to the lowest
+    chunk id), i.e. ArgTopK(-m, o); returned ascending."""
+    m = min_chunk_cosine(K_rope, c)
+    order = np.argsort(m, kind="stable")
+    return np.sort(order[:min(o, m.shape[0])]).astype(np.int64)
 
 
 # --------------------------------------------------------------------------
@@ -248,10 +286,10 @@ def merge_partials(parts):
 
 
 def sr_decode_problem(q_heads, L_g, A_k, A_v, B_k_head, B_v_head, k, c, T, rope_base, scale,
-                      rows=None):
+                      rows=None, outliers=None):
     """One (layer, sequence, KV head) problem.  rows=None: use Algorithm 2."""
     if rows is None:
-        rows = sr_select(q_heads, L_g, k, c, T)
+        rows = sr_select(q_heads, L_g, k, c, T, outliers)
     K_hat = sr_reconstruct_keys(A_k, B_k_head, rows, rope_base)
     V_hat = sr_reconstruct(A_v, B_v_head, rows)
     o, lse = attend(q_heads, K_hat, V_hat, scale)
@@ -259,7 +297,7 @@ def sr_decode_problem(q_heads, L_g, A_k, A_v, B_k_head, B_v_head, k, c, T, rope_
 
 
 def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scale=None,
-                   sel_idx=None, sel_cnt=None, problems=None):
+                   sel_idx=None, sel_cnt=None, problems=None, outliers=None):
     """Whole-window decode step in the library's tensor layouts.
 
     A_k (B,T,r_k)  A_v (B,T,r_v)  B_k (B,G,r_k,d)  B_v (B,G,r_v,d)
@@ -269,6 +307,8 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
     If sel_idx/sel_cnt are given the selection is taken from them (any order,
     duplicates allowed) and Algorithm 2 is skipped.  `problems` restricts the
     work to a list of (l, b, g) triples (the rest of the outputs stay zero).
+    `outliers` (B,G,H_kv,o) int: static outlier chunk ids united with every selection (Algorithm 2 line 5);
+    the row stride of sel_idx is then (ceil(k/c) + o) * c.
     """
     Bsz, T, _ = A_k.shape
     G = B_k.shape[1]
@@ -276,7 +316,8 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
     n_rep = H_q // H_kv
     if scale is None:
         scale = 1.0 / math.sqrt(d_h)
-    k_cap = (-(-k // c)) * c if sel_idx is None else sel_idx.shape[-1]
+    n_out = 0 if outliers is None else outliers.shape[-1]
+    k_cap = (-(-k // c) + n_out) * c if sel_idx is None else sel_idx.shape[-1]
     o_idx = np.full((G, Bsz, H_kv, k_cap), -1, dtype=np.int32)
     o_cnt = np.zeros((G, Bsz, H_kv), dtype=np.int32)
     out = np.zeros((G, Bsz, H_q, d_h))
@@ -291,7 +332,7 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
         rows, o, ls = sr_decode_problem(
             qh, None if landmarks is None else landmarks[b, l, g], A_k[b], A_v[b],
             B_k[b, l][:, g * d_h:(g + 1) * d_h], B_v[b, l][:, g * d_h:(g + 1) * d_h],
-            k, c, T, rope_base, scale, rows)
+            k, c, T, rope_base, scale, rows, None if outliers is None else outliers[b, l, g])
         o_idx[l, b, g, :len(rows)] = rows
         o_cnt[l, b, g] = len(rows)
         out[l, b, g * n_rep:(g + 1) * n_rep] = o

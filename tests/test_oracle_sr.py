@@ -358,3 +358,71 @@ def test_step_with_tail_layouts_and_per_sequence_lengths():
                 Kc = np.concatenate([Kh, tk[l, b, g, :n_t]]); Vc = np.concatenate([Vh, tv[l, b, g, :n_t]])
                 ref = O.dense_attend(q[l, b, g * n_rep:(g + 1) * n_rep], Kc, Vc, scale)
                 np.testing.assert_allclose(out[l, b, g * n_rep:(g + 1) * n_rep], ref, atol=1e-10)
+
+
+# ------------------------------------------------------------------ static outliers (Alg. 1 lines 4-5, Alg. 2 line 5)
+
+def test_union_with_outliers_is_a_set_union_and_keeps_the_topk():
+    rng = np.random.default_rng(50)
+    T, c, d_h = 333, 8, 16
+    n_c = -(-T // c)
+    L = _bf(rng.standard_normal((n_c, d_h)))
+    q = _bf(rng.standard_normal((2, d_h)))
+    plain = O.sr_select(q, L, 40, c, T)
+    out = np.array([3, 3, n_c - 1, -5, 10 ** 6, int(plain[0]) // c, 17])       # repeats, out of range, one already in
+    rows = O.sr_select(q, L, 40, c, T, outliers=out)
+    want = set(plain.tolist())
+    for j in (3, n_c - 1, 17, int(plain[0]) // c):
+        want |= set(range(j * c, min(T, j * c + c)))
+    assert rows.tolist() == sorted(want)                                      # brute force on sets
+    assert set(plain.tolist()) <= set(rows.tolist())
+    # outliers that the top-k already holds change nothing; an empty list changes nothing
+    inside = np.unique(plain // c)[:3]
+    np.testing.assert_array_equal(O.sr_select(q, L, 40, c, T, outliers=inside), plain)
+    np.testing.assert_array_equal(O.sr_select(q, L, 40, c, T, outliers=np.array([], dtype=np.int64)), plain)
+
+
+def test_min_chunk_cosine_and_static_outliers():
+    c = 4
+    e0, e1 = np.eye(6)[0], np.eye(6)[1]
+    K = np.stack([e0, e0, e0, e0,                    # identical rows: cosine 1
+                  e0, e0, e0, -e0 + 4 * e1,          # one row far from the mean
+                  e0, e1, e0, e1,                    # two directions: each row at 45 degrees from the mean
+                  2 * e0, 5 * e0])                   # ragged chunk, parallel rows of different length: cosine 1
+    m = O.min_chunk_cosine(K, c)
+    np.testing.assert_allclose(m[0], 1.0, atol=1e-12)
+    np.testing.assert_allclose(m[2], math.cos(math.pi / 4), atol=1e-12)
+    np.testing.assert_allclose(m[3], 1.0, atol=1e-12)
+    mean1 = K[4:8].mean(axis=0)
+    np.testing.assert_allclose(m[1], min(K[j] @ mean1 / np.linalg.norm(K[j]) / np.linalg.norm(mean1) for j in range(4, 8)), atol=1e-12)
+    assert m[1] < m[2]
+    np.testing.assert_array_equal(O.static_outliers(K, c, 2), [1, 2])          # the two least homogeneous chunks
+    np.testing.assert_array_equal(O.static_outliers(K, c, 1), [1])
+    np.testing.assert_array_equal(O.static_outliers(K, c, 9), [0, 1, 2, 3])    # o larger than n_c
+    # scaling a row does not change its cosine; a zero row has cosine 0
+    K2 = K.copy(); K2[0] *= 7.0
+    np.testing.assert_allclose(O.min_chunk_cosine(K2, c)[0], 1.0, atol=1e-12)
+    K3 = K.copy(); K3[1] = 0.0
+    np.testing.assert_allclose(O.min_chunk_cosine(K3, c)[0], 0.0, atol=1e-12)
+
+
+def test_step_with_outliers_layout_and_count():
+    rng = np.random.default_rng(51)
+    G, Bsz, H_kv, n_rep, d_h, T, r, c = 2, 2, 2, 2, 8, 70, 6, 8
+    n_c = -(-T // c)
+    A_k, A_v = _bf(rng.standard_normal((Bsz, T, r))), _bf(rng.standard_normal((Bsz, T, r)))
+    B_k, B_v = _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h))), _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h)))
+    lm = _bf(rng.standard_normal((Bsz, G, H_kv, n_c, d_h)))
+    q = _bf(rng.standard_normal((G, Bsz, H_kv * n_rep, d_h)))
+    outl = rng.integers(0, n_c, size=(Bsz, G, H_kv, 3))
+    idx, cnt, out, lse = O.sr_decode_step(A_k, A_v, B_k, B_v, lm, q, 16, c, H_kv, 10000.0, outliers=outl)
+    assert idx.shape[-1] == (2 + 3) * c
+    for l in range(G):
+        for b in range(Bsz):
+            for g in range(H_kv):
+                rows = O.sr_select(q[l, b, g * n_rep:(g + 1) * n_rep], lm[b, l, g], 16, c, T, outl[b, l, g])
+                assert cnt[l, b, g] == len(rows)
+                np.testing.assert_array_equal(idx[l, b, g, :len(rows)], rows)
+                assert np.all(idx[l, b, g, len(rows):] == -1)
+                for j in outl[b, l, g]:
+                    assert j * c in rows
