@@ -103,7 +103,8 @@ XKV_API int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_grou
  *   -0 equals +0), sort them ascending, expand chunk j to rows c*j .. min(c*j+c, T)-1.
  * q        bf16 [G][batch][H_q][d_h], post-RoPE decode queries (rows of layers outside the range are
  *          not read).
- * k        token budget, 1 <= k <= k_max.  k_cap = ceil(k/c)*c is the row stride of sel_idx.
+ * k        token budget, 1 <= k <= k_max.  k_cap = ceil(k/c)*c is the row stride of sel_idx
+ *          ((ceil(k/c) + n_outliers)*c after xkv_group_set_outliers, see there).
  * sel_idx  out, int32 [G][batch][H_kv][k_cap]; entries at and beyond sel_cnt are set to -1.
  * sel_cnt  out, int32 [G][batch][H_kv]; number of rows (k_ch*c, less if the ragged last chunk is in).
  * Scores must be finite; the result for NaN inputs is unspecified (but in range).
@@ -111,6 +112,21 @@ XKV_API int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_grou
  */
 XKV_API int xkv_sr_select(xkv_group* grp, int layer_begin, int layer_end, const void* q, int32_t k,
                   int32_t* sel_idx, int32_t* sel_cnt, void* stream);
+
+/*
+ * Static outlier chunks (Algorithm 1 line 5 finds them at prefill; Algorithm 2 line 5 uses them): from now on
+ * xkv_sr_select unites the top-k chunks of every (layer, sequence, KV head) with that head's outlier chunks.
+ * outliers    int32 [batch][G][H_kv][n_outliers] chunk ids, device memory, BORROWED until the handle is destroyed
+ *             or the list is replaced.  Ids outside [0, n_c) are ignored; a repeated id counts once.
+ * n_outliers  0 <= n_outliers <= XKV_MAX_OUTLIERS; 0 (with any pointer) switches the union off.
+ * With outliers the row stride of sel_idx is k_cap = (ceil(k/c) + n_outliers) * c, sel_cnt varies between
+ * ceil(k/c)*c and k_cap (less by the ragged last chunk), rows stay ascending without repeats, and
+ * xkv_sr_reconstruct_attend accepts k_cap up to (ceil(k_max/c) + n_outliers) * c.
+ * The call waits for `stream` and may replace the handle's scratch: no work of this handle may be in flight on
+ * another stream.  Errors: INVALID_ARG (also: handle without landmarks), OOM, CUDA.
+ */
+#define XKV_MAX_OUTLIERS 4096
+XKV_API int xkv_group_set_outliers(xkv_group* grp, const int32_t* outliers, int32_t n_outliers, void* stream);
 
 /*
  * Eq. 3 plus attention for layers layer_begin <= l < layer_end, every sequence, every KV head g:

@@ -298,6 +298,38 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   return XKV_OK;
 }
 
+int xkv_group_set_outliers(xkv_group* g, const int32_t* outliers, int32_t n_outliers, void* stream) {
+  if (!g || n_outliers < 0 || n_outliers > XKV_MAX_OUTLIERS) return XKV_ERR_INVALID_ARG;
+  if (n_outliers > 0 && (!outliers || ((uintptr_t)outliers & 3u))) return XKV_ERR_INVALID_ARG;
+  if (!g->cfg.landmarks) return XKV_ERR_INVALID_ARG;
+  // nothing of this handle may be in flight while its scratch is replaced
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+  const int c = g->dev.c;
+  const int old_cap = g->k_cap_max;
+  g->k_cap_max = (int)(((int64_t)g->cfg.k_max + c - 1) / c) * c + n_outliers * c;
+  if (g->k_cap_max > old_cap) {
+    // the partial results of reconstruct+attend are sized by the largest row count of a selection
+    const size_t pf0 = attend_part_floats(g), pf1 = fused_part_floats(g);
+    const size_t bytes = (pf0 > pf1 ? pf0 : pf1) * sizeof(float);
+    void* p = nullptr;
+    e = cudaMalloc(&p, bytes ? bytes : 16);
+    if (e != cudaSuccess) {
+      g->k_cap_max = old_cap;
+      set_cuda_error(e);
+      (void)cudaGetLastError();
+      return e == cudaErrorMemoryAllocation ? XKV_ERR_OOM : XKV_ERR_CUDA;
+    }
+    for (int i = 0; i < g->n_owned; ++i) {
+      if (g->owned[i] == (void*)g->dev.part) { cudaFree(g->owned[i]); g->owned[i] = p; }
+    }
+    g->dev.part = (float*)p;
+  }
+  g->dev.outliers = n_outliers > 0 ? outliers : nullptr;
+  g->dev.n_out = n_outliers;
+  return XKV_OK;
+}
+
 int xkv_tail_workspace_bytes(const xkv_group* g, int32_t tail_cap, uint64_t* bytes) {
   if (!g || !bytes || tail_cap < 1 || tail_cap > XKV_TAIL_MAX_ROWS) return XKV_ERR_INVALID_ARG;
   *bytes = (uint64_t)tail_part_floats(g, tail_cap) * sizeof(float);

@@ -36,6 +36,8 @@ struct GroupDev {
   float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
   float* part;                      // attention partials, see xkv_attend.cu
   unsigned int* flags;              // device flag word
+  const int32_t* outliers;          // [batch][G][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
+  int n_out;
 };
 
 }  // namespace xkv

@@ -163,8 +163,8 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, i
 // by an ordered compaction.  CACHED: n_c fits one super-block and the keys stay in registers.
 template <bool CACHED>
 __global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel_idx,
-            int32_t* __restrict__ sel_cnt) {
+topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out,
+            int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
   __shared__ uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_tot[kTopkThreads / 32];
   __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
@@ -279,8 +279,52 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
   }
 
   // Ordered compaction: chunk j is taken if key > thr, or key == thr and fewer than need_eq equal
-  // keys precede it.  Positions follow ascending j.
+  // keys precede it, or (Algorithm 2 line 5) it is one of the head's static outlier chunks.  Positions follow
+  // ascending j.
+  __shared__ uint32_t obits[kTopkThreads * kTopkItems / 32];   // outlier chunks of the current super-block
+  __shared__ uint32_t sh_last_taken;
+  // packed (low 16 bits, high 16 bits) exclusive prefix over the CTA in thread order; the total goes to sh_a
+  auto block_scan = [&](uint32_t mine) -> uint32_t {
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t t = warp_tot[lane];
+      uint32_t ti = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, ti, o);
+        if (lane >= o) ti += v;
+      }
+      warp_tot[lane] = ti - t;                      // exclusive prefix of warp totals
+      if (lane == 31) sh_a = ti;                    // super-block total
+    }
+    __syncthreads();
+    return inc - mine + warp_tot[warp];
+  };
+  auto write_chunk = [&](uint32_t pos, int j) {
+    const int rows = min(c, T - j * c);
+    if (c == 8 && rows == 8 && out_vec) {
+      int4* o4 = reinterpret_cast<int4*>(out + (size_t)pos * 8);
+      o4[0] = make_int4(j * 8, j * 8 + 1, j * 8 + 2, j * 8 + 3);
+      o4[1] = make_int4(j * 8 + 4, j * 8 + 5, j * 8 + 6, j * 8 + 7);
+    } else {
+      for (int t = 0; t < rows; ++t) out[(size_t)pos * c + t] = j * c + t;
+    }
+  };
+  const int32_t* outl = nullptr;                    // this problem's outlier chunk ids
+  if (n_out > 0) {
+    const int l = (int)(prob / per_layer), b = (int)((prob / dev.H_kv) % dev.batch), g = (int)(prob % dev.H_kv);
+    outl = outliers + (((size_t)b * dev.G + l) * dev.H_kv + g) * (size_t)n_out;
+    if (tid == 0) sh_last_taken = 0;
+  }
   uint32_t run_gt = 0, run_eq = 0;                  // totals of the super-blocks already done
+  uint32_t run_taken = 0;                           // chunks written so far (outlier path)
   uint32_t last_key = 0;
   for (int base = 0; base < n_c; base += super) {
     const int j0 = base + tid * kTopkItems;
@@ -306,66 +350,71 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, int32_t* __restrict__ sel
       }
     }
     const uint32_t mine = (uint32_t)__popc(gtm) | ((uint32_t)__popc(eqm) << 16);
-    uint32_t inc = mine;                            // inclusive warp scan of packed (gt, eq) counts
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += v;
-    }
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-      const uint32_t t = warp_tot[lane];
-      uint32_t ti = t;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, ti, o);
-        if (lane >= o) ti += v;
-      }
-      warp_tot[lane] = ti - t;                      // exclusive prefix of warp totals
-      if (lane == 31) sh_a = ti;                    // super-block total
-    }
-    __syncthreads();
-    const uint32_t excl = inc - mine + warp_tot[warp];
+    const uint32_t excl = block_scan(mine);
+    const uint32_t tot1 = sh_a;
     uint32_t gt_before = run_gt + (excl & 0xffffu);
     uint32_t eq_before = run_eq + (excl >> 16);
+    if (n_out == 0) {
 #pragma unroll
-    for (int i = 0; i < kTopkItems; ++i) {
-      const bool is_gt = (gtm >> i) & 1u, is_eq = (eqm >> i) & 1u;
-      const bool take = is_gt || (is_eq && eq_before < need_eq);
-      if (take) {
-        const uint32_t pos = gt_before + min(eq_before, need_eq);
-        const int j = j0 + i;
-        const int rows = min(c, T - j * c);
-        if (c == 8 && rows == 8 && out_vec) {
-          int4* o4 = reinterpret_cast<int4*>(out + (size_t)pos * 8);
-          o4[0] = make_int4(j * 8, j * 8 + 1, j * 8 + 2, j * 8 + 3);
-          o4[1] = make_int4(j * 8 + 4, j * 8 + 5, j * 8 + 6, j * 8 + 7);
-        } else {
-          for (int t = 0; t < rows; ++t) out[(size_t)pos * c + t] = j * c + t;
+      for (int i = 0; i < kTopkItems; ++i) {
+        const bool is_gt = (gtm >> i) & 1u, is_eq = (eqm >> i) & 1u;
+        const bool take = is_gt || (is_eq && eq_before < need_eq);
+        if (take) write_chunk(gt_before + min(eq_before, need_eq), j0 + i);
+        gt_before += is_gt ? 1u : 0u;
+        eq_before += is_eq ? 1u : 0u;
+      }
+    } else {
+      // membership in the top-k first, then the union with the outlier chunks, then positions over the union
+      uint32_t takem = 0;
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) {
+        const bool is_gt = (gtm >> i) & 1u, is_eq = (eqm >> i) & 1u;
+        if (is_gt || (is_eq && eq_before < need_eq)) takem |= 1u << i;
+        gt_before += is_gt ? 1u : 0u;
+        eq_before += is_eq ? 1u : 0u;
+      }
+      for (int w = tid; w < super / 32; w += kTopkThreads) obits[w] = 0u;
+      __syncthreads();                                // also: everybody has read sh_a and warp_tot of the first scan
+      const int hi = min(base + super, n_c);
+      for (int o = tid; o < n_out; o += kTopkThreads) {
+        const int jo = outl[o];
+        if (jo >= base && jo < hi) atomicOr(&obits[(jo - base) >> 5], 1u << ((jo - base) & 31));
+      }
+      __syncthreads();
+      static_assert(kTopkItems == 16, "two threads share one word of the outlier bitmap");
+      takem |= (obits[tid >> 1] >> ((tid & 1) * 16)) & 0xffffu;
+      const uint32_t excl2 = block_scan((uint32_t)__popc(takem));
+      uint32_t pos = run_taken + excl2;
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) {
+        if ((takem >> i) & 1u) {
+          write_chunk(pos++, j0 + i);
+          if (j0 + i == n_c - 1) sh_last_taken = 1u;
         }
       }
-      gt_before += is_gt ? 1u : 0u;
-      eq_before += is_eq ? 1u : 0u;
+      run_taken += sh_a;
     }
-    run_gt += sh_a & 0xffffu;
-    run_eq += sh_a >> 16;
+    run_gt += tot1 & 0xffffu;
+    run_eq += tot1 >> 16;
     __syncthreads();
   }
-  // Row count: k_ch whole chunks unless the ragged last chunk was taken (it is then the last one).
-  const int taken = all ? n_c : k_ch;
-  // the last chunk has the highest index, so it wins a tie only if every equal key fits
+  // Row count: whole chunks unless the ragged last chunk was taken (it is then the last one).
+  // Without outliers: k_ch chunks; the last chunk has the highest index, so it wins a tie only if every equal key fits.
   __shared__ uint32_t sh_last;                    // key of chunk n_c-1, published by the thread that owns it
   {
     const int owner = ((n_c - 1) % super) / kTopkItems;
     if (tid == owner) sh_last = last_key;
     __syncthreads();
   }
-  int cnt = taken * c;
-  {
+  int cnt;
+  if (n_out == 0) {
+    cnt = (all ? n_c : k_ch) * c;
     bool last_in = all;
     if (!all) last_in = sh_last > thr || (sh_last == thr && run_eq <= need_eq);
     if (last_in) cnt -= (n_c * c - T);
+  } else {
+    cnt = (int)run_taken * c;
+    if (sh_last_taken) cnt -= (n_c * c - T);
   }
   for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
   if (tid == 0) sel_cnt[prob] = cnt;
@@ -381,7 +430,7 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   const int c = dev.c;
   const int k_ch_raw = (k + c - 1) / c;
   const int k_ch = k_ch_raw < dev.n_c ? k_ch_raw : dev.n_c;
-  const int k_cap = k_ch_raw * c;
+  const int k_cap = (k_ch_raw + dev.n_out) * c;      // room for the union with the outlier chunks
   const size_t smem = 1024 + (size_t)(dev.d_h / 64) * kScoreRows * 128 + (size_t)dev.n_rep * dev.d_h * 4;
   dim3 grid(tiles, problems);
   cudaError_t e;
@@ -398,9 +447,11 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (dev.n_c <= kTopkThreads * kTopkItems)
-    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
+                   dev.n_out, sel_idx, sel_cnt);
   else
-    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, sel_idx, sel_cnt);
+    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
+                   dev.n_out, sel_idx, sel_cnt);
   count_launch();
   return e;
 }

@@ -75,6 +75,8 @@ _lib.xkv_tail_workspace_bytes.restype = ctypes.c_int
 _lib.xkv_sr_reconstruct_attend_tail.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, ctypes.c_int32, _P, _P, _P,
                                                 ctypes.c_int32, _P, ctypes.c_uint64, _P, _P, _P]
 _lib.xkv_sr_reconstruct_attend_tail.restype = ctypes.c_int
+_lib.xkv_group_set_outliers.argtypes = [_P, _P, ctypes.c_int32, _P]
+_lib.xkv_group_set_outliers.restype = ctypes.c_int
 _lib.xkv_group_destroy.argtypes = [_P]
 _lib.xkv_group_destroy.restype = ctypes.c_int
 _lib.xkv_group_status.argtypes = [_P, ctypes.POINTER(ctypes.c_uint32), _P]
@@ -200,6 +202,14 @@ def xkv_sr_reconstruct_attend(grp: Group, layer_begin: int, layer_end: int, q, s
                                         k_cap, _ptr(out), _ptr(lse), _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_sr_reconstruct_attend")
+
+
+def xkv_group_set_outliers(grp: Group, outliers, n_outliers: int, stream=None) -> None:
+    """`outliers`: int32 device tensor [batch][G][H_kv][n_outliers]; the caller keeps it alive."""
+    st = _lib.xkv_group_set_outliers(grp.handle, _ptr(outliers), n_outliers, _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_group_set_outliers")
+    grp.outliers = outliers     # keep the borrowed tensor alive with the handle
 
 
 def xkv_tail_workspace_bytes(grp: Group, tail_cap: int) -> int:

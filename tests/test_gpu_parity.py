@@ -223,3 +223,61 @@ def test_more_chunks_than_one_topk_superblock():
         np.testing.assert_array_equal(gidx[l, 0, hk], oidx[l, 0, hk])
         assert gcnt[l, 0, hk] == ocnt[l, 0, hk]
     g.close()
+
+
+def test_selection_with_static_outliers_union():
+    """Algorithm 2 line 5: outlier chunks are united with the top-k (ascending, no repeats, variable count), then
+    reconstruct+attend runs on the longer selections."""
+    s = synth.config(1, T=2045, k=128, batch=2)                          # ragged last chunk
+    inp = C.case_from_factors(s)
+    n_out = 5
+    rng = np.random.default_rng(7)
+    outl = rng.integers(0, s.n_c, size=(s.batch, s.G, s.H_kv, n_out)).astype(np.int32)
+    outl[0, 0, 0] = [3, 3, s.n_c - 1, -4, 10 ** 6]                       # repeats, the ragged last chunk, out of range
+    g = C.GpuCase(s, inp)
+    plain_idx, plain_cnt = g.select(0)
+    outl[1, 1, 1, :2] = plain_idx[1, 1, 1, [0, 8]] // s.c                 # two outliers that the top-k already holds
+    o_dev = torch.from_numpy(outl).cuda()
+    g.xkv.xkv_group_set_outliers(g.grp, o_dev, n_out)
+    k_cap = (-(-s.k // s.c) + n_out) * s.c
+    idx = torch.full((s.G, s.batch, s.H_kv, k_cap), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((s.G, s.batch, s.H_kv), -7, dtype=torch.int32, device="cuda")
+    g.xkv.xkv_sr_select(g.grp, 0, s.G, g.inp.q[0], s.k, idx, cnt)
+    torch.cuda.synchronize()
+    gidx, gcnt = idx.cpu().numpy(), cnt.cpu().numpy()
+    oidx, ocnt, oout, olse = O.sr_decode_step(C.f32(inp.A_k), C.f32(inp.A_v), C.f32(inp.B_k), C.f32(inp.B_v),
+                                              C.f32(inp.landmarks), C.f32(inp.q[0]), k=s.k, c=s.c, H_kv=s.H_kv,
+                                              rope_base=s.rope_base, outliers=outl)
+    np.testing.assert_array_equal(gidx, oidx)
+    np.testing.assert_array_equal(gcnt, ocnt)
+    assert gcnt.min() >= plain_cnt.min() and gcnt.max() > plain_cnt.max()
+    gout, glse = g.attend(gidx, gcnt, 0)
+    assert C.rel_err(gout, oout) <= TOL
+    np.testing.assert_allclose(glse, olse, atol=2e-2)
+    # switching the union off restores the plain selection
+    g.xkv.xkv_group_set_outliers(g.grp, None, 0)
+    again_idx, again_cnt = g.select(0)
+    np.testing.assert_array_equal(again_idx, plain_idx)
+    np.testing.assert_array_equal(again_cnt, plain_cnt)
+    assert g.status() == (0, 0)
+    g.close()
+
+
+def test_outliers_with_more_chunks_than_one_superblock():
+    s = synth.config(1, T=8 * 20000, k=256, H_kv=1, H_q=2, G=1, r_k=16, r_v=16)     # n_c = 20000 > 16384
+    inp = C.case_from_factors(s)
+    n_out = 7
+    outl = np.array([[[[0, 16383, 16384, 19999, 5, 5, 12345]]]], dtype=np.int32)
+    g = C.GpuCase(s, inp)
+    o_dev = torch.from_numpy(outl).cuda()
+    g.xkv.xkv_group_set_outliers(g.grp, o_dev, n_out)
+    k_cap = (-(-s.k // s.c) + n_out) * s.c
+    idx = torch.full((s.G, s.batch, s.H_kv, k_cap), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((s.G, s.batch, s.H_kv), -7, dtype=torch.int32, device="cuda")
+    g.xkv.xkv_sr_select(g.grp, 0, s.G, g.inp.q[0], s.k, idx, cnt)
+    torch.cuda.synchronize()
+    rows = O.sr_select(C.f32(inp.q[0])[0, 0], C.f32(inp.landmarks)[0, 0, 0], s.k, s.c, s.T, outl[0, 0, 0])
+    assert cnt.item() == len(rows)
+    np.testing.assert_array_equal(idx.cpu().numpy()[0, 0, 0, :len(rows)], rows)
+    assert g.status() == (0, 0)
+    g.close()
