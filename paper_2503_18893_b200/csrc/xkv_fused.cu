@@ -791,6 +791,7 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
     pre[i] = m < r ? *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld) : make_uint4(0, 0, 0, 0);
   }
   grid_dependency_wait();                             // the partials come from the kernel launched before this one
+  grid_dependency_launch();                           // the next kernel of the stream may start its own set-up
   const float* part = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h * (r + 2);
   const int nts = tail.part ? min(tail.n_split, kTailMaxSplit) : 0;
   const size_t tstride = (size_t)n_rep * (DH + 2);

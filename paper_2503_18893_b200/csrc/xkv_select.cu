@@ -97,6 +97,7 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
     fence_mbar_init();
   }
   __syncthreads();
+  grid_dependency_wait();          // the queries may come from the kernel launched before this one
   if (threadIdx.x == 0) {
     mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
     const int y = (int)(prob_lm * dev.n_c + j0);
@@ -437,14 +438,13 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   if (dev.d_h == 128) {
     e = cudaFuncSetAttribute(score_pool_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    score_pool_kernel<128><<<grid, kScoreThreads, smem, s>>>(tmap, dev, q, l0);
+    e = launch_pdl(score_pool_kernel<128>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
   } else {
     e = cudaFuncSetAttribute(score_pool_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    score_pool_kernel<64><<<grid, kScoreThreads, smem, s>>>(tmap, dev, q, l0);
+    e = launch_pdl(score_pool_kernel<64>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
   }
   count_launch();
-  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (dev.n_c <= kTopkThreads * kTopkItems)
     e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
