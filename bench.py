@@ -51,6 +51,9 @@ def parse_args():
     ap.add_argument("--groups", type=int, default=None, help="number of windows (default: the config's)")
     ap.add_argument("--tail", type=int, default=0,
                     help="rows of uncompressed generated tokens attended to besides the selected rows (default none)")
+    ap.add_argument("--op", default="decode", choices=["decode", "landmarks"],
+                    help="decode: the hot path (default).  landmarks: the prefill-side Algorithm 1 kernel alone "
+                         "(not the headline metric; prints its own JSON line)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-problems", type=int, default=None, help="oracle sample size in (layer,head) problems")
     return ap.parse_args()
@@ -208,8 +211,49 @@ def workload_config(shape, n_gpus):
                   "between steps)"}
 
 
+def run_landmarks(args):
+    """Times xkv_build_landmarks (Algorithm 1 with 48 outlier chunks per head) on one window of the workload's keys:
+    the keys the factors represent, A_k @ B_k[l], formed with torch once outside the timed region."""
+    import torch
+    from paper_2503_18893_b200 import synth, xkv
+    torch.cuda.set_device(0)
+    s = make_shape(args)
+    A_k, _, B_k, _ = synth.make_factors(s, 0, "cuda")
+    keys = torch.stack([torch.stack([(A_k[b].float() @ B_k[b, l].float()).to(torch.bfloat16) for l in range(s.G)])
+                        for b in range(s.batch)]).contiguous()                    # (batch, G, T, d)
+    n_out = 48
+    lm = torch.empty((s.batch, s.G, s.H_kv, s.n_c, s.d_h), dtype=torch.bfloat16, device="cuda")
+    mc = torch.empty((s.G, s.batch, s.H_kv, s.n_c), dtype=torch.float32, device="cuda")
+    outl = torch.empty((s.G, s.batch, s.H_kv, n_out), dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")              # larger than L2
+    call = lambda mcos, n, o: xkv.xkv_build_landmarks(keys, lm, G=s.G, batch=s.batch, T=s.T, H_kv=s.H_kv, d_h=s.d_h,
+                                                      chunk=s.c, rope_base=s.rope_base, min_cos=mcos, n_outliers=n,
+                                                      outliers=o)
+    res = {}
+    for name, a in (("landmarks_only", (None, 0, None)), ("landmarks_min_cos_outliers", (mc, n_out, outl))):
+        ts = []
+        for i in range(args.warmup + args.steps):
+            flush.zero_()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); call(*a); e1.record()
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                ts.append(e0.elapsed_time(e1))
+        res[name] = statistics.mean(ts)
+    pk = peaks()
+    key_bytes = keys.numel() * 2 + lm.numel() * 2
+    print(json.dumps({"op": "xkv_build_landmarks", "config": workload_config(s, 1)["workload"] + " (one window)",
+                      "key_bytes": key_bytes, "ms": res, "l2": "flushed between calls",
+                      "achieved_gbs_landmarks_only": key_bytes / (res["landmarks_only"] * 1e-3) / 1e9,
+                      "frac_of_hbm_peak": key_bytes / (res["landmarks_only"] * 1e-3) / 1e9 / pk["hbm_gbs"],
+                      "peak_source": pk["source"]}))
+    return 0
+
+
 def main():
     args = parse_args()
+    if args.op == "landmarks":
+        return run_landmarks(args)
     if args.impl == "reference":
         return run_reference(args)
 

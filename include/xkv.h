@@ -116,7 +116,7 @@ XKV_API int xkv_sr_select(xkv_group* grp, int layer_begin, int layer_end, const 
 /*
  * Static outlier chunks (Algorithm 1 line 5 finds them at prefill; Algorithm 2 line 5 uses them): from now on
  * xkv_sr_select unites the top-k chunks of every (layer, sequence, KV head) with that head's outlier chunks.
- * outliers    int32 [batch][G][H_kv][n_outliers] chunk ids, device memory, BORROWED until the handle is destroyed
+ * outliers    int32 [G][batch][H_kv][n_outliers] chunk ids, device memory, BORROWED until the handle is destroyed
  *             or the list is replaced.  Ids outside [0, n_c) are ignored; a repeated id counts once.
  * n_outliers  0 <= n_outliers <= XKV_MAX_OUTLIERS; 0 (with any pointer) switches the union off.
  * With outliers the row stride of sel_idx is k_cap = (ceil(k/c) + n_outliers) * c, sel_cnt varies between
@@ -170,6 +170,32 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
                                            const void* tail_k, const void* tail_v, const int32_t* tail_len,
                                            int32_t tail_cap, void* workspace, uint64_t workspace_bytes,
                                            void* out, float* lse, void* stream);
+
+/*
+ * Algorithm 1 (App. B.1), the prefill side of the selector, for every sequence, layer and KV head g:
+ *   landmark[j]  = mean over the rows x of chunk j of rope(K[x]),  chunk j = rows c*j .. min(c*j+c, T)-1   (lines 1-3)
+ *   min_cos[j]   = min over those rows of cos(rope(K[x]), landmark[j])  (fp32, the unrounded mean; a zero vector
+ *                  has cosine 0)                                                                        (line 4)
+ *   outliers     = the n_outliers chunks with the smallest min_cos, ties to the lowest chunk id, ids ascending,
+ *                  padded with -1 if n_outliers > n_c                                                    (line 5)
+ * No handle and no allocation: everything the call needs is passed in.
+ * keys        bf16 [batch][G][T][H_kv*d_h] (head g owns columns g*d_h .. g*d_h+d_h-1), device.  With
+ *             rope_base > 0 the rows are rotated here (rotate-half, position = row, angles formed in fp64);
+ *             with rope_base <= 0 they are taken as already rotated.
+ * landmarks   out bf16 [batch][G][H_kv][n_c][d_h]: the layout xkv_group_config.landmarks expects.
+ * min_cos     out fp32 [G][batch][H_kv][n_c]; may be NULL if n_outliers == 0.
+ * outliers    out int32 [G][batch][H_kv][n_outliers]: the layout xkv_group_set_outliers expects; NULL if none.
+ * Limits: d_h in {64, 128}, H_kv * d_h <= 2048, 0 <= n_outliers <= XKV_MAX_OUTLIERS, 1 <= T < 2^24.
+ * Errors: INVALID_ARG, ARCH, CUDA.
+ */
+typedef struct {
+  uint32_t struct_size; /* sizeof(xkv_landmark_config) */
+  int32_t G, batch, T, H_kv, d_h;
+  int32_t chunk;        /* c (0 means 8) */
+  float rope_base;
+} xkv_landmark_config;
+XKV_API int xkv_build_landmarks(const xkv_landmark_config* cfg, const void* keys, void* landmarks, float* min_cos,
+                                int32_t n_outliers, int32_t* outliers, void* stream);
 
 /* Free the handle and the device memory it owns (synchronises the device first). NULL is allowed. */
 XKV_API int xkv_group_destroy(xkv_group* grp);

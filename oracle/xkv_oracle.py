@@ -307,7 +307,7 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
     If sel_idx/sel_cnt are given the selection is taken from them (any order,
     duplicates allowed) and Algorithm 2 is skipped.  `problems` restricts the
     work to a list of (l, b, g) triples (the rest of the outputs stay zero).
-    `outliers` (B,G,H_kv,o) int: static outlier chunk ids united with every selection (Algorithm 2 line 5);
+    `outliers` (G,B,H_kv,o) int: static outlier chunk ids united with every selection (Algorithm 2 line 5);
     the row stride of sel_idx is then (ceil(k/c) + o) * c.
     """
     Bsz, T, _ = A_k.shape
@@ -332,7 +332,7 @@ def sr_decode_step(A_k, A_v, B_k, B_v, landmarks, q, k, c, H_kv, rope_base, scal
         rows, o, ls = sr_decode_problem(
             qh, None if landmarks is None else landmarks[b, l, g], A_k[b], A_v[b],
             B_k[b, l][:, g * d_h:(g + 1) * d_h], B_v[b, l][:, g * d_h:(g + 1) * d_h],
-            k, c, T, rope_base, scale, rows, None if outliers is None else outliers[b, l, g])
+            k, c, T, rope_base, scale, rows, None if outliers is None else outliers[l, b, g])
         o_idx[l, b, g, :len(rows)] = rows
         o_cnt[l, b, g] = len(rows)
         out[l, b, g * n_rep:(g + 1) * n_rep] = o

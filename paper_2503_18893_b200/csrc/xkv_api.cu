@@ -298,6 +298,31 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   return XKV_OK;
 }
 
+int xkv_build_landmarks(const xkv_landmark_config* c, const void* keys, void* landmarks, float* min_cos,
+                        int32_t n_outliers, int32_t* outliers, void* stream) {
+  if (!c || c->struct_size != sizeof(xkv_landmark_config) || !keys || !landmarks) return XKV_ERR_INVALID_ARG;
+  if (c->G < 1 || c->batch < 1 || c->T < 1 || c->T >= (1 << 24) || c->H_kv < 1 || (c->d_h != 64 && c->d_h != 128) ||
+      c->H_kv * c->d_h > 2048 || c->chunk < 0 || c->chunk > 4096 || isnan(c->rope_base) || isinf(c->rope_base))
+    return XKV_ERR_INVALID_ARG;
+  if (n_outliers < 0 || n_outliers > XKV_MAX_OUTLIERS || (n_outliers > 0 && (!outliers || !min_cos))) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)keys & 1u) || ((uintptr_t)landmarks & 1u) || ((uintptr_t)min_cos & 15u) || ((uintptr_t)outliers & 3u))
+    return XKV_ERR_INVALID_ARG;
+  int device = 0, cc_major = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  if (cc_major != 10) return XKV_ERR_ARCH;
+  const int ch = c->chunk ? c->chunk : 8;
+  const int n_c = (c->T + ch - 1) / ch;
+  cudaStream_t s = (cudaStream_t)stream;
+  e = launch_landmarks((const __nv_bfloat16*)keys, (__nv_bfloat16*)landmarks, min_cos, c->G, c->batch, c->T, c->H_kv,
+                       c->d_h, ch, c->rope_base, s);
+  if (e == cudaSuccess && n_outliers > 0)
+    e = launch_topk_rows(min_cos, c->G * c->batch * c->H_kv, n_c, n_outliers, -1.0f, outliers, s);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
 int xkv_group_set_outliers(xkv_group* g, const int32_t* outliers, int32_t n_outliers, void* stream) {
   if (!g || n_outliers < 0 || n_outliers > XKV_MAX_OUTLIERS) return XKV_ERR_INVALID_ARG;
   if (n_outliers > 0 && (!outliers || ((uintptr_t)outliers & 3u))) return XKV_ERR_INVALID_ARG;

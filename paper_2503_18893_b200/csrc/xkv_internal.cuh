@@ -36,7 +36,7 @@ struct GroupDev {
   float* pooled;                    // [G][batch][H_kv][n_c] pooled landmark scores
   float* part;                      // attention partials, see xkv_attend.cu
   unsigned int* flags;              // device flag word
-  const int32_t* outliers;          // [batch][G][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
+  const int32_t* outliers;          // [G][batch][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
   int n_out;
 };
 
@@ -91,6 +91,12 @@ cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift,
 // xkv_select.cu
 cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
                           int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
+
+cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, cudaStream_t s);
+
+// xkv_landmarks.cu
+cudaError_t launch_landmarks(const __nv_bfloat16* keys, __nv_bfloat16* landmarks, float* min_cos, int G, int batch, int T,
+                             int H_kv, int d_h, int c, float rope_base, cudaStream_t s);
 
 int select_static(const xkv_select_static_config* c, int l0, int l1, const void* q, int32_t k, int32_t* sel_idx,
                   int32_t* sel_cnt, cudaStream_t s);

@@ -143,18 +143,18 @@ __device__ __forceinline__ uint32_t score_key(float f) {
 }
 
 // Keys of this thread's 16 consecutive chunks of one super-block (0 beyond n_c; callers mask by index).
-__device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, uint32_t (&key)[kTopkItems]) {
+__device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, float sign, uint32_t (&key)[kTopkItems]) {
   if (j0 + kTopkItems <= n_c && ((n_c & 3) == 0)) {
     const float4* p = reinterpret_cast<const float4*>(S + j0);
 #pragma unroll
     for (int i = 0; i < kTopkItems / 4; ++i) {
       const float4 v = p[i];
-      key[4 * i] = score_key(v.x); key[4 * i + 1] = score_key(v.y);
-      key[4 * i + 2] = score_key(v.z); key[4 * i + 3] = score_key(v.w);
+      key[4 * i] = score_key(v.x * sign); key[4 * i + 1] = score_key(v.y * sign);
+      key[4 * i + 2] = score_key(v.z * sign); key[4 * i + 3] = score_key(v.w * sign);
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < kTopkItems; ++i) key[i] = (j0 + i < n_c) ? score_key(S[j0 + i]) : 0u;
+    for (int i = 0; i < kTopkItems; ++i) key[i] = (j0 + i < n_c) ? score_key(S[j0 + i] * sign) : 0u;
   }
 }
 
@@ -164,7 +164,7 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, i
 // by an ordered compaction.  CACHED: n_c fits one super-block and the keys stay in registers.
 template <bool CACHED>
 __global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out,
+topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out, float sign,
             int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
   __shared__ uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_tot[kTopkThreads / 32];
@@ -183,7 +183,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
   grid_dependency_wait();                      // the pooled scores come from the kernel launched before
   grid_dependency_launch();
   uint32_t creg[kTopkItems];
-  if (CACHED) load_keys(S, tid * kTopkItems, n_c, creg);
+  if (CACHED) load_keys(S, tid * kTopkItems, n_c, sign, creg);
 
   uint32_t thr = 0, need_eq = 0;
   const bool all = (k_ch >= n_c);
@@ -197,7 +197,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 #pragma unroll
         for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
       } else {
-        load_keys(S, j0, n_c, key);
+        load_keys(S, j0, n_c, sign, key);
       }
 #pragma unroll
       for (int i = 0; i < kTopkItems; ++i) {
@@ -231,7 +231,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 #pragma unroll
           for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
         } else {
-          load_keys(S, j0, n_c, key);
+          load_keys(S, j0, n_c, sign, key);
         }
 #pragma unroll
         for (int i = 0; i < kTopkItems; ++i) {
@@ -320,8 +320,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
   };
   const int32_t* outl = nullptr;                    // this problem's outlier chunk ids
   if (n_out > 0) {
-    const int l = (int)(prob / per_layer), b = (int)((prob / dev.H_kv) % dev.batch), g = (int)(prob % dev.H_kv);
-    outl = outliers + (((size_t)b * dev.G + l) * dev.H_kv + g) * (size_t)n_out;
+    outl = outliers + (size_t)prob * (size_t)n_out;          // [G][batch][H_kv][n_out], like sel_idx
     if (tid == 0) sh_last_taken = 0;
   }
   uint32_t run_gt = 0, run_eq = 0;                  // totals of the super-blocks already done
@@ -339,7 +338,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 #pragma unroll
         for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
       } else {
-        load_keys(S, j0, n_c, key);
+        load_keys(S, j0, n_c, sign, key);
       }
 #pragma unroll
       for (int i = 0; i < kTopkItems; ++i) {
@@ -418,7 +417,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
     if (sh_last_taken) cnt -= (n_c * c - T);
   }
   for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
-  if (tid == 0) sel_cnt[prob] = cnt;
+  if (tid == 0 && sel_cnt) sel_cnt[prob] = cnt;
 }
 
 }  // namespace
@@ -448,10 +447,28 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   if (e != cudaSuccess) return e;
   if (dev.n_c <= kTopkThreads * kTopkItems)
     e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
-                   dev.n_out, sel_idx, sel_cnt);
+                   dev.n_out, 1.0f, sel_idx, sel_cnt);
   else
     e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
-                   dev.n_out, sel_idx, sel_cnt);
+                   dev.n_out, 1.0f, sel_idx, sel_cnt);
+  count_launch();
+  return e;
+}
+
+// The k entries with the largest sign * scores[p][j] of each of `problems` score rows of length n, ids ascending
+// (ties to the lowest id), padded with -1: out [problems][k].  Used for the static outlier chunks (Algorithm 1 line 5).
+cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, cudaStream_t s) {
+  GroupDev dev{};
+  dev.G = 1; dev.batch = problems; dev.H_kv = 1; dev.T = n; dev.c = 1; dev.n_c = n;
+  dev.pooled = const_cast<float*>(scores);
+  const int k_ch = k < n ? k : n;
+  cudaError_t e;
+  if (n <= kTopkThreads * kTopkItems)
+    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, 0, k_ch, k, (const int32_t*)nullptr, 0,
+                   sign, out, (int32_t*)nullptr);
+  else
+    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, 0, k_ch, k, (const int32_t*)nullptr, 0,
+                   sign, out, (int32_t*)nullptr);
   count_launch();
   return e;
 }

@@ -75,6 +75,16 @@ _lib.xkv_tail_workspace_bytes.restype = ctypes.c_int
 _lib.xkv_sr_reconstruct_attend_tail.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, ctypes.c_int32, _P, _P, _P,
                                                 ctypes.c_int32, _P, ctypes.c_uint64, _P, _P, _P]
 _lib.xkv_sr_reconstruct_attend_tail.restype = ctypes.c_int
+
+
+class xkv_landmark_config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("G", ctypes.c_int32), ("batch", ctypes.c_int32),
+                ("T", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("d_h", ctypes.c_int32), ("chunk", ctypes.c_int32),
+                ("rope_base", ctypes.c_float)]
+
+
+_lib.xkv_build_landmarks.argtypes = [ctypes.POINTER(xkv_landmark_config), _P, _P, _P, ctypes.c_int32, _P, _P]
+_lib.xkv_build_landmarks.restype = ctypes.c_int
 _lib.xkv_group_set_outliers.argtypes = [_P, _P, ctypes.c_int32, _P]
 _lib.xkv_group_set_outliers.restype = ctypes.c_int
 _lib.xkv_group_destroy.argtypes = [_P]
@@ -204,8 +214,18 @@ def xkv_sr_reconstruct_attend(grp: Group, layer_begin: int, layer_end: int, q, s
         raise XKVError(st, "xkv_sr_reconstruct_attend")
 
 
+def xkv_build_landmarks(keys, landmarks, *, G, batch, T, H_kv, d_h, chunk=8, rope_base=10000.0, min_cos=None,
+                        n_outliers=0, outliers=None, stream=None) -> None:
+    """Algorithm 1 on device tensors in the layouts of include/xkv.h."""
+    cfg = xkv_landmark_config(ctypes.sizeof(xkv_landmark_config), G, batch, T, H_kv, d_h, chunk, rope_base)
+    st = _lib.xkv_build_landmarks(ctypes.byref(cfg), _ptr(keys), _ptr(landmarks), _ptr(min_cos), n_outliers,
+                                  _ptr(outliers), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_build_landmarks")
+
+
 def xkv_group_set_outliers(grp: Group, outliers, n_outliers: int, stream=None) -> None:
-    """`outliers`: int32 device tensor [batch][G][H_kv][n_outliers]; the caller keeps it alive."""
+    """`outliers`: int32 device tensor [G][batch][H_kv][n_outliers]; the caller keeps it alive."""
     st = _lib.xkv_group_set_outliers(grp.handle, _ptr(outliers), n_outliers, _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_group_set_outliers")

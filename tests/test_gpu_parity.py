@@ -232,7 +232,7 @@ def test_selection_with_static_outliers_union():
     inp = C.case_from_factors(s)
     n_out = 5
     rng = np.random.default_rng(7)
-    outl = rng.integers(0, s.n_c, size=(s.batch, s.G, s.H_kv, n_out)).astype(np.int32)
+    outl = rng.integers(0, s.n_c, size=(s.G, s.batch, s.H_kv, n_out)).astype(np.int32)
     outl[0, 0, 0] = [3, 3, s.n_c - 1, -4, 10 ** 6]                       # repeats, the ragged last chunk, out of range
     g = C.GpuCase(s, inp)
     plain_idx, plain_cnt = g.select(0)

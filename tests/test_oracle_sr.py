@@ -414,15 +414,15 @@ def test_step_with_outliers_layout_and_count():
     B_k, B_v = _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h))), _bf(rng.standard_normal((Bsz, G, r, H_kv * d_h)))
     lm = _bf(rng.standard_normal((Bsz, G, H_kv, n_c, d_h)))
     q = _bf(rng.standard_normal((G, Bsz, H_kv * n_rep, d_h)))
-    outl = rng.integers(0, n_c, size=(Bsz, G, H_kv, 3))
+    outl = rng.integers(0, n_c, size=(G, Bsz, H_kv, 3))
     idx, cnt, out, lse = O.sr_decode_step(A_k, A_v, B_k, B_v, lm, q, 16, c, H_kv, 10000.0, outliers=outl)
     assert idx.shape[-1] == (2 + 3) * c
     for l in range(G):
         for b in range(Bsz):
             for g in range(H_kv):
-                rows = O.sr_select(q[l, b, g * n_rep:(g + 1) * n_rep], lm[b, l, g], 16, c, T, outl[b, l, g])
+                rows = O.sr_select(q[l, b, g * n_rep:(g + 1) * n_rep], lm[b, l, g], 16, c, T, outl[l, b, g])
                 assert cnt[l, b, g] == len(rows)
                 np.testing.assert_array_equal(idx[l, b, g, :len(rows)], rows)
                 assert np.all(idx[l, b, g, len(rows):] == -1)
-                for j in outl[b, l, g]:
+                for j in outl[l, b, g]:
                     assert j * c in rows
