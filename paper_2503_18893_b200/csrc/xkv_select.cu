@@ -134,6 +134,7 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
 constexpr int kTopkThreads = 1024;
 constexpr int kTopkItems = 16;    // consecutive chunks per thread and super-block
 constexpr int kTopkBins = 2048;   // histogram bins per radix pass
+constexpr int kTopkCand = 256;    // at most this many keys are ranked against one another directly
 
 // Order-preserving map float -> uint32 (larger float = larger key), with -0 folded onto +0.
 __device__ __forceinline__ uint32_t score_key(float f) {
@@ -169,7 +170,7 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
   __shared__ uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_tot[kTopkThreads / 32];
   __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
-  __shared__ uint32_t sh_a, sh_b;
+  __shared__ uint32_t sh_a, sh_b, sh_c;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_layer = dev.batch * dev.H_kv;
@@ -264,19 +265,56 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
       __syncthreads();
       const uint32_t above = warp_tot[warp] + (suf - mine);    // keys in bins above 2t+1
       if (above < need && above + mine >= need) {              // exactly one thread
-        if (above + h1 >= need) { sh_a = 2 * tid + 1; sh_b = need - above; }
-        else { sh_a = 2 * tid; sh_b = need - above - h1; }
+        if (above + h1 >= need) { sh_a = 2 * tid + 1; sh_b = need - above; sh_c = h1; }
+        else { sh_a = 2 * tid; sh_b = need - above - h1; sh_c = h0; }
       }
       __syncthreads();
-      const uint32_t bsel = sh_a;
+      const uint32_t bsel = sh_a, in_bin = sh_c;
       need = sh_b;
       lo += bsel << sh;
       span = min(span - (bsel << sh), (sh ? (1u << sh) : 1u) - 1u);
       __syncthreads();
-      if (sh == 0) break;
+      if (sh == 0) { thr = lo; need_eq = need; break; }
+      if (in_bin <= (uint32_t)kTopkCand) {
+        // Few keys are left in the window: collect them (in any order) and rank them against one another.
+        // The `need`-th largest of them is the threshold; need_eq = how many keys equal to it are still wanted.
+        uint32_t* cand = hist;
+        if (tid == 0) sh_a = 0;
+        __syncthreads();
+        for (int base = 0; base < n_c; base += super) {
+          uint32_t key[kTopkItems];
+          const int j0 = base + tid * kTopkItems;
+          if (CACHED) {
+#pragma unroll
+            for (int i = 0; i < kTopkItems; ++i) key[i] = creg[i];
+          } else {
+            load_keys(S, j0, n_c, sign, key);
+          }
+#pragma unroll
+          for (int i = 0; i < kTopkItems; ++i) {
+            if (j0 + i < n_c && key[i] >= lo && key[i] - lo <= span) cand[atomicAdd(&sh_a, 1u)] = key[i];
+          }
+        }
+        __syncthreads();
+        const uint32_t n_cand = sh_a;                          // == in_bin
+        __syncthreads();
+        if ((uint32_t)tid < n_cand) {
+          const uint32_t mykey = cand[tid];
+          uint32_t gt = 0, eq = 0;
+          for (uint32_t i = 0; i < n_cand; ++i) {
+            const uint32_t c2 = cand[i];
+            gt += c2 > mykey ? 1u : 0u;
+            eq += c2 == mykey ? 1u : 0u;
+          }
+          if (gt < need && need <= gt + eq) { sh_a = mykey; sh_b = need - gt; }   // equal keys write the same pair
+        }
+        __syncthreads();
+        thr = sh_a;
+        need_eq = sh_b;
+        __syncthreads();
+        break;
+      }
     }
-    thr = lo;
-    need_eq = need;
   }
 
   // Ordered compaction: chunk j is taken if key > thr, or key == thr and fewer than need_eq equal
@@ -355,13 +393,15 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
     uint32_t gt_before = run_gt + (excl & 0xffffu);
     uint32_t eq_before = run_eq + (excl >> 16);
     if (n_out == 0) {
-#pragma unroll
-      for (int i = 0; i < kTopkItems; ++i) {
-        const bool is_gt = (gtm >> i) & 1u, is_eq = (eqm >> i) & 1u;
-        const bool take = is_gt || (is_eq && eq_before < need_eq);
-        if (take) write_chunk(gt_before + min(eq_before, need_eq), j0 + i);
-        gt_before += is_gt ? 1u : 0u;
-        eq_before += is_eq ? 1u : 0u;
+      // only a few percent of the chunks are taken: walk the set bits instead of all items
+      uint32_t m = gtm | eqm;
+      while (m) {
+        const int i = __ffs(m) - 1;
+        m &= m - 1;
+        const uint32_t below = (1u << i) - 1u;
+        const uint32_t g_b = gt_before + (uint32_t)__popc(gtm & below), e_b = eq_before + (uint32_t)__popc(eqm & below);
+        const bool is_gt = (gtm >> i) & 1u;
+        if (is_gt || e_b < need_eq) write_chunk(g_b + min(e_b, need_eq), j0 + i);
       }
     } else {
       // membership in the top-k first, then the union with the outlier chunks, then positions over the union
