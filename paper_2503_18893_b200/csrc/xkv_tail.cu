@@ -64,14 +64,20 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
   const __nv_bfloat16* Kh = tail_k + head_rows * DH;
   const __nv_bfloat16* Vh = tail_v + head_rows * DH;
   constexpr int PPR = DH / 8;                          // 16-byte pieces per row
+  // two copy groups: the logits start as soon as the keys are in, the values land meanwhile
   for (int i = tid; i < rows * PPR; i += kTailThreads) {
     const int r = i / PPR, c = i % PPR;
     ptx::cp_async16(ptx::smem_u32(k_s + r * KS + c * 16), Kh + (size_t)r * DH + c * 8, 16u);
+  }
+  ptx::cp_async_commit();
+  for (int i = tid; i < rows * PPR; i += kTailThreads) {
+    const int r = i / PPR, c = i % PPR;
     ptx::cp_async16(ptx::smem_u32(v_s + r * DH + c * 8), Vh + (size_t)r * DH + c * 8, 16u);
   }
+  ptx::cp_async_commit();
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
   for (int i = tid; i < NR * DH; i += kTailThreads) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
-  asm volatile("cp.async.wait_all;" ::: "memory");
+  ptx::cp_async_wait<1>();                             // the keys of this thread's copies are in
   __syncthreads();
 
   // ---- logits of row `tid` against every head
@@ -122,6 +128,7 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
     const float mn = m_s[h];
     p_s[h * kTailThreads + tid] = (valid && mn != -INFINITY) ? exp2f(z[h] - mn) : 0.0f;
   }
+  ptx::cp_async_wait<0>();                             // the values too
   __syncthreads();
   // ---- value phase: thread -> output column d and, for d_h = 64, one half of the tile's rows
   constexpr int PARTS = kTailThreads / DH;
