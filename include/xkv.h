@@ -185,8 +185,10 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
  * landmarks   out bf16 [batch][G][H_kv][n_c][d_h]: the layout xkv_group_config.landmarks expects.
  * min_cos     out fp32 [G][batch][H_kv][n_c]; may be NULL if n_outliers == 0.
  * outliers    out int32 [G][batch][H_kv][n_outliers]: the layout xkv_group_set_outliers expects; NULL if none.
- * Limits: d_h in {64, 128}, H_kv * d_h <= 2048, 0 <= n_outliers <= XKV_MAX_OUTLIERS, 1 <= T < 2^24.
- * Errors: INVALID_ARG, ARCH, CUDA.
+ * Limits: d_h in {64, 128}; H_kv * d_h / 16 (threads per key row) must divide 256, i.e. H_kv * d_h is a power of
+ * two between 64 and 4096 (else UNSUPPORTED); keys and landmarks 16-byte aligned; 0 <= n_outliers <=
+ * XKV_MAX_OUTLIERS; 1 <= T < 2^24.
+ * Errors: INVALID_ARG, UNSUPPORTED, ARCH, CUDA.
  */
 typedef struct {
   uint32_t struct_size; /* sizeof(xkv_landmark_config) */

@@ -302,9 +302,11 @@ int xkv_build_landmarks(const xkv_landmark_config* c, const void* keys, void* la
                         int32_t n_outliers, int32_t* outliers, void* stream) {
   if (!c || c->struct_size != sizeof(xkv_landmark_config) || !keys || !landmarks) return XKV_ERR_INVALID_ARG;
   if (c->G < 1 || c->batch < 1 || c->T < 1 || c->T >= (1 << 24) || c->H_kv < 1 || (c->d_h != 64 && c->d_h != 128) ||
-      c->H_kv * c->d_h > 2048 || c->chunk < 0 || c->chunk > 4096 || isnan(c->rope_base) || isinf(c->rope_base))
+      c->H_kv * c->d_h > 4096 || c->chunk < 0 || c->chunk > 4096 || isnan(c->rope_base) || isinf(c->rope_base))
     return XKV_ERR_INVALID_ARG;
   if (n_outliers < 0 || n_outliers > XKV_MAX_OUTLIERS || (n_outliers > 0 && (!outliers || !min_cos))) return XKV_ERR_INVALID_ARG;
+  if (256 % (c->H_kv * c->d_h / 16) != 0) return XKV_ERR_UNSUPPORTED;   // threads per key row must divide the CTA
+  if (((uintptr_t)keys & 15u) || ((uintptr_t)landmarks & 15u)) return XKV_ERR_INVALID_ARG;   // 16-byte loads and stores
   if (((uintptr_t)keys & 1u) || ((uintptr_t)landmarks & 1u) || ((uintptr_t)min_cos & 15u) || ((uintptr_t)outliers & 3u))
     return XKV_ERR_INVALID_ARG;
   int device = 0, cc_major = 0;
