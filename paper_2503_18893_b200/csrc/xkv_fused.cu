@@ -74,10 +74,19 @@ __host__ __device__ constexpr Bars bar_layout(int na) {
 // cta that owns global tile t when cta i owns tiles [i*N/C, (i+1)*N/C)
 __host__ __device__ __forceinline__ int cta_of_tile(long long t, int C, int N) { return (int)(((t + 1) * C - 1) / N); }
 
-struct Ctx {
+// PROF = false: `prof` is a compile-time null pointer and every diagnostic branch of the kernel folds away (the
+// loops of the kernel have to stay small: the warps of a scheduler share its instruction cache).
+template <bool PROF>
+struct CtxT {
   volatile int* abort;
   unsigned int* flags;
-  unsigned long long* prof;   // per-CTA diagnostic counters (cycles), nullptr unless profiling was requested
+  unsigned long long* prof;   // per-CTA diagnostic counters (cycles)
+};
+template <>
+struct CtxT<false> {
+  volatile int* abort;
+  unsigned int* flags;
+  static constexpr unsigned long long* prof = nullptr;
 };
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -86,6 +95,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait on an mbarrier phase.  Returns false if another thread of the CTA has given up, or if the
 // phase does not complete within kWaitLimitNs (then this thread raises the flag and makes the others give up).
+template <class Ctx>
 __device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
@@ -101,6 +111,7 @@ __device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_
   return false;
 }
 // `slot` >= 0 (passed warp-uniformly by one warp per role when diagnostics are on) adds the cycles waited.
+template <class Ctx>
 __device__ __forceinline__ bool wait_bar(const Ctx& c, uint32_t bar, uint32_t parity, int slot = -1) {
   if (c.prof == nullptr || slot < 0) return wait_bar_raw(c, bar, parity);
   const long long c0 = clock64();
@@ -179,7 +190,7 @@ __host__ __device__ constexpr int ring_slots() {
 
 // NR: query heads per KV head rounded up to 4, 8 or 16.  WB: most 128-column blocks of r_v (registers of the
 // value epilogue): NR * WB <= 64.
-template <int DH, int NR, int WB>
+template <int DH, int NR, int WB, bool PROF>
 __global__ void __launch_bounds__(kThreads, 1)
 sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched sc, const __nv_bfloat16* __restrict__ q,
                 const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt) {
@@ -208,7 +219,10 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int word) { return bar0 + 8u * (uint32_t)word; };
-  Ctx ctx{abort_flag, dev.flags, sc.prof ? sc.prof + (size_t)blockIdx.x * 64 : nullptr};
+  CtxT<PROF> ctx;
+  ctx.abort = abort_flag;
+  ctx.flags = dev.flags;
+  if constexpr (PROF) ctx.prof = sc.prof ? sc.prof + (size_t)blockIdx.x * 64 : nullptr;
   // the staged rotary path needs the fine table to cover exactly 8 positions
   const bool rope_smem = dev.use_rope && dev.rope_shift == 3;
   // both phases are padded to an even number of 64-column slabs so that slabs pair up inside ring-slot pairs
@@ -895,11 +909,18 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   static_assert(kNB >= 2 && kNB < ring_slots<DH, NR>(), "B ring must be shorter than the row ring");
   static_assert(NR * WB <= 64 && WB <= kMaxBlocks, "value epilogue registers");
   const size_t smem = fused_smem_bytes<DH, NR>();
-  cudaError_t e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   CUtensorMap mk;
   memcpy(&mk, grp->bk_tmap, sizeof(mk));
-  e = launch_pdl(sr_fused_kernel<DH, NR, WB>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+  cudaError_t e;
+  if (grp->prof) {     // the variant with the diagnostic counters compiled in
+    e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, true>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+  } else {
+    e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+  }
   count_launch();
   if (e != cudaSuccess) return e;
   const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
