@@ -229,6 +229,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   const int nks_k = (dev.r_k + 63) >> 6, nks_v = (dev.r_v + 63) >> 6;
   const int nst_k = (nks_k + 1) & ~1, nst_v = (nks_v + 1) & ~1;
 
+  __shared__ long long ts_dbg[16];
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 128); mbar_init(BAR(bl.fullv + s), 128); }
     for (int s = 0; s < S / 2; ++s) { mbar_init(BAR(bl.emptyk + s), 1); mbar_init(BAR(bl.emptyv + s), 1); }
@@ -362,6 +363,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 #pragma unroll
         for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
         cp_async_arrive_noinc(BAR((phase ? bl.fullv : bl.full) + slot));   // arrives when this thread's copies have landed
+        if (PROF && ctx.prof && pt == 0) ts_dbg[slot] = clock64();
         if (++slot == S) slot = 0;
       }
     };
@@ -468,6 +470,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           const bool real = ks < nks_k;
           if (real && !wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
           if (!wait_bar(ctx, BAR(bl.full + slot), (seen >> slot) & 1u, ps + 3)) { ok = false; break; }
+          if (PROF && ctx.prof && lane == 0) { atomicAdd(ctx.prof + 20, (unsigned long long)(clock64() - ts_dbg[slot])); atomicAdd(ctx.prof + 21, 1ull); }
           seen ^= 1u << slot;
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
