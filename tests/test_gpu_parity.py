@@ -281,3 +281,22 @@ def test_outliers_with_more_chunks_than_one_superblock():
     np.testing.assert_array_equal(idx.cpu().numpy()[0, 0, 0, :len(rows)], rows)
     assert g.status() == (0, 0)
     g.close()
+
+
+def test_plain_tile_kernel_agrees_with_the_tensor_core_path(monkeypatch):
+    """The CUDA-core implementation that forms V_hat literally (the fallback for shapes the tensor-core kernel does
+    not cover) against the oracle and against the fused path on the same inputs."""
+    s = synth.config(1, T=2048, k=256)
+    inp = C.case_from_factors(s)
+    oidx, ocnt, oout, olse = C.oracle_step(s, inp, 0)
+    g = C.GpuCase(s, inp)
+    fout, flse = g.attend(oidx, ocnt, 0)
+    g.close()
+    monkeypatch.setenv("XKV_ATTEND_IMPL", "tile")
+    g2 = C.GpuCase(s, inp)
+    tout, tlse = g2.attend(oidx, ocnt, 0)
+    assert g2.status() == (0, 0)
+    g2.close()
+    assert C.rel_err(tout, oout) <= TOL
+    np.testing.assert_allclose(tlse, olse, atol=2e-2)
+    assert C.rel_err(tout, fout.astype(np.float64)) <= TOL
