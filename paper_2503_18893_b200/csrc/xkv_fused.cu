@@ -95,20 +95,25 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait on an mbarrier phase.  Returns false if another thread of the CTA has given up, or if the
 // phase does not complete within kWaitLimitNs (then this thread raises the flag and makes the others give up).
-template <class Ctx>
-__device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is one out-of-line function: the kernel's loops wait in dozens of places and have to stay
+// small (the warps of a scheduler share its instruction cache).
+__device__ __noinline__ bool wait_bar_slow(volatile int* abort_flag, unsigned int* flags, uint32_t bar, uint32_t parity) {
   const unsigned long long t0 = global_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 0u) {
-      if (*c.abort) return false;
+      if (*abort_flag) return false;
       if (global_ns() - t0 > kWaitLimitNs) break;
     }
   }
-  *c.abort = 1;
-  atomicOr(c.flags, XKV_FLAG_TIMEOUT);
+  *abort_flag = 1;
+  atomicOr(flags, XKV_FLAG_TIMEOUT);
   return false;
+}
+template <class Ctx>
+__device__ __forceinline__ bool wait_bar_raw(const Ctx& c, uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_bar_slow(c.abort, c.flags, bar, parity);
 }
 // `slot` >= 0 (passed warp-uniformly by one warp per role when diagnostics are on) adds the cycles waited.
 template <class Ctx>
