@@ -280,17 +280,21 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   };
   // Walks this CTA's tiles, skipping tiles that start at or beyond the problem's row count.
   struct TileIter {
-    long long t; int py, ti, cnt, l, b, g; long long prob;
+    int t, py, ti, cnt, l, b, g, pyn; long long prob;   // t: tile ordinal of the call; pyn/ti: problem and tile in it
   };
-  auto iter_begin = [&](TileIter& it_) { it_.t = t_begin - 1; it_.py = -1; it_.cnt = 0; it_.prob = 0; };
+  // the problem and tile-in-problem of the first tile, once (a division); the walk then only counts
+  const int py_first = (int)(t_begin / sc.tpp), ti_first = (int)(t_begin % sc.tpp);
+  auto iter_begin = [&](TileIter& it_) {
+    it_.t = (int)t_begin - 1; it_.py = -1; it_.cnt = 0; it_.prob = 0; it_.pyn = py_first; it_.ti = ti_first - 1;
+  };
   // advance to the next non-empty tile; returns false at the end of the range.  `on_problem(py)` runs whenever
   // the walk enters a new problem (also for problems whose tiles are all empty), before its tiles.
   auto iter_next = [&](TileIter& it_, auto&& on_problem) -> bool {
     for (;;) {
       ++it_.t;
-      if (it_.t >= t_end) return false;
-      const int py = (int)(it_.t / sc.tpp);
-      it_.ti = (int)(it_.t % sc.tpp);
+      if (it_.t >= (int)t_end) return false;
+      if (++it_.ti == sc.tpp) { it_.ti = 0; ++it_.pyn; }
+      const int py = it_.pyn;
       if (py != it_.py) {
         on_problem(py);
         it_.py = py;
