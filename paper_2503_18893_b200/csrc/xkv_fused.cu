@@ -135,10 +135,13 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
   // loops and share its instruction cache (32 pairs per pass: 77 us per call, 8: 73 us, 4: 71 us)
 #pragma unroll 1
   for (int pass = 0; pass < HALF / 4; ++pass) {
+    uint32_t xa[4], xb[4];
+    tmem_ld4_nb(acc + (uint32_t)(pass * 4), xa);
+    tmem_ld4_nb(acc + (uint32_t)(HALF + pass * 4), xb);
+    tc_wait_ld_nb(xa, xb);            // the table and query loads below do not depend on it and may be issued above it
     float x1[4], x2[4];
-    tmem_ld<4>(acc + (uint32_t)(pass * 4), x1);
-    tmem_ld<4>(acc + (uint32_t)(HALF + pass * 4), x2);
-    tc_wait_ld();
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { x1[e] = __uint_as_float(xa[e]); x2[e] = __uint_as_float(xb[e]); }
 #pragma unroll
     for (int i4 = 0; i4 < 1; ++i4) {
       float r1[4], r2[4];
@@ -824,6 +827,13 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
   const int nts = tail.part ? min(tail.n_split, kTailMaxSplit) : 0;
   const size_t tstride = (size_t)n_rep * (DH + 2);
   const float* tpart = tail.part ? tail.part + ((size_t)py * tail.n_split) * tstride + (size_t)h * (DH + 2) : nullptr;
+  // this thread's column of the first segments' partial sums: fetched together with the statistics below, so
+  // that the merge costs one round trip to L2 instead of two
+  constexpr int kSegPre = 8;
+  static_assert(kMaxBlocks * 128 <= kMergeThreads, "one rank column per thread");
+  float pv[kSegPre];
+#pragma unroll
+  for (int s = 0; s < kSegPre; ++s) pv[s] = (s < nseg && tid < r) ? __ldcg(part + s * stride + tid) : 0.0f;
   if (tid < 32) {                                     // one warp: maxima, weights of the segments, denominator
     float mx = -INFINITY;
     for (int s = tid; s < nseg; s += 32) mx = fmaxf(mx, part[s * stride + r]);
@@ -848,10 +858,12 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
     if (tid == 0) { ML_s[0] = mx; ML_s[1] = Ls; }
   }
   __syncthreads();
-  for (int m = tid; m < r; m += kMergeThreads) {
+  if (tid < r) {                                      // r <= kMergeThreads
     float acc = 0.0f;
-    for (int s = 0; s < nseg; ++s) acc = fmaf(wgt_s[s], part[s * stride + m], acc);
-    w_s[m] = acc;
+#pragma unroll
+    for (int s = 0; s < kSegPre; ++s) if (s < nseg) acc = fmaf(wgt_s[s], pv[s], acc);
+    for (int s = kSegPre; s < nseg; ++s) acc = fmaf(wgt_s[s], part[s * stride + tid], acc);
+    w_s[tid] = acc;
   }
   __syncthreads();
   float acc[8];

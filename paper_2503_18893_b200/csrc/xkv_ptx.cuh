@@ -116,6 +116,18 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&v)[N]) {
   for (int i = 0; i < N; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// The same load of 4 columns and the wait for it without the compiler-level memory barrier: ordinary loads may be
+// scheduled across them (both stay in program order with respect to each other, being volatile).  The wait takes the
+// loaded registers as in/out operands, so every use of the values is ordered after it.
+__device__ __forceinline__ void tmem_ld4_nb(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld_nb(uint32_t (&a)[4], uint32_t (&b)[4]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]));
+}
+
 // Shared-memory matrix descriptor of a K-major tile with 128-byte rows and 128-byte swizzle
 // (8-row groups 1024 bytes apart).  The tile base must be 1024-byte aligned; `byte_off` selects the
 // 32-byte K step inside the 128-byte row.
