@@ -188,7 +188,7 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
 template <int DH, int NR>
 __host__ __device__ constexpr int misc_smem_bytes() {
   return (int)(2 * kPBytes + sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR + 8 * NR) +
-               sizeof(int) * (2 * kTile + 8) + 8 * (3 * 16 + kNB + 24) + 16);
+               sizeof(int) * (3 * kTile + 8) + 8 * (3 * 16 + kNB + 24) + 16);
 }
 // Slots of the gathered-row ring: whatever fits beside the B ring.
 template <int DH, int NR>
@@ -219,8 +219,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   float* q_s = reinterpret_cast<float*>(lo_s + 8 * kRopeStride);                 // [NR][DH]
   float* alpha_s = q_s + NR * DH;                                                // [2][NR]
   float* red_s = alpha_s + 2 * NR;                                               // [2][4][NR]
-  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [2][128]
-  int* algn_s = pos_s + 2 * kTile;                                               // [2][4]
+  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [3][128]
+  int* algn_s = pos_s + 3 * kTile;                                               // [2][4]
   uint64_t* bars = reinterpret_cast<uint64_t*>(algn_s + 8);
   constexpr Bars bl = bar_layout(S);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + bl.total);
@@ -343,14 +343,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     };
     int p_next = have ? load_pos(nxt) : -1;   // row index of the next tile, fetched one tile ahead
     // one phase of one tile: the 64-column slabs of its gathered rows, in ring order
-    auto issue_phase = [&](int phase, int buf, int b) {
+    auto issue_phase = [&](int phase, int pbuf, int b) {
       const int r = phase ? dev.r_v : dev.r_k;
       const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
       const int nst = phase ? nst_v : nst_k;
       const __nv_bfloat16* rp[8];                      // this thread's piece of each of its eight rows
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const int pr = pos_s[buf * kTile + i * 16 + (pt >> 3)];
+        const int pr = pos_s[pbuf * kTile + i * 16 + (pt >> 3)];
         rp[i] = A + ((long long)b * dev.T + (pr < 0 ? 0 : pr)) * r + (int)c8 * 8;
       }
 #pragma unroll 1
@@ -382,6 +382,10 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     // Ring order: K(0), K(1), V(0), K(2), V(1), ...  The value phase of a tile needs the softmax weights that
     // the key epilogue derives from its key phase, so the next tile's key phase is put in between.
     int nv = 0, b_pend = 0;           // value phases issued; `it` counts key phases issued
+    // Row positions are kept for three tiles: the value phase of tile i is issued after the key phase of tile
+    // i+1, and a warp that runs ahead may already be publishing tile i+2 (all four warps meet at `posfull` once
+    // per tile, so nobody can be publishing tile i+3 before everybody has issued the value phase of tile i).
+    int pb_k = 0, pb_v = 0;           // position buffers of the next key phase / the next value phase
     while (ok) {
       const bool do_k = have;
       if (do_k) {
@@ -392,7 +396,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         const int buf = it & 1;
         // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
         if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
-        pos_s[buf * kTile + pt] = p;
+        pos_s[pb_k * kTile + pt] = p;
         if (rope_smem) {
           // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
           const int hidx = p < 0 ? -1 : (p >> 3);
@@ -416,13 +420,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         // publish the row positions of the tile (to the other producer threads and to the key epilogue)
         mbar_arrive(BAR(bl.posfull + buf));
         if (!wait_bar(ctx, BAR(bl.posfull + buf), (uint32_t)((it >> 1) & 1), ps + 2)) { ok = false; break; }
-        issue_phase(0, buf, cur.b);
+        issue_phase(0, pb_k, cur.b);
         if (!ok) break;
+        if (++pb_k == 3) pb_k = 0;
       }
       const int k_issued = it + (do_k ? 1 : 0);
       if (nv < k_issued - (do_k ? 1 : 0)) {
-        // positions of tile nv are still in its buffer: that buffer is next written for tile nv + 2
-        issue_phase(1, nv & 1, b_pend);
+        issue_phase(1, pb_v, b_pend);
+        if (++pb_v == 3) pb_v = 0;
         ++nv;
       } else if (!do_k) {
         break;
@@ -607,6 +612,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     bool ok = true;
     uint32_t grp_par = 0;
     const int ps = warp == 0 ? 24 : -1000;
+    int pbuf = 0;                                       // position buffer of the tile (three in rotation)
     const long long role_t0 = clock64();
     // where this row's weights go in the bf16 operand tile: [row block j/64][head][64 rows], 128-byte swizzle
     const uint32_t p_off = (uint32_t)(j >> 6) * 2048u + (uint32_t)(j & 7) * 2u;
@@ -661,7 +667,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       if (!wait_bar(ctx, BAR(bl.posfull + buf), par, ps + 1)) { ok = false; break; }   // positions published
       if (!wait_bar(ctx, BAR(bl.kfull + buf), par, ps + 2)) { ok = false; break; }
       tc_fence_after();
-      const int pos = pos_s[buf * kTile + j];
+      const int pos = pos_s[pbuf * kTile + j];
+      if (++pbuf == 3) pbuf = 0;
       const int pp = pos < 0 ? 0 : pos;
       float z[NR];
 #pragma unroll
@@ -835,17 +842,30 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
 #pragma unroll
   for (int s = 0; s < kSegPre; ++s) pv[s] = (s < nseg && tid < r) ? __ldcg(part + s * stride + tid) : 0.0f;
   if (tid < 32) {                                     // one warp: maxima, weights of the segments, denominator
+    // maxima and denominators of this lane's segments in one batch of loads
+    constexpr int kPer = (kMergeMaxSeg + 31) / 32;
+    float sm[kPer], sl[kPer];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int s = tid + 32 * i;
+      sm[i] = s < nseg ? __ldcg(part + s * stride + r) : -INFINITY;
+      sl[i] = s < nseg ? __ldcg(part + s * stride + r + 1) : 0.0f;
+    }
     float mx = -INFINITY;
-    for (int s = tid; s < nseg; s += 32) mx = fmaxf(mx, part[s * stride + r]);
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) mx = fmaxf(mx, sm[i]);
     for (int s = tid; s < nts; s += 32) mx = fmaxf(mx, tpart[s * tstride + DH]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     float Ls = 0.0f;
-    for (int s = tid; s < nseg; s += 32) {
-      const float ms = part[s * stride + r];
-      const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
-      wgt_s[s] = w;
-      Ls += w * part[s * stride + r + 1];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int s = tid + 32 * i;
+      if (s < nseg) {
+        const float w = (sm[i] == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(sm[i] - mx);
+        wgt_s[s] = w;
+        Ls += w * sl[i];
+      }
     }
     for (int s = tid; s < nts; s += 32) {
       const float ms = tpart[s * tstride + DH];
