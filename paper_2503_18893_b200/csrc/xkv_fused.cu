@@ -59,7 +59,7 @@ struct Sched {
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, fullv, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, grp, total;
+  int full, fullv, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, vfree, grp, total;
 };
 __host__ __device__ constexpr Bars bar_layout(int na) {
   Bars b{};
@@ -67,7 +67,7 @@ __host__ __device__ constexpr Bars bar_layout(int na) {
   // the kind it waits for is never confused by the other kind's completions
   b.full = 0; b.fullv = na; b.emptyk = 2 * na; b.emptyv = 2 * na + na / 2; b.bfull = 3 * na; b.kfull = b.bfull + kNB;
   b.kempty = b.kfull + 2; b.wfull = b.kempty + 2; b.wempty = b.wfull + 2; b.pfull = b.wempty + 2;
-  b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.grp = b.posfull + 2; b.total = b.grp + 1;
+  b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.vfree = b.posfull + 4; b.grp = b.vfree + 4; b.total = b.grp + 1;
   return b;
 }
 
@@ -188,7 +188,7 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
 template <int DH, int NR>
 __host__ __device__ constexpr int misc_smem_bytes() {
   return (int)(2 * kPBytes + sizeof(float2) * (2 * 16 + 8) * kRopeStride + sizeof(float) * (NR * DH + 2 * NR + 8 * NR) +
-               sizeof(int) * (3 * kTile + 8) + 8 * (3 * 16 + kNB + 24) + 16);
+               sizeof(int) * (4 * kTile + 8) + 8 * (3 * 16 + kNB + 24) + 16);
 }
 // Slots of the gathered-row ring: whatever fits beside the B ring.
 template <int DH, int NR>
@@ -210,6 +210,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   constexpr int S = ring_slots<DH, NR>();          // gathered-row slots, all of which may be in flight
   static_assert(S >= 4 && S <= 16, "ring size");   // slot pairs are tracked in 3 bits by the loader
   static_assert(kNB <= 8, "loader fifo");
+  // the row slabs are two rings: SK for the key stream, SV for the value stream (both even)
+  constexpr int SK = (S % 4 == 0) ? S / 2 : S / 2 + 1, SV = S - SK;
+  static_assert(SK >= 2 && SV >= 2 && SK % 2 == 0 && SV % 2 == 0, "ring split");
   const uint32_t bring = base + (uint32_t)S * kSlabBytes;                         // B-slab ring
   // carve-up after the two rings
   uint8_t* P_gen = gen + (size_t)(S + kNB) * kSlabBytes;                         // [2][kPBytes] bf16 weights (MMA operand)
@@ -219,8 +222,8 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   float* q_s = reinterpret_cast<float*>(lo_s + 8 * kRopeStride);                 // [NR][DH]
   float* alpha_s = q_s + NR * DH;                                                // [2][NR]
   float* red_s = alpha_s + 2 * NR;                                               // [2][4][NR]
-  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [3][128]
-  int* algn_s = pos_s + 3 * kTile;                                               // [2][4]
+  int* pos_s = reinterpret_cast<int*>(red_s + 2 * 4 * NR);                       // [4][128]
+  int* algn_s = pos_s + 4 * kTile;                                               // [2][4]
   uint64_t* bars = reinterpret_cast<uint64_t*>(algn_s + 8);
   constexpr Bars bl = bar_layout(S);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + bl.total);
@@ -237,17 +240,17 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   const int nks_k = (dev.r_k + 63) >> 6, nks_v = (dev.r_v + 63) >> 6;
   const int nst_k = (nks_k + 1) & ~1, nst_v = (nks_v + 1) & ~1;
 
-  __shared__ long long ts_dbg[16];
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 128); mbar_init(BAR(bl.fullv + s), 128); }
+    for (int s = 0; s < S; ++s) { mbar_init(BAR(bl.full + s), 64); mbar_init(BAR(bl.fullv + s), 64); }   // 64 threads per stream
     for (int s = 0; s < S / 2; ++s) { mbar_init(BAR(bl.emptyk + s), 1); mbar_init(BAR(bl.emptyv + s), 1); }
     for (int s = 0; s < kNB; ++s) mbar_init(BAR(bl.bfull + s), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(BAR(bl.kfull + b), 1); mbar_init(BAR(bl.kempty + b), 128);
       mbar_init(BAR(bl.wfull + b), 1); mbar_init(BAR(bl.wempty + b), 128);
       mbar_init(BAR(bl.pfull + b), 128);
-      mbar_init(BAR(bl.rfree + b), 128); mbar_init(BAR(bl.posfull + b), 128);
+      mbar_init(BAR(bl.rfree + b), 128);
     }
+    for (int b = 0; b < 4; ++b) { mbar_init(BAR(bl.posfull + b), 64); mbar_init(BAR(bl.vfree + b), 64); }
     mbar_init(BAR(bl.grp), 128);
     *abort_flag = 0;
     fence_mbar_init();
@@ -316,168 +319,180 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 
   if (warp >= 8 && warp < 12) {
     // =============================== producers: gather rows of A ===============================
-    // Eight consecutive lanes copy the eight 16-byte pieces of one 128-byte row slab, so that every
-    // request of a warp covers whole 128-byte lines; thread pt serves rows (pt>>3) + 16*i, i = 0..7.
-    const int pt = tid - 256, pw = warp - 8;
-    const uint32_t c8 = (uint32_t)(pt & 7);
-    int slot = 0;                     // ring position
-    // per slot pair (bit p): has it been used, was its last occupant a value-phase pair, and the parity of the
-    // number of key-phase / value-phase pairs issued into it so far
-    uint32_t occ_any = 0, occ_v = 0, cnt_k = 0, cnt_v = 0;
-    // rows (pt>>3) + 16*i share the swizzle phase (pt>>3)&7; slot-relative destination of the i = 0 piece
-    const uint32_t dst0 = (uint32_t)(pt >> 3) * 128u + ((c8 ^ ((uint32_t)(pt >> 3) & 7u)) << 4);
-    const int ps = pw == 0 ? 0 : -1000;
+    // Two independent streams with a ring of their own each: warps 8-9 gather the rows of A_k of every tile into
+    // the key ring, warps 10-11 the same rows of A_v into the value ring.  A stream waits only for releases of its
+    // own ring, so the key MMAs of consecutive tiles follow one another without waiting for the value phase that
+    // sits between them in time (with one shared ring the key slabs of tile i+2 could not be requested before the
+    // last value slab of tile i, which itself waited for the last key MMA of tile i+1).
+    // Eight consecutive lanes copy the eight 16-byte pieces of one 128-byte row slab, so that every request of a
+    // warp covers whole 128-byte lines; thread t of a stream serves rows (t>>3) + 8*i, i = 0..15.
+    const bool kstream = warp < 10;
+    const int t64 = (tid - 256) & 63, pw = (warp - 8) & 1;
+    const uint32_t c8 = (uint32_t)(t64 & 7), r8 = (uint32_t)(t64 >> 3);
+    // rows r8 + 8*i share the swizzle phase r8; slab-relative destination of the i = 0 piece
+    const uint32_t dst0 = r8 * 128u + ((c8 ^ r8) << 4);
+    const int ps = (warp == 8) ? 0 : (warp == 10 ? 48 : -1000);
     const long long role_t0 = clock64();
-    int it = 0;
+    int slot = 0;                     // position in this stream's ring
+    uint32_t used = 0, rel_par = 0;   // per slot pair: filled before; parity of the release to wait for next
+    int it = 0, pb = 0;               // tiles done; position buffer of the tile (four in rotation)
     bool ok = true;
-    TileIter cur, nxt;
-    iter_begin(nxt);
-    bool have = iter_next(nxt, no_op);
-    auto load_pos = [&](const TileIter& x) {
-      int p = -1;
-      if (x.ti * kTile + pt < x.cnt) {
-        p = sel_idx[x.prob * sc.k_cap + x.ti * kTile + pt];
-        if (p < 0 || p >= dev.T) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
-      }
-      return p;
-    };
-    int p_next = have ? load_pos(nxt) : -1;   // row index of the next tile, fetched one tile ahead
-    // one phase of one tile: the 64-column slabs of its gathered rows, in ring order
-    auto issue_phase = [&](int phase, int pbuf, int b) {
-      const int r = phase ? dev.r_v : dev.r_k;
-      const __nv_bfloat16* A = phase ? dev.A_v : dev.A_k;
-      const int nst = phase ? nst_v : nst_k;
-      const __nv_bfloat16* rp[8];                      // this thread's piece of each of its eight rows
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int pr = pos_s[pbuf * kTile + i * 16 + (pt >> 3)];
-        rp[i] = A + ((long long)b * dev.T + (pr < 0 ? 0 : pr)) * r + (int)c8 * 8;
-      }
+    const int RS = kstream ? SK : SV;                           // slabs in this stream's ring
+    const uint32_t ring0 = base + (kstream ? 0u : (uint32_t)SK * kSlabBytes) + dst0;
+    const int bar_full = kstream ? bl.full : bl.fullv, bar_empty = kstream ? bl.emptyk : bl.emptyv;
+    const int r = kstream ? dev.r_k : dev.r_v;
+    const uint32_t row_bytes = (uint32_t)r * 2u;
+    const int nst = kstream ? nst_k : nst_v;
+    const __nv_bfloat16* Abase = kstream ? dev.A_k : dev.A_v;
+    // one phase of one tile: the 64-column slabs of its gathered rows, two at a time (slots are released in
+    // pairs, one tcgen05.commit per two slabs); ro: the tile rows of this thread
+    auto issue_phase = [&](const uint32_t (&ro)[16], int b) {
+      const char* Ab = reinterpret_cast<const char*>(Abase + (long long)b * dev.T * r) + c8 * 16u;
 #pragma unroll 1
-      for (int ks = 0; ks < nst; ++ks) {
-        // slots are released in pairs (one tcgen05.commit per two slabs): when entering a pair, wait for the
-        // release of its previous occupant (occupant number c of its kind completes phase c of that barrier)
-        if ((slot & 1) == 0) {
-          const int pr = slot >> 1;
-          const uint32_t bit = 1u << pr;
-          if (occ_any & bit) {
-            const bool was_v = (occ_v & bit) != 0;
-            const uint32_t par = (((was_v ? cnt_v : cnt_k) >> pr) & 1u) ^ 1u;
-            if (!wait_bar(ctx, BAR((was_v ? bl.emptyv : bl.emptyk) + pr), par, ps + 3)) { ok = false; return; }
-          }
-          occ_any |= bit;
-          if (phase) { occ_v |= bit; cnt_v ^= bit; } else { occ_v &= ~bit; cnt_k ^= bit; }
+      for (int ks = 0; ks < nst; ks += 2) {
+        const int pr = slot >> 1;
+        const uint32_t bit = 1u << pr;
+        if (used & bit) {             // wait for the release of the pair's previous occupant
+          if (!wait_bar(ctx, BAR(bar_empty + pr), (rel_par >> pr) & 1u, ps + 3)) { ok = false; return; }
+          rel_par ^= bit;
         }
-        const uint32_t st = base + (uint32_t)slot * kSlabBytes + dst0;
-        const bool in = ks * 64 + (int)c8 * 8 < r;     // false in a ragged last slab or a padding slab: zero-fill
-        const uint32_t nbytes = in ? 16u : 0u;
-        const int adv = in ? ks * 64 : 0;
+        used |= bit;
+        const uint32_t st = ring0 + (uint32_t)slot * kSlabBytes;
+        // false in a ragged last slab or a padding slab: zero-fill (the source stays inside the row)
+        const bool in0 = ks * 64 + (int)c8 * 8 < r, in1 = (ks + 1) * 64 + (int)c8 * 8 < r;
+        const uint32_t n0 = in0 ? 16u : 0u, n1 = in1 ? 16u : 0u;
+        const char* s0 = Ab + (in0 ? ks * 128 : 0);
+        const char* s1 = Ab + (in1 ? ks * 128 + 128 : 0);
+        const uint32_t bar = BAR(bar_full + slot);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16(st + (uint32_t)i * 2048u, rp[i] + adv, nbytes);
-        cp_async_arrive_noinc(BAR((phase ? bl.fullv : bl.full) + slot));   // arrives when this thread's copies have landed
-        if (PROF && ctx.prof && pt == 0) ts_dbg[slot] = clock64();
-        if (++slot == S) slot = 0;
+        for (int i = 0; i < 16; ++i) cp_async16(st + (uint32_t)i * 1024u, s0 + (size_t)ro[i] * row_bytes, n0);
+        cp_async_arrive_noinc(bar);                        // arrives when this thread's copies have landed
+#pragma unroll
+        for (int i = 0; i < 16; ++i) cp_async16(st + kSlabBytes + (uint32_t)i * 1024u, s1 + (size_t)ro[i] * row_bytes, n1);
+        cp_async_arrive_noinc(bar + 8u);
+        slot += 2;
+        if (slot == RS) slot = 0;
       }
     };
-    // Ring order: K(0), K(1), V(0), K(2), V(1), ...  The value phase of a tile needs the softmax weights that
-    // the key epilogue derives from its key phase, so the next tile's key phase is put in between.
-    int nv = 0, b_pend = 0;           // value phases issued; `it` counts key phases issued
-    // Row positions are kept for three tiles: the value phase of tile i is issued after the key phase of tile
-    // i+1, and a warp that runs ahead may already be publishing tile i+2 (all four warps meet at `posfull` once
-    // per tile, so nobody can be publishing tile i+3 before everybody has issued the value phase of tile i).
-    int pb_k = 0, pb_v = 0;           // position buffers of the next key phase / the next value phase
-    while (ok) {
-      const bool do_k = have;
-      if (do_k) {
-        cur = nxt;
-        const int p = p_next;
-        have = iter_next(nxt, no_op);
-        if (have) p_next = load_pos(nxt);
-        const int buf = it & 1;
-        // the key epilogue must be done with this buffer's positions and rotary rows (tile it-2)
-        if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
-        pos_s[pb_k * kTile + pt] = p;
-        if (rope_smem) {
-          // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once
-          const int hidx = p < 0 ? -1 : (p >> 3);
-          int gmax = hidx;
-          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
-          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
-          gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 4));
-          const bool aligned = __all_sync(0xffffffffu, p < 0 || hidx == gmax);
-          if (lane == 0) algn_s[buf * 4 + pw] = aligned ? 1 : 0;
-          if (aligned) {
+    auto load_rows = [&](uint32_t (&ro)[16]) {             // rows without a selected token read row 0 (weight 0)
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
-              const int gm = __shfl_sync(0xffffffffu, gmax, a * 8);
-              if (lane * 2 < HALF) {
-                cp_async16(smem_u32(hi_s + (size_t)(buf * 16 + pw * 4 + a) * kRopeStride + lane * 2),
-                           dev.rope_hi + (size_t)(gm < 0 ? 0 : gm) * HALF + lane * 2, 16u);
+      for (int i = 0; i < 16; ++i) {
+        const int p = pos_s[pb * kTile + (int)r8 + 8 * i];
+        ro[i] = p < 0 ? 0u : (uint32_t)p;
+      }
+    };
+    if (kstream) {
+      // ---- key stream: also publishes the row positions and the coarse rotary rows of every tile
+      TileIter cur, nxt;
+      iter_begin(nxt);
+      bool have = iter_next(nxt, no_op);
+      // thread t loads the positions of tile rows t and t + 64, one tile ahead; the range check is made when the
+      // value is used, so that nobody waits for the load here
+      auto load_pos = [&](const TileIter& x, int row) {
+        return (x.ti * kTile + row < x.cnt) ? sel_idx[x.prob * sc.k_cap + x.ti * kTile + row] : -1;
+      };
+      auto checked = [&](const TileIter& x, int row, int p) {
+        if (x.ti * kTile + row < x.cnt && (p < 0 || p >= dev.T)) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
+        return p;
+      };
+      int pn0 = have ? load_pos(nxt, t64) : -1, pn1 = have ? load_pos(nxt, t64 + 64) : -1;
+      while (ok && have) {
+        cur = nxt;
+        const int pq[2] = {checked(cur, t64, pn0), checked(cur, t64 + 64, pn1)};
+        have = iter_next(nxt, no_op);
+        if (have) { pn0 = load_pos(nxt, t64); pn1 = load_pos(nxt, t64 + 64); }
+        const int buf = it & 1;
+        // the key epilogue must be done with this buffer's rotary rows (tile it-2), and the value stream with
+        // the positions of tile it-4
+        if (!wait_bar(ctx, BAR(bl.rfree + buf), (uint32_t)(((it >> 1) & 1) ^ 1), ps + 1)) { ok = false; break; }
+        if (it >= 4 && !wait_bar(ctx, BAR(bl.vfree + pb), (uint32_t)(((it >> 2) & 1) ^ 1), ps + 1)) { ok = false; break; }
+        pos_s[pb * kTile + t64] = pq[0];
+        pos_s[pb * kTile + t64 + 64] = pq[1];
+        if (rope_smem) {
+          // rows 8a..8a+7 of the tile usually share one coarse rotary row (a landmark chunk): stage it once.
+          // Warp pw handles the 32-row blocks pw and pw + 2 (lane = row inside the block).
+#pragma unroll
+          for (int hb = 0; hb < 2; ++hb) {
+            const int blk = pw + 2 * hb, p = pq[hb];
+            const int hidx = p < 0 ? -1 : (p >> 3);
+            int gmax = hidx;
+            gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+            gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+            gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, 4));
+            const bool aligned = __all_sync(0xffffffffu, p < 0 || hidx == gmax);
+            if (lane == 0) algn_s[buf * 4 + blk] = aligned ? 1 : 0;
+            if (aligned) {
+#pragma unroll
+              for (int a = 0; a < 4; ++a) {
+                const int gm = __shfl_sync(0xffffffffu, gmax, a * 8);
+                if (lane * 2 < HALF) {
+                  cp_async16(smem_u32(hi_s + (size_t)(buf * 16 + blk * 4 + a) * kRopeStride + lane * 2),
+                             dev.rope_hi + (size_t)(gm < 0 ? 0 : gm) * HALF + lane * 2, 16u);
+                }
               }
             }
           }
         }
-        // publish the row positions of the tile (to the other producer threads and to the key epilogue)
-        mbar_arrive(BAR(bl.posfull + buf));
-        if (!wait_bar(ctx, BAR(bl.posfull + buf), (uint32_t)((it >> 1) & 1), ps + 2)) { ok = false; break; }
-        issue_phase(0, pb_k, cur.b);
-        if (!ok) break;
-        if (++pb_k == 3) pb_k = 0;
+        // publish the row positions of the tile (to both streams and to the key epilogue)
+        mbar_arrive(BAR(bl.posfull + pb));
+        if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
+        uint32_t ro[16];
+        load_rows(ro);
+        issue_phase(ro, cur.b);
+        ++it;
+        if (++pb == 4) pb = 0;
       }
-      const int k_issued = it + (do_k ? 1 : 0);
-      if (nv < k_issued - (do_k ? 1 : 0)) {
-        issue_phase(1, pb_v, b_pend);
-        if (++pb_v == 3) pb_v = 0;
-        ++nv;
-      } else if (!do_k) {
-        break;
+    } else {
+      // ---- value stream
+      TileIter cur;
+      iter_begin(cur);
+      while (ok && iter_next(cur, no_op)) {
+        if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
+        uint32_t ro[16];
+        load_rows(ro);
+        mbar_arrive(BAR(bl.vfree + pb));                   // this thread is done with the position buffer
+        issue_phase(ro, cur.b);
+        ++it;
+        if (++pb == 4) pb = 0;
       }
-      if (do_k) { b_pend = cur.b; ++it; }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
-    if (ctx.prof && pt == 0) { ctx.prof[0] = (unsigned long long)(clock64() - role_t0); ctx.prof[4] = (unsigned long long)it; }
+    if (ctx.prof && (warp == 8 || warp == 10) && lane == 0) {
+      ctx.prof[ps] = (unsigned long long)(clock64() - role_t0);
+      if (warp == 8) ctx.prof[4] = (unsigned long long)it;
+    }
   } else if (warp == 12 || warp == 14) {
     // =============================== MMA issue: warp 12 the key phases, warp 14 the value phases ===============
-    // Both walk the same ring order; each steps over the other's stages.  Two issuing threads, because one thread
-    // spends 70-130 cycles per tcgen05.mma and about 235 per tcgen05.commit.
+    // Two issuing threads, each walking its own ring (one thread spends 70-130 cycles per tcgen05.mma and about
+    // 235 per tcgen05.commit).
     const bool kside = warp == 12;
     // the whole warp walks the loop (all values are warp-uniform); one lane issues the tensor-core instructions
     constexpr uint32_t idesc_k = idesc_bf16_f32(128, 128);                     // keys: both operands K-major
     constexpr uint32_t idesc_v = idesc_bf16_f32(128, 16) | (1u << 15);         // values: A is read along its rows (MN-major)
     const int ps = kside ? 8 : 40;
     const long long role_t0 = clock64();
-    int slot = 0, bslot = 0;                          // positions in the two rings and their round parities
+    int slot = 0, bslot = 0;                          // positions in the row ring and the B ring
     uint32_t bring_par = 0;
-    // The `full` barriers are per slot and per kind of occupant (key-phase or value-phase slab), and this warp is
-    // the only one that releases its kind: it sees every phase of its barriers in order, so one parity bit per
-    // slot is enough.  With one barrier per slot for both kinds, the warp that steps over the other kind's stage
-    // could be lapped by it or test it too early, and a one-bit parity cannot tell those cases apart.
+    // This warp is the only consumer of its ring's `full` barriers and sees every phase of them in order, so one
+    // parity bit per slot is enough.
     uint32_t seen = 0;
     // descriptors differ between slots only in the start-address field (units of 16 bytes)
     const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
     const uint32_t rows_lo0 = (uint32_t)(smem_desc_sw128(base, 0) & 0xFFFFFFFFull);
     const uint32_t b_lo0 = (uint32_t)(smem_desc_sw128(bring, 0) & 0xFFFFFFFFull);
-    // value phase: A = two adjacent row slabs read transposed (64 rank columns each, 16384 bytes apart),
-    // rows advance in 8-row groups of 1024 bytes; B = the weights of 16 heads x 16 rows
-    const uint32_t rows_t_lo0 = (rows_lo0 & 0xFFFFu) | ((uint32_t)(kSlabBytes >> 4) << 16);
+    // value phase: A = two adjacent row slabs of the value ring read transposed (64 rank columns each, 16384
+    // bytes apart), rows advance in 8-row groups of 1024 bytes; B = the weights of 16 heads x 16 rows
+    const uint32_t rows_t_lo0 = (((rows_lo0 & 0xFFFFu) + (uint32_t)SK * (kSlabBytes >> 4)) & 0xFFFFu) | ((uint32_t)(kSlabBytes >> 4) << 16);
     const uint32_t p_lo0 = (uint32_t)(smem_desc_sw128(P_addr, 0) & 0xFFFFFFFFull);
-    int it = 0, nv = 0;               // key phases and value phases issued
-    bool ok = true, more = true;
+    int it = 0;
+    bool ok = true;
     TileIter cur;
     iter_begin(cur);
-    // same order as the producers: K(0), K(1), V(0), K(2), V(1), ...
-    while (ok) {
-      const bool do_k = more && iter_next(cur, no_op);
-      if (!do_k) more = false;
-      // ---- keys: K_hat = A_k[S] B_k
-      const long long ph0 = ctx.prof ? clock64() : 0;
-      if (do_k && !kside) {
-        slot += nst_k;
-        while (slot >= S) slot -= S;
-        ++it;
-      } else if (do_k) {
-        const int buf = it & 1;
-        const uint32_t par = (uint32_t)((it >> 1) & 1);
+    while (ok && iter_next(cur, no_op)) {
+      const int buf = it & 1;
+      const uint32_t par = (uint32_t)((it >> 1) & 1);
+      if (kside) {
+        // ---- keys: K_hat = A_k[S] B_k
         const int last_kk = (((dev.r_k - 1) & 63) >> 4) + 1;    // 16-column steps in the last real slab
         const uint32_t acc = tmem + (uint32_t)(buf * 128);
         if (!wait_bar(ctx, BAR(bl.kempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
@@ -487,7 +502,6 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           const bool real = ks < nks_k;
           if (real && !wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
           if (!wait_bar(ctx, BAR(bl.full + slot), (seen >> slot) & 1u, ps + 3)) { ok = false; break; }
-          if (PROF && ctx.prof && lane == 0) { atomicAdd(ctx.prof + 20, (unsigned long long)(clock64() - ts_dbg[slot])); atomicAdd(ctx.prof + 21, 1ull); }
           seen ^= 1u << slot;
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
@@ -507,22 +521,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           }
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
-          if (++slot == S) slot = 0;
+          if (++slot == SK) slot = 0;
           if (real && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
-        if (!ok) break;
-        ++it;
-      }
-      const long long ph1 = ctx.prof ? clock64() : 0;
-      if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + ps + 6, (unsigned long long)(ph1 - ph0)); }
-      // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
-      if (nv < it - (do_k ? 1 : 0) && kside) {
-        slot += nst_v;
-        while (slot >= S) slot -= S;
-        ++nv;
-      } else if (nv < it - (do_k ? 1 : 0)) {
-        const int buf = nv & 1;
-        const uint32_t par = (uint32_t)((nv >> 1) & 1);
+      } else {
+        // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
         if (!wait_bar(ctx, BAR(bl.wempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
         if (!wait_bar(ctx, BAR(bl.pfull + buf), par, ps + 5)) { ok = false; break; }
         tc_fence_after();
@@ -549,14 +552,10 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
           slot += 2;
-          if (slot == S) slot = 0;
+          if (slot == SV) slot = 0;
         }
-        if (!ok) break;
-        ++nv;
-        if (ctx.prof && lane == 0) { atomicAdd(ctx.prof + ps + 7, (unsigned long long)(clock64() - ph1)); }
-      } else if (!do_k) {
-        break;
       }
+      ++it;
     }
     if (ctx.prof && lane == 0) ctx.prof[ps] = (unsigned long long)(clock64() - role_t0);
     __syncwarp();
@@ -564,11 +563,15 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     // =============================== B_k slab loader (TMA) ===============================
     // B slab n goes to slot n % kNB, which held slab n - kNB.  That slab's MMAs are known to be complete
     //   - if it belongs to an earlier tile: when the previous tile's key accumulator was committed (kfull);
-    //   - if it belongs to this tile: when the row-ring pair of its stage was released (key-kind barrier).
+    //   - if it belongs to this tile: when the key-ring pair of its stage was released.
     // In both cases the barrier's previous phase is already known to be complete and its next phase cannot
     // complete before the slab being loaded is consumed, so the parity test is unambiguous.
+    // Without padding slabs and with at least kNB slabs per tile the second rule also covers a slab of the previous
+    // tile (the pair after next in the same ring position needs the slab being loaded): then the first slabs of a
+    // tile do not have to wait for the end of the previous tile's key phase.
+    const bool by_pair = nks_k == nst_k && nks_k >= kNB && kNB <= SK;
     int bslot = 0, it = 0, slot = 0;
-    uint32_t cnt_k = 0;                  // per slot pair: parity of the number of key-phase pairs that used it
+    uint32_t cnt_k = 0;                  // per slot pair: parity of the number of pairs that used it
     uint32_t fifo = 0;                   // per B slot, 4 bits: slot pair (3) and phase parity (1) of the slab it holds
     bool ok = true;
     TileIter cur;
@@ -579,13 +582,13 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 #pragma unroll 1
       for (int ks = 0; ks < nks_k; ++ks) {
         int sl = slot + ks;
-        while (sl >= S) sl -= S;
+        while (sl >= SK) sl -= SK;
         if ((ks & 1) == 0) {             // key stages start on even slots: entering a slot pair
           const int pr = sl >> 1;
           my = (uint32_t)pr | (((cnt_k >> pr) & 1u) << 3);
           cnt_k ^= 1u << pr;
         }
-        if (ks >= kNB) {
+        if (ks >= kNB || (by_pair && it > 0)) {
           const uint32_t e = (fifo >> (4 * bslot)) & 15u;
           if (!wait_bar(ctx, BAR(bl.emptyk + (int)(e & 7u)), e >> 3, 17)) { ok = false; break; }
         } else if (it > 0 && it * nks_k + ks >= kNB) {
@@ -596,9 +599,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, &bk_map, ks * 64, head_row, BAR(bl.bfull + bslot));
         if (++bslot == kNB) bslot = 0;
       }
-      // ring order is K(0), K(1), V(0), K(2), V(1), ...: every key phase but the first is followed by a value phase
-      slot += nst_k + (it > 0 ? nst_v : 0);
-      while (slot >= S) slot -= S;
+      // (a padding slab after an odd number of real slabs sits in the pair that was entered for the last real one)
+      slot += nst_k;
+      while (slot >= SK) slot -= SK;
       ++it;
     }
   } else if (warp < 4) {
@@ -612,7 +615,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     bool ok = true;
     uint32_t grp_par = 0;
     const int ps = warp == 0 ? 24 : -1000;
-    int pbuf = 0;                                       // position buffer of the tile (three in rotation)
+    int pbuf = 0;                                       // position buffer of the tile (four in rotation)
     const long long role_t0 = clock64();
     // where this row's weights go in the bf16 operand tile: [row block j/64][head][64 rows], 128-byte swizzle
     const uint32_t p_off = (uint32_t)(j >> 6) * 2048u + (uint32_t)(j & 7) * 2u;
@@ -664,11 +667,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     while (ok && iter_next(cur, on_problem)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
-      if (!wait_bar(ctx, BAR(bl.posfull + buf), par, ps + 1)) { ok = false; break; }   // positions published
+      if (!wait_bar(ctx, BAR(bl.posfull + pbuf), (uint32_t)((it >> 2) & 1), ps + 1)) { ok = false; break; }   // positions published
       if (!wait_bar(ctx, BAR(bl.kfull + buf), par, ps + 2)) { ok = false; break; }
       tc_fence_after();
       const int pos = pos_s[pbuf * kTile + j];
-      if (++pbuf == 3) pbuf = 0;
+      if (++pbuf == 4) pbuf = 0;
       const int pp = pos < 0 ? 0 : pos;
       float z[NR];
 #pragma unroll
