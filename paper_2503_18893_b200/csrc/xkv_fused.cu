@@ -12,19 +12,21 @@
 // so the rebuilt value rows are consumed in factored form and never materialised.  Rebuilt key rows live in
 // TMEM only.  Every gathered byte is written to shared memory once and read by the tensor core once.
 //
-// Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-11 gather producers (cp.async of the selected rows into
-// a ring of 16 KB slabs), 12 MMA issue for the key phases, 13 TMA loader of the B_k slabs (a short ring: they
-// come from L2), 14 MMA issue for the value phases.  The row ring is filled in the order K(0), K(1), V(0), K(2),
-// V(1), ...; both issuing warps walk that order and each steps over the other's stages.  Slots are released in
-// pairs by tcgen05.commit, and every barrier has exactly one kind of occupant, so that one parity bit per waiter
-// is enough.  Every wait is bounded; a wait that runs out raises XKV_FLAG_TIMEOUT and the CTA winds down.
+// Warp roles: 0-3 key epilogue, 4-7 value epilogue, 8-9 gather producers of the key stream, 10-11 of the value
+// stream (cp.async of the selected rows of A_k / A_v into two rings of 16 KB slabs, one per stream), 12 MMA issue
+// for the key phases, 13 TMA loader of the B_k slabs (a short ring: they come from L2), 14 MMA issue for the value
+// phases.  The two streams are coupled only through the data: a value phase needs the weights that the key
+// epilogue derives from the same tile's key phase.  Slots are released in pairs by tcgen05.commit; every barrier
+// has one producer side and waiters that see each of its phases in order, so that one parity bit per waiter is
+// enough.  Every wait is bounded; a wait that runs out raises XKV_FLAG_TIMEOUT and the CTA winds down.
 // The kernel starts under programmatic dependent launch: set-up overlaps the tail of the selection kernels.
 //
-// Diagnostic counters (cycles, per CTA, 64 words; see xkv_debug_read_profile): 0 producer total, 1-3 producer
-// waits (rotary buffer, positions, ring), 4 tiles; key-phase MMA warp: 8 total, 9 accumulator wait, 10 B ring,
-// 11 row ring, 12 issue, 14 phase; value-phase MMA warp: 40 total, 41 accumulator wait, 43 row ring, 44 issue,
-// 45 weights, 47 phase; 17/18 loader waits; 24 key epilogue total, 25 positions, 26 accumulator, 27 group
-// barrier, 28 weights buffer; 32 value epilogue total, 33 accumulator.
+// Diagnostic counters (cycles, per CTA, 64 words; see xkv_debug_read_profile): 0 key-stream producer total, 1-3 its
+// waits (rotary/position buffers, positions, ring), 4 tiles; 48 value-stream producer total, 50-51 its waits
+// (positions, ring); key-phase MMA warp: 8 total, 9 accumulator wait, 10 B ring, 11 row ring, 12 issue;
+// value-phase MMA warp: 40 total, 41 accumulator wait, 43 row ring, 44 issue, 45 weights; 17/18 loader waits;
+// 24 key epilogue total, 25 positions, 26 accumulator, 27 group barrier, 28 weights buffer; 32 value epilogue
+// total, 33 accumulator.
 #include <cuda.h>
 
 #include "xkv_internal.cuh"
