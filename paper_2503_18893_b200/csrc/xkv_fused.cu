@@ -186,6 +186,20 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
   }
 }
 
+// The variants that ordinary tiles do not take (no RoPE; a tile whose 8-row groups are not whole landmark chunks, or
+// a rotary table that is not staged) are kept out of line: the key epilogue's loop has to stay small.
+template <int NR>
+struct LogitsOut { float z[NR]; };
+template <int DH, int NR, bool ROPE>
+__device__ __noinline__ LogitsOut<NR> key_logits_rare(uint32_t acc, const float2* __restrict__ hi, const float2* __restrict__ lo,
+                                                      const float* __restrict__ q_s) {
+  LogitsOut<NR> o;
+#pragma unroll
+  for (int h = 0; h < NR; ++h) o.z[h] = 0.0f;
+  key_logits<DH, NR, ROPE, false>(acc, hi, lo, q_s, o.z);
+  return o;
+}
+
 // Shared memory besides the two rings: weights, rotary rows, queries, positions, barriers.
 template <int DH, int NR>
 __host__ __device__ constexpr int misc_smem_bytes() {
@@ -281,41 +295,47 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
   const int per_layer = dev.batch * dev.H_kv;
   const int n_rep = dev.n_rep;
 
-  // decode a problem ordinal of the call into (l, b, g)
-  auto prob_of = [&](int py, int& l, int& b, int& g) {
-    g = py % dev.H_kv; b = (py / dev.H_kv) % dev.batch; l = sc.l0 + py / per_layer;
-    return ((long long)l * dev.batch + b) * dev.H_kv + g;
-  };
   // Walks this CTA's tiles, skipping tiles that start at or beyond the problem's row count.
   struct TileIter {
     int t, py, ti, cnt, l, b, g, pyn; long long prob;   // t: tile ordinal of the call; pyn/ti: problem and tile in it
   };
-  // the problem and tile-in-problem of the first tile, once (a division); the walk then only counts
+  // The problem and tile-in-problem of the first tile, the (layer, sequence, head) of that problem and this CTA's
+  // segment number in it, once (divisions); the walk then only counts.  Later problems of the CTA start inside
+  // its tile range, so the CTA holds their first segment.
   const int py_first = (int)(t_begin / sc.tpp), ti_first = (int)(t_begin % sc.tpp);
+  const int g_first = py_first % dev.H_kv, b_first = (py_first / dev.H_kv) % dev.batch, l_first = sc.l0 + py_first / per_layer;
+  const int seg_first = (int)blockIdx.x - cta_of_tile((long long)py_first * sc.tpp, C, N);
   auto iter_begin = [&](TileIter& it_) {
     it_.t = (int)t_begin - 1; it_.py = -1; it_.cnt = 0; it_.prob = 0; it_.pyn = py_first; it_.ti = ti_first - 1;
   };
-  // advance to the next non-empty tile; returns false at the end of the range.  `on_problem(py)` runs whenever
-  // the walk enters a new problem (also for problems whose tiles are all empty), before its tiles.
-  auto iter_next = [&](TileIter& it_, auto&& on_problem) -> bool {
+  // advance to the next non-empty tile; returns false at the end of the range.  Whenever the walk moves to a new
+  // problem (also one whose tiles are all empty), `on_leave()` runs with the old problem still in `it_` (not before
+  // the first one) and `on_enter()` with the new one, before its tiles.
+  auto iter_next = [&](TileIter& it_, auto&& on_leave, auto&& on_enter) -> bool {
     for (;;) {
       ++it_.t;
       if (it_.t >= (int)t_end) return false;
       if (++it_.ti == sc.tpp) { it_.ti = 0; ++it_.pyn; }
       const int py = it_.pyn;
       if (py != it_.py) {
-        on_problem(py);
+        if (it_.py < 0) {
+          it_.l = l_first; it_.b = b_first; it_.g = g_first;
+        } else {
+          on_leave();
+          if (++it_.g == dev.H_kv) { it_.g = 0; if (++it_.b == dev.batch) { it_.b = 0; ++it_.l; } }
+        }
         it_.py = py;
-        it_.prob = prob_of(py, it_.l, it_.b, it_.g);
+        it_.prob = ((long long)it_.l * dev.batch + it_.b) * dev.H_kv + it_.g;
         it_.cnt = min(sel_cnt[it_.prob], sc.k_cap);
+        on_enter();
       }
       if (it_.ti * kTile < it_.cnt) return true;
     }
   };
-  auto no_op = [](int) {};
+  auto no_op = []() {};
   // partial slot of the segment (this CTA's share) of problem ordinal py
   auto part_of = [&](int py, long long prob) {
-    const int seg = (int)blockIdx.x - cta_of_tile((long long)py * sc.tpp, C, N);
+    const int seg = py == py_first ? seg_first : 0;
     return dev.part + ((size_t)prob * sc.n_slots + seg) * (size_t)n_rep * (dev.r_v + 2);
   };
 
@@ -387,7 +407,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       // ---- key stream: also publishes the row positions and the coarse rotary rows of every tile
       TileIter cur, nxt;
       iter_begin(nxt);
-      bool have = iter_next(nxt, no_op);
+      bool have = iter_next(nxt, no_op, no_op);
       // thread t loads the positions of tile rows t and t + 64, one tile ahead; the range check is made when the
       // value is used, so that nobody waits for the load here
       auto load_pos = [&](const TileIter& x, int row) {
@@ -401,7 +421,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       while (ok && have) {
         cur = nxt;
         const int pq[2] = {checked(cur, t64, pn0), checked(cur, t64 + 64, pn1)};
-        have = iter_next(nxt, no_op);
+        have = iter_next(nxt, no_op, no_op);
         if (have) { pn0 = load_pos(nxt, t64); pn1 = load_pos(nxt, t64 + 64); }
         const int buf = it & 1;
         // the key epilogue must be done with this buffer's rotary rows (tile it-2), and the value stream with
@@ -448,7 +468,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       // ---- value stream
       TileIter cur;
       iter_begin(cur);
-      while (ok && iter_next(cur, no_op)) {
+      while (ok && iter_next(cur, no_op, no_op)) {
         if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
         uint32_t ro[16];
         load_rows(ro);
@@ -490,7 +510,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     bool ok = true;
     TileIter cur;
     iter_begin(cur);
-    while (ok && iter_next(cur, no_op)) {
+    while (ok && iter_next(cur, no_op, no_op)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
       if (kside) {
@@ -500,31 +520,42 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         if (!wait_bar(ctx, BAR(bl.kempty + buf), par ^ 1u, ps + 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int ks = 0; ks < nst_k && ok; ++ks) {
-          const bool real = ks < nks_k;
-          if (real && !wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
+        for (int ks = 0; ks < nst_k && ok; ks += 2) {
+          // one ring-slot pair per iteration: wait for both slabs and their B slabs, then issue all steps at once
+          const bool real1 = ks + 1 < nks_k;             // the second slab of the last pair may be padding
+          const int bslot1 = (bslot + 1 == kNB) ? 0 : bslot + 1;
+          const uint32_t bpar1 = (bslot + 1 == kNB) ? (bring_par ^ 1u) : bring_par;
+          if (!wait_bar(ctx, BAR(bl.bfull + bslot), bring_par, ps + 2)) { ok = false; break; }
+          if (real1 && !wait_bar(ctx, BAR(bl.bfull + bslot1), bpar1, ps + 2)) { ok = false; break; }
           if (!wait_bar(ctx, BAR(bl.full + slot), (seen >> slot) & 1u, ps + 3)) { ok = false; break; }
-          seen ^= 1u << slot;
+          if (!wait_bar(ctx, BAR(bl.full + slot + 1), (seen >> (slot + 1)) & 1u, ps + 3)) { ok = false; break; }
+          seen ^= 3u << slot;
           tc_fence_after();
           const long long i0 = ctx.prof ? clock64() : 0;
           if (lane == 0) {
-            if (real) {
-              const uint64_t a_desc = desc_hi | (rows_lo0 + (uint32_t)slot * (kSlabBytes >> 4));
-              const uint64_t b_desc = desc_hi | (b_lo0 + (uint32_t)bslot * (kSlabBytes >> 4));
-              const int nkk = (ks == nks_k - 1) ? last_kk : 4;
-              tc_mma_bf16(acc, a_desc, b_desc, idesc_k, ks ? 1u : 0u);
+            const uint64_t a_desc = desc_hi | (rows_lo0 + (uint32_t)slot * (kSlabBytes >> 4));
+            const uint64_t b_desc = desc_hi | (b_lo0 + (uint32_t)bslot * (kSlabBytes >> 4));
+            const uint64_t b_desc1 = desc_hi | (b_lo0 + (uint32_t)bslot1 * (kSlabBytes >> 4));
+            const int nkk0 = (ks == nks_k - 1) ? last_kk : 4;
+            const int nkk1 = !real1 ? 0 : ((ks + 1 == nks_k - 1) ? last_kk : 4);
+            tc_mma_bf16(acc, a_desc, b_desc, idesc_k, ks ? 1u : 0u);
 #pragma unroll
-              for (int kk = 1; kk < 4; ++kk) {
-                if (kk < nkk) tc_mma_bf16(acc, a_desc + 2u * kk, b_desc + 2u * kk, idesc_k, 1u);   // +32 bytes per step
-              }
+            for (int kk = 1; kk < 4; ++kk) {
+              if (kk < nkk0) tc_mma_bf16(acc, a_desc + 2u * kk, b_desc + 2u * kk, idesc_k, 1u);   // +32 bytes per step
             }
-            if (slot & 1) tc_commit(BAR(bl.emptyk + (slot >> 1)));   // releases both slabs of the pair (and their B slabs)
-            if (ks == nst_k - 1) tc_commit(BAR(bl.kfull + buf));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              if (kk < nkk1) tc_mma_bf16(acc, a_desc + (uint32_t)(kSlabBytes >> 4) + 2u * kk, b_desc1 + 2u * kk, idesc_k, 1u);
+            }
+            tc_commit(BAR(bl.emptyk + (slot >> 1)));   // releases both slabs of the pair (and their B slabs)
+            if (ks + 2 >= nst_k) tc_commit(BAR(bl.kfull + buf));
           }
           __syncwarp();
           if (ctx.prof && lane == 0) atomicAdd(ctx.prof + ps + 4, (unsigned long long)(clock64() - i0));
-          if (++slot == SK) slot = 0;
-          if (real && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
+          slot += 2;
+          if (slot == SK) slot = 0;
+          bslot = bslot1; bring_par = bpar1;
+          if (real1 && ++bslot == kNB) { bslot = 0; bring_par ^= 1u; }
         }
       } else {
         // ---- values: W += A_v[S]^T P^T, one accumulator of 16 columns per 128 rank columns
@@ -578,7 +609,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     bool ok = true;
     TileIter cur;
     iter_begin(cur);
-    while (ok && lane == 0 && iter_next(cur, no_op)) {
+    while (ok && lane == 0 && iter_next(cur, no_op, no_op)) {
       const int head_row = (int)((((size_t)cur.b * dev.G + cur.l) * dev.H_kv + cur.g) * kDP);
       uint32_t my = 0;
 #pragma unroll 1
@@ -656,17 +687,15 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         part[1] = ls;
       }
     };
-    auto on_problem = [&](int py) {
-      if (cur.py >= 0) flush(cur.py);
-      int l, b, g;
-      prob_of(py, l, b, g);
+    auto on_leave = [&]() { flush(cur.py); };
+    auto on_enter = [&]() {
 #pragma unroll
       for (int h = 0; h < NR; ++h) { m_run[h] = -INFINITY; l_thr[h] = 0.0f; }
-      const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
+      const __nv_bfloat16* qg = q + (((long long)cur.l * dev.batch + cur.b) * dev.H_q + (long long)cur.g * n_rep) * DH;
       for (int i = j; i < NR * DH; i += 128) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
       group_sync();
     };
-    while (ok && iter_next(cur, on_problem)) {
+    while (ok && iter_next(cur, on_leave, on_enter)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
       if (!wait_bar(ctx, BAR(bl.posfull + pbuf), (uint32_t)((it >> 2) & 1), ps + 1)) { ok = false; break; }   // positions published
@@ -679,14 +708,16 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 #pragma unroll
       for (int h = 0; h < NR; ++h) z[h] = 0.0f;
       const uint32_t acc = tmem + lane_base + (uint32_t)(buf * 128);
-      if (!dev.use_rope) {
-        key_logits<DH, NR, false, false>(acc, nullptr, nullptr, q_s, z);
-      } else if (rope_smem && algn_s[buf * 4 + warp]) {
+      if (rope_smem && algn_s[buf * 4 + warp]) {
         key_logits<DH, NR, true, true>(acc, hi_s + (size_t)(buf * 16 + (j >> 3)) * kRopeStride,
                                        lo_s + (size_t)(pp & 7) * kRopeStride, q_s, z);
       } else {
-        key_logits<DH, NR, true, false>(acc, dev.rope_hi + (size_t)(pp >> dev.rope_shift) * HALF,
-                                        dev.rope_lo + (size_t)(pp & rmask) * HALF, q_s, z);
+        const LogitsOut<NR> o = dev.use_rope
+            ? key_logits_rare<DH, NR, true>(acc, dev.rope_hi + (size_t)(pp >> dev.rope_shift) * HALF,
+                                            dev.rope_lo + (size_t)(pp & rmask) * HALF, q_s)
+            : key_logits_rare<DH, NR, false>(acc, nullptr, nullptr, q_s);
+#pragma unroll
+        for (int h = 0; h < NR; ++h) z[h] = o.z[h];
       }
       tc_fence_before();
       mbar_arrive(BAR(bl.kempty + buf));                // accumulator may be overwritten
@@ -752,14 +783,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         }
       }
     };
-    auto on_problem = [&](int) {
-      if (cur.py >= 0) flush(cur.py);
+    auto on_leave = [&]() { flush(cur.py); };
+    auto on_enter = [&]() {
 #pragma unroll
       for (int bk = 0; bk < WB; ++bk)
 #pragma unroll
         for (int h = 0; h < NR; ++h) w[bk][h] = 0.0f;
     };
-    while (ok && iter_next(cur, on_problem)) {
+    while (ok && iter_next(cur, on_leave, on_enter)) {
       const int buf = it & 1;
       const uint32_t par = (uint32_t)((it >> 1) & 1);
       if (!wait_bar(ctx, BAR(bl.wfull + buf), par, ps + 1)) { ok = false; break; }
