@@ -403,25 +403,27 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         ro[i] = p < 0 ? 0u : (uint32_t)p;
       }
     };
-    if (kstream) {
-      // ---- key stream: also publishes the row positions and the coarse rotary rows of every tile
-      TileIter cur, nxt;
-      iter_begin(nxt);
-      bool have = iter_next(nxt, no_op, no_op);
-      // thread t loads the positions of tile rows t and t + 64, one tile ahead; the range check is made when the
-      // value is used, so that nobody waits for the load here
-      auto load_pos = [&](const TileIter& x, int row) {
-        return (x.ti * kTile + row < x.cnt) ? sel_idx[x.prob * sc.k_cap + x.ti * kTile + row] : -1;
-      };
-      auto checked = [&](const TileIter& x, int row, int p) {
-        if (x.ti * kTile + row < x.cnt && (p < 0 || p >= dev.T)) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
-        return p;
-      };
-      int pn0 = have ? load_pos(nxt, t64) : -1, pn1 = have ? load_pos(nxt, t64 + 64) : -1;
-      while (ok && have) {
-        cur = nxt;
-        const int pq[2] = {checked(cur, t64, pn0), checked(cur, t64 + 64, pn1)};
-        have = iter_next(nxt, no_op, no_op);
+    // One loop for both streams (one copy of the issue code).  The key stream also publishes the row positions and
+    // the coarse rotary rows of every tile: thread t loads the positions of tile rows t and t + 64, one tile ahead;
+    // the range check is made when the value is used, so that nobody waits for the load here.
+    TileIter cur, nxt;
+    iter_begin(nxt);
+    bool have = iter_next(nxt, no_op, no_op);
+    auto load_pos = [&](const TileIter& x, int row) {
+      return (x.ti * kTile + row < x.cnt) ? sel_idx[x.prob * sc.k_cap + x.ti * kTile + row] : -1;
+    };
+    auto checked = [&](const TileIter& x, int row, int p) {
+      if (x.ti * kTile + row < x.cnt && (p < 0 || p >= dev.T)) { atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE); p = -1; }
+      return p;
+    };
+    int pn0 = -1, pn1 = -1;
+    if (kstream && have) { pn0 = load_pos(nxt, t64); pn1 = load_pos(nxt, t64 + 64); }
+    while (ok && have) {
+      cur = nxt;
+      int pq[2] = {-1, -1};
+      if (kstream) { pq[0] = checked(cur, t64, pn0); pq[1] = checked(cur, t64 + 64, pn1); }
+      have = iter_next(nxt, no_op, no_op);
+      if (kstream) {
         if (have) { pn0 = load_pos(nxt, t64); pn1 = load_pos(nxt, t64 + 64); }
         const int buf = it & 1;
         // the key epilogue must be done with this buffer's rotary rows (tile it-2), and the value stream with
@@ -457,26 +459,14 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         }
         // publish the row positions of the tile (to both streams and to the key epilogue)
         mbar_arrive(BAR(bl.posfull + pb));
-        if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
-        uint32_t ro[16];
-        load_rows(ro);
-        issue_phase(ro, cur.b);
-        ++it;
-        if (++pb == 4) pb = 0;
       }
-    } else {
-      // ---- value stream
-      TileIter cur;
-      iter_begin(cur);
-      while (ok && iter_next(cur, no_op, no_op)) {
-        if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
-        uint32_t ro[16];
-        load_rows(ro);
-        mbar_arrive(BAR(bl.vfree + pb));                   // this thread is done with the position buffer
-        issue_phase(ro, cur.b);
-        ++it;
-        if (++pb == 4) pb = 0;
-      }
+      if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
+      uint32_t ro[16];
+      load_rows(ro);
+      if (!kstream) mbar_arrive(BAR(bl.vfree + pb));       // this thread is done with the position buffer
+      issue_phase(ro, cur.b);
+      ++it;
+      if (++pb == 4) pb = 0;
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     if (ctx.prof && (warp == 8 || warp == 10) && lane == 0) {
@@ -1032,9 +1022,11 @@ bool fused_supported(const xkv_group* grp) {
 
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
                          const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s, TailParts tail) {
-  const int n_rep = grp->dev.n_rep;
+  const int n_rep = grp->dev.n_rep, blocks = (grp->dev.r_v + 127) / 128;   // WB: the smallest variant that holds r_v
 #define XKV_DISPATCH(DH)                                                                                 \
+  if (n_rep <= 4 && blocks <= 4) return launch_fused_t<DH, 4, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
   if (n_rep <= 4) return launch_fused_t<DH, 4, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
+  if (n_rep <= 8 && blocks <= 4) return launch_fused_t<DH, 8, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
   if (n_rep <= 8) return launch_fused_t<DH, 8, 8>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);  \
   return launch_fused_t<DH, 16, 4>(grp, l0, l1, q, sel_idx, sel_cnt, k_cap, out, lse, s, tail);
   if (grp->dev.d_h == 128) { XKV_DISPATCH(128) }
