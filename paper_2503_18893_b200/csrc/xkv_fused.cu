@@ -713,19 +713,22 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       mbar_arrive(BAR(bl.kempty + buf));                // accumulator may be overwritten
       mbar_arrive(BAR(bl.rfree + buf));                 // positions and rotary rows of this tile are consumed
       // tile max per head over the 128 rows
+      // (one redux.sync per head on the order-preserving integer image of the float: exact, and a fraction of
+      // the code of a shuffle tree)
       float tmax[NR];
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
         z[h] = pos < 0 ? -INFINITY : z[h] * scale2;
-        float v = z[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-        tmax[h] = v;
+        int zi = __float_as_int(z[h]);
+        zi ^= (zi >> 31) & 0x7fffffff;
+        int mi = __reduce_max_sync(0xffffffffu, zi);
+        mi ^= (mi >> 31) & 0x7fffffff;
+        tmax[h] = __int_as_float(mi);
       }
       float* red = red_s + (it & 1) * 4 * NR;
       if (lane == 0) {
 #pragma unroll
-        for (int h = 0; h < NR; ++h) red[warp * NR + h] = tmax[h];
+        for (int h = 0; h < NR; ++h) red[h * 4 + warp] = tmax[h];   // [head][warp]: one 16-byte load per head below
       }
       group_sync();
       if (!ok) break;
@@ -734,10 +737,11 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       uint8_t* Pw = P_gen + buf * kPBytes + p_off;
 #pragma unroll
       for (int h = 0; h < NR; ++h) {
-        const float tm = fmaxf(fmaxf(red[h], red[NR + h]), fmaxf(red[2 * NR + h], red[3 * NR + h]));
+        const float4 t4 = *reinterpret_cast<const float4*>(red + h * 4);
+        const float tm = fmaxf(fmaxf(t4.x, t4.y), fmaxf(t4.z, t4.w));
         const float m_new = fmaxf(m_run[h], tm);
-        const float alpha = (m_run[h] == -INFINITY) ? 0.0f : exp2f(m_run[h] - m_new);
-        const float p = (m_new == -INFINITY) ? 0.0f : exp2f(z[h] - m_new);
+        const float alpha = (m_run[h] == -INFINITY) ? 0.0f : ex2_approx(m_run[h] - m_new);
+        const float p = (m_new == -INFINITY) ? 0.0f : ex2_approx(z[h] - m_new);
         const __nv_bfloat16 pb = __float2bfloat16(p);
         l_thr[h] = l_thr[h] * alpha + __bfloat162float(pb);   // the denominator sums the weights as they are used
         m_run[h] = m_new;
