@@ -12,7 +12,7 @@ namespace xkv {
 constexpr int kDP = 128;          // rows of a repacked B head block (d_h padded to 128 with zeros)
 constexpr int kMaxRep = 16;       // query heads per KV head
 constexpr int kAttTile = 128;     // selected rows per attention tile
-constexpr int kLandmarkBoxRows = 256;   // landmark rows per TMA box = chunks scored per CTA of the landmark scan
+constexpr int kLandmarkBoxRows = 64;   // landmark rows per TMA box = chunks scored per CTA of the landmark scan
 constexpr int kTailSplitRows = 128;     // tail rows per partial result
 constexpr int kTailMaxSplit = XKV_TAIL_MAX_ROWS / kTailSplitRows;
 constexpr int kMaxSplit = 64;     // most partial results per (layer, sequence, head) problem

@@ -17,7 +17,7 @@ namespace xkv {
 namespace {
 
 constexpr int kScoreRows = kLandmarkBoxRows;   // landmark rows (chunks) per CTA
-constexpr int kScoreThreads = 128;   // two rows per thread
+constexpr int kScoreThreads = 32;    // two rows per thread
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 using namespace ptx;
@@ -74,7 +74,7 @@ __device__ __forceinline__ void score_pass(uint32_t tile, const float* __restric
   }
 }
 
-// grid.x = ceil(n_c / 256) tiles, grid.y = (layers in call) * batch * H_kv problems.
+// grid.x = ceil(n_c / kScoreRows) tiles, grid.y = (layers in call) * batch * H_kv problems.
 template <int DH>
 __global__ void __launch_bounds__(kScoreThreads)
 score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const __nv_bfloat16* __restrict__ q,
