@@ -944,6 +944,10 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
     float o = 0.0f;
 #pragma unroll 4
     for (int i = f; i < RPP; i += FOLD) o += red[i * DH + d];
+    // the partial results over the uncompressed tail are already in output space; spread over all threads, so
+    // that their loads are one round trip and not a chain of them
+#pragma unroll 4
+    for (int s = f; s < nts; s += FOLD) o = fmaf(twgt_s[s], tpart[s * tstride + d], o);
     __syncthreads();
     red[f * DH + d] = o;
   }
@@ -952,8 +956,6 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
     float o = 0.0f;
 #pragma unroll
     for (int f = 0; f < FOLD; ++f) o += red[f * DH + tid];
-#pragma unroll 8
-    for (int s = 0; s < nts; ++s) o = fmaf(twgt_s[s], tpart[s * tstride + tid], o);   // the tail is already in output space
     const float M = ML_s[0], L = ML_s[1];
     const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
     out[qh * DH + tid] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
