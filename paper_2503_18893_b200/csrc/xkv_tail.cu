@@ -38,8 +38,8 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
   constexpr int KS = tail_k_stride<DH>();
   uint8_t* k_s = tail_smem;                                           // [128][KS]
   __nv_bfloat16* v_s = reinterpret_cast<__nv_bfloat16*>(k_s + kTailThreads * KS);     // [128][DH]
-  float* q_s = reinterpret_cast<float*>(v_s + kTailThreads * DH);     // [NR][DH]
-  float* p_s = q_s + NR * DH;                                         // [NR][128] weights of the tile
+  float* q_s = reinterpret_cast<float*>(v_s + kTailThreads * DH);     // [DH][NR]
+  float* p_s = q_s + NR * DH;                                         // [128][NR] weights of the tile
   __shared__ float red_s[NR * (kTailThreads / 32)];
   __shared__ float m_s[NR];
   __shared__ float fold_s[kTailThreads];               // d_h = 64: the two halves of the row range meet here
@@ -76,34 +76,47 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
   }
   ptx::cp_async_commit();
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
-  for (int i = tid; i < NR * DH; i += kTailThreads) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
+  // queries head-minor, [dim][head]: one 16-byte load gives one dimension of four heads, which pair up in the
+  // packed multiply-adds below
+  for (int i = tid; i < NR * DH; i += kTailThreads) {
+    const int h = i / DH, dd = i - h * DH;
+    q_s[dd * NR + h] = h < n_rep ? __bfloat162float(qg[i]) : 0.0f;
+  }
   ptx::cp_async_wait<1>();                             // the keys of this thread's copies are in
   __syncthreads();
 
   // ---- logits of row `tid` against every head
   const bool valid = tid < rows;
   float z[NR];
+  {
+    // two heads per fma.rn.f32x2 (each half is an ordinary fused multiply-add: same sums, half the instructions
+    // of a kernel that is bound by their number)
+    float2 z2[NR / 2];
 #pragma unroll
-  for (int h = 0; h < NR; ++h) z[h] = 0.0f;
-  if (valid) {
-    const uint4* kr = reinterpret_cast<const uint4*>(k_s + tid * KS);
-#pragma unroll 4
-    for (int cc = 0; cc < DH / 8; ++cc) {
-      const uint4 v = kr[cc];
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-      float kf[8];
+    for (int hp = 0; hp < NR / 2; ++hp) z2[hp] = make_float2(0.0f, 0.0f);
+    if (valid) {
+      const uint4* kr = reinterpret_cast<const uint4*>(k_s + tid * KS);
+#pragma unroll 2
+      for (int cc = 0; cc < DH / 8; ++cc) {
+        const uint4 v = kr[cc];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float kf[8];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) { kf[2 * e] = __uint_as_float(w[e] << 16); kf[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
+        for (int e = 0; e < 4; ++e) { kf[2 * e] = __uint_as_float(w[e] << 16); kf[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
 #pragma unroll
-      for (int h = 0; h < NR; ++h) {
-        const float4 q0 = *reinterpret_cast<const float4*>(q_s + h * DH + cc * 8);
-        const float4 q1 = *reinterpret_cast<const float4*>(q_s + h * DH + cc * 8 + 4);
-        z[h] = fmaf(q0.x, kf[0], z[h]); z[h] = fmaf(q0.y, kf[1], z[h]);
-        z[h] = fmaf(q0.z, kf[2], z[h]); z[h] = fmaf(q0.w, kf[3], z[h]);
-        z[h] = fmaf(q1.x, kf[4], z[h]); z[h] = fmaf(q1.y, kf[5], z[h]);
-        z[h] = fmaf(q1.z, kf[6], z[h]); z[h] = fmaf(q1.w, kf[7], z[h]);
+        for (int e = 0; e < 8; ++e) {
+          const float2 kk = make_float2(kf[e], kf[e]);
+#pragma unroll
+          for (int h4 = 0; h4 < NR / 4; ++h4) {
+            const float4 q4 = *reinterpret_cast<const float4*>(q_s + (cc * 8 + e) * NR + h4 * 4);
+            z2[2 * h4] = __ffma2_rn(make_float2(q4.x, q4.y), kk, z2[2 * h4]);
+            z2[2 * h4 + 1] = __ffma2_rn(make_float2(q4.z, q4.w), kk, z2[2 * h4 + 1]);
+          }
+        }
       }
     }
+#pragma unroll
+    for (int hp = 0; hp < NR / 2; ++hp) { z[2 * hp] = z2[hp].x; z[2 * hp + 1] = z2[hp].y; }
   }
   // ---- tile maximum per head
 #pragma unroll
@@ -122,29 +135,42 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
     m_s[tid] = tm;
   }
   __syncthreads();
-  // ---- weights (kept in fp32: the CUDA-core value phase has no operand format to round to)
+  // ---- weights (kept in fp32: the CUDA-core value phase has no operand format to round to), row-major and
+  // head-minor like the queries, and their sums per head
 #pragma unroll
   for (int h = 0; h < NR; ++h) {
     const float mn = m_s[h];
-    p_s[h * kTailThreads + tid] = (valid && mn != -INFINITY) ? exp2f(z[h] - mn) : 0.0f;
+    const float p = (valid && mn != -INFINITY) ? exp2f(z[h] - mn) : 0.0f;
+    p_s[tid * NR + h] = p;
+    float v = p;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;      // (the maxima in red_s were consumed before the last barrier)
   }
   ptx::cp_async_wait<0>();                             // the values too
   __syncthreads();
   // ---- value phase: thread -> output column d and, for d_h = 64, one half of the tile's rows
   constexpr int PARTS = kTailThreads / DH;
   const int d = tid % DH, vpart = tid / DH;
-  float acc[NR], l_run[NR];
+  float acc[NR];
+  {
+    float2 a2[NR / 2];
 #pragma unroll
-  for (int h = 0; h < NR; ++h) { acc[h] = 0.0f; l_run[h] = 0.0f; }
+    for (int hp = 0; hp < NR / 2; ++hp) a2[hp] = make_float2(0.0f, 0.0f);
+    const int row_lo = vpart * (kTailThreads / PARTS), row_hi = min(rows, row_lo + kTailThreads / PARTS);
 #pragma unroll 4
-  for (int jj = vpart; jj < rows; jj += PARTS) {
-    const float vv = __bfloat162float(v_s[jj * DH + d]);
+    for (int jj = row_lo; jj < row_hi; ++jj) {
+      const float vv = __bfloat162float(v_s[jj * DH + d]);
+      const float2 v2 = make_float2(vv, vv);
 #pragma unroll
-    for (int h = 0; h < NR; ++h) {
-      const float p = p_s[h * kTailThreads + jj];
-      acc[h] = fmaf(p, vv, acc[h]);
-      l_run[h] += p;                                   // every thread of a part sums the same weights
+      for (int h4 = 0; h4 < NR / 4; ++h4) {
+        const float4 p4 = *reinterpret_cast<const float4*>(p_s + jj * NR + h4 * 4);
+        a2[2 * h4] = __ffma2_rn(make_float2(p4.x, p4.y), v2, a2[2 * h4]);
+        a2[2 * h4 + 1] = __ffma2_rn(make_float2(p4.z, p4.w), v2, a2[2 * h4 + 1]);
+      }
     }
+#pragma unroll
+    for (int hp = 0; hp < NR / 2; ++hp) { acc[2 * hp] = a2[hp].x; acc[2 * hp + 1] = a2[hp].y; }
   }
 
   // ---- write the partial: [py][split][head][DH + 2]
@@ -152,15 +178,14 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
 #pragma unroll
   for (int h = 0; h < NR; ++h) {
     if (h < n_rep) {
-      float a = acc[h], ls = l_run[h];
+      float a = acc[h];
+      float ls = 0.0f;
+#pragma unroll
+      for (int w = 0; w < kTailThreads / 32; ++w) ls += red_s[h * (kTailThreads / 32) + w];
       if (PARTS > 1) {                                   // d_h = 64: add the other half of the rows
         if (vpart == 1) fold_s[d] = a;
         __syncthreads();
         if (vpart == 0) a += fold_s[d];
-        __syncthreads();
-        if (vpart == 1 && d == 0) fold_s[0] = ls;
-        __syncthreads();
-        if (vpart == 0) ls += fold_s[0];
         __syncthreads();
       }
       if (vpart == 0) {
