@@ -92,13 +92,10 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
   const long long prob_lm = ((long long)b * dev.G + l) * dev.H_kv + g;       // landmark order
   const long long prob_out = ((long long)l * dev.batch + b) * dev.H_kv + g;  // [G][batch][H_kv] order
 
-  if (threadIdx.x == 0) {
+  grid_dependency_wait();          // the queries may come from the kernel launched before this one
+  if (threadIdx.x == 0) {          // the thread that initialises the barrier also issues the loads: nothing to wait for
     mbar_init(bar, 1);
     fence_mbar_init();
-  }
-  __syncthreads();
-  grid_dependency_wait();          // the queries may come from the kernel launched before this one
-  if (threadIdx.x == 0) {
     mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
     const int y = (int)(prob_lm * dev.n_c + j0);
 #pragma unroll
