@@ -27,9 +27,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, sr_fused_kernel (95.52 + 5.15 MB) + merge_segments_kernel
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, sr_fused_kernel (95.46 + 3.38 MB) + merge_segments_kernel
 # (5.65 MB), one window of config 3
-NCU_ATTEND_DRAM_BYTES = 106.3e6
+NCU_ATTEND_DRAM_BYTES = 104.5e6
 METRIC = "SR decode steps/sec per layer group at 128K ctx"
 UNIT = "group-steps/s"
 
