@@ -5,6 +5,7 @@
 // Each CTA writes, per query head, (acc[d_h], m, l): the unnormalised output, the running maximum of the scaled
 // logits in log2 units and the sum of 2^(z - m).  The segment merge of the fused kernel folds these in.
 #include <math.h>
+#include <stdlib.h>
 
 #include "xkv_internal.cuh"
 #include "xkv_ptx.cuh"
@@ -196,6 +197,213 @@ tail_partial_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, c
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The same partials on the tensor core, for d_h = 128.  Per 128-row tile: logits S[row][head] = K q^T
+// (tcgen05.mma, M = rows, N = 16 heads, K = d_h, both operands K-major), softmax statistics and weights by
+// thread = row = TMEM lane, then O^T[d][head] = V^T P^T (A = the value tile read along its rows, MN-major,
+// B = the bf16 weights), read back by thread = d = TMEM lane.  The sixteen small MMAs replace ~2 k multiply-adds
+// per thread, so a CTA spends its time on its loads.  Weights are rounded to bf16 for the MMA; the denominator
+// sums the rounded weights, like the reconstructed rows' path does.
+constexpr int kTcSlab = kTailThreads * 128;           // 128 rows x 64 bf16, 128-byte swizzle
+constexpr uint32_t kTcWaitLimit = 1u << 22;
+
+template <int NR>
+constexpr size_t tail_tc_smem_bytes() {
+  return 1024 + 4 * (size_t)kTcSlab + 2 * 2048 + 4096 + 64;   // K and V tiles (two slabs each), q operand, weights, barriers
+}
+
+__device__ __forceinline__ bool tc_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kTcWaitLimit; ++i) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+
+template <int NR>
+__global__ void __launch_bounds__(kTailThreads)
+tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ tail_k,
+               const __nv_bfloat16* __restrict__ tail_v, const int32_t* __restrict__ tail_len, int tail_cap,
+               int n_split, float* __restrict__ part) {
+  using namespace ptx;
+  constexpr int DH = 128;
+  extern __shared__ uint8_t tc_smem[];
+  __shared__ float red_s[NR * (kTailThreads / 32)];
+  __shared__ float m_s[NR];
+  const uint32_t base = (smem_u32(tc_smem) + 1023u) & ~1023u;
+  uint8_t* gen = tc_smem + (base - smem_u32(tc_smem));
+  const uint32_t k_addr = base, v_addr = base + 2 * kTcSlab, q_addr = base + 4 * kTcSlab, p_addr = q_addr + 4096;
+  uint8_t* q_gen = gen + 4 * kTcSlab;
+  uint8_t* p_gen = q_gen + 4096;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(p_gen + 4096);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
+  const uint32_t bar_s = smem_u32(bars), bar_o = bar_s + 8;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int py = blockIdx.x, split = blockIdx.y;
+  const int per_layer = dev.batch * dev.H_kv, n_rep = dev.n_rep;
+  const int g = py % dev.H_kv, b = (py / dev.H_kv) % dev.batch, l = l0 + py / per_layer;
+  const float scale2 = dev.att_scale * kLog2e;
+
+  if (tid == 0) {
+    mbar_init(bar_s, 1);
+    mbar_init(bar_o, 1);
+    fence_mbar_init();
+  }
+  // operands that stay zero: heads that do not exist (q rows, weight rows)
+  for (int i = tid; i < 8192 / 4; i += kTailThreads) reinterpret_cast<uint32_t*>(q_gen)[i] = 0u;
+  if (warp == 0) {
+    tmem_alloc(smem_u32(tmem_slot), 32);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  grid_dependency_wait();                              // q (and the tail rows) may come from the kernel before
+  grid_dependency_launch();
+  int len = tail_len ? tail_len[b] : tail_cap;
+  if (len < 0 || len > tail_cap) {
+    if (tid == 0 && split == 0) atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE);
+    len = len < 0 ? 0 : tail_cap;
+  }
+  const int r_begin = split * kTailSplitRows;
+  const int rows = max(0, min(len - r_begin, kTailSplitRows));
+
+  // ---- stage K and V in the tensor core's layout: 64-column slabs, 128-byte rows, 16-byte units swizzled by the
+  // row; rows beyond `rows` are zero-filled (a weight of zero times garbage would still be garbage)
+  const size_t head_rows = (((size_t)l * dev.batch + b) * dev.H_kv + g) * (size_t)tail_cap + r_begin;
+  const __nv_bfloat16* Kh = tail_k + head_rows * DH;
+  const __nv_bfloat16* Vh = tail_v + head_rows * DH;
+  for (int i = tid; i < kTailThreads * 16; i += kTailThreads) {
+    const int r = i >> 4, c = i & 15;                  // row, 16-byte piece of the 256-byte row
+    const uint32_t off = (uint32_t)(c >> 3) * kTcSlab + (uint32_t)r * 128u + ((((uint32_t)c & 7u) ^ ((uint32_t)r & 7u)) << 4);
+    const uint32_t nb = r < rows ? 16u : 0u;
+    const size_t src = (size_t)(r < rows ? r : 0) * DH + c * 8;
+    cp_async16(k_addr + off, Kh + src, nb);
+    cp_async16(v_addr + off, Vh + src, nb);
+  }
+  cp_async_commit();
+  // q as the B operand of the logits: [16 heads][128 dims], K-major, same slab/swizzle scheme
+  const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
+  for (int i = tid; i < n_rep * 16; i += kTailThreads) {
+    const int h = i >> 4, c = i & 15;
+    const uint4 v = *reinterpret_cast<const uint4*>(qg + h * DH + c * 8);
+    *reinterpret_cast<uint4*>(q_gen + (c >> 3) * 2048 + h * 128 + (((c & 7) ^ (h & 7)) << 4)) = v;
+  }
+  cp_async_wait<0>();
+  fence_proxy_async();                                 // the tensor core reads what this thread wrote or copied
+  __syncthreads();
+
+  const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
+  constexpr uint32_t idesc_s = idesc_bf16_f32(128, 16);
+  constexpr uint32_t idesc_o = idesc_bf16_f32(128, 16) | (1u << 15);          // A read along its rows (MN-major)
+  // ---- logits
+  if (tid == 0) {
+    const uint32_t k_lo = (uint32_t)(smem_desc_sw128(k_addr, 0) & 0xFFFFFFFFull);
+    const uint32_t q_lo = (uint32_t)(smem_desc_sw128(q_addr, 0) & 0xFFFFFFFFull);
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {                   // 16 dims per step: 32 bytes along the row, next slab after four
+      const uint32_t a = k_lo + (uint32_t)(kk >> 2) * (kTcSlab >> 4) + (uint32_t)(kk & 3) * 2u;
+      const uint32_t bq = q_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
+      tc_mma_bf16(tmem, desc_hi | a, desc_hi | bq, idesc_s, kk ? 1u : 0u);
+    }
+    tc_commit(bar_s);
+  }
+  bool ok = tc_wait_bounded(bar_s, 0);
+  tc_fence_after();
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  const bool valid = tid < rows;
+  float z[NR];
+  if (ok) {
+    tmem_ld<NR>(tmem + lane_base, z);
+    tc_wait_ld();
+  } else {
+#pragma unroll
+    for (int h = 0; h < NR; ++h) z[h] = 0.0f;
+  }
+  // ---- tile maximum per head
+#pragma unroll
+  for (int h = 0; h < NR; ++h) {
+    z[h] = valid ? z[h] * scale2 : -INFINITY;
+    float v = z[h];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;
+  }
+  __syncthreads();
+  if (tid < NR) {
+    float tm = red_s[tid * (kTailThreads / 32)];
+#pragma unroll
+    for (int w = 1; w < kTailThreads / 32; ++w) tm = fmaxf(tm, red_s[tid * (kTailThreads / 32) + w]);
+    m_s[tid] = tm;
+  }
+  __syncthreads();
+  // ---- weights as the bf16 B operand [row block][head][64 rows] and their sums (of the rounded values)
+  {
+    uint8_t* Pw = p_gen + (tid >> 6) * 2048 + (tid & 7) * 2;
+    const uint32_t p_unit = (uint32_t)((tid & 63) >> 3);
+#pragma unroll
+    for (int h = 0; h < NR; ++h) {
+      const float mn = m_s[h];
+      const float p = (valid && mn != -INFINITY) ? ex2_approx(z[h] - mn) : 0.0f;
+      const __nv_bfloat16 pb = __float2bfloat16(p);
+      if (h < n_rep) *reinterpret_cast<__nv_bfloat16*>(Pw + h * 128 + ((p_unit ^ (uint32_t)(h & 7)) << 4)) = pb;
+      float v = __bfloat162float(pb);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;    // (the maxima were consumed before the last barrier)
+    }
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  // ---- values: O^T[d][head] = V^T P^T
+  if (tid == 0 && ok) {
+    const uint32_t v_lo = ((uint32_t)(smem_desc_sw128(v_addr, 0) & 0xFFFFull)) | ((uint32_t)(kTcSlab >> 4) << 16);
+    const uint32_t p_lo = (uint32_t)(smem_desc_sw128(p_addr, 0) & 0xFFFFFFFFull);
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {                   // 16 tile rows per step: 2048 bytes down the slab, 32 bytes along P
+      const uint32_t bp = p_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
+      tc_mma_bf16(tmem + 16u, desc_hi | (v_lo + (uint32_t)kk * (2048u >> 4)), desc_hi | bp, idesc_o, kk ? 1u : 0u);
+    }
+    tc_commit(bar_o);
+  }
+  if (ok) ok = tc_wait_bounded(bar_o, 0);
+  tc_fence_after();
+  float acc[NR];
+  if (ok) {
+    tmem_ld<NR>(tmem + lane_base + 16u, acc);
+    tc_wait_ld();
+  } else {
+    if (tid == 0) atomicOr(dev.flags, XKV_FLAG_TIMEOUT);
+#pragma unroll
+    for (int h = 0; h < NR; ++h) acc[h] = 0.0f;
+  }
+  // ---- write the partial: [py][split][head][DH + 2]
+  float* dst = part + (((size_t)py * n_split + split) * n_rep) * (DH + 2);
+#pragma unroll
+  for (int h = 0; h < NR; ++h) {
+    if (h < n_rep) {
+      dst[(size_t)h * (DH + 2) + tid] = acc[h];
+      if (tid == 0) {
+        float ls = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kTailThreads / 32; ++w) ls += red_s[h * (kTailThreads / 32) + w];
+        dst[(size_t)h * (DH + 2) + DH] = m_s[h];
+        dst[(size_t)h * (DH + 2) + DH + 1] = ls;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 32);
+  }
+}
+
 }  // namespace
 
 int tail_splits(int tail_cap) { return (tail_cap + kTailSplitRows - 1) / kTailSplitRows; }
@@ -221,12 +429,24 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
       e = launch_pdl(tail_partial_kernel<DH, NR>, grid, block, tail_smem_bytes<DH, NR>(), s, dev, l0, q, tail_k,     \
                      tail_v, tail_len, tail_cap, n_split, part);                                                    \
   } while (0)
-  if (dev.d_h == 128) {
+#define XKV_TAIL_TC(NR)                                                                                            \
+  do {                                                                                                              \
+    e = cudaFuncSetAttribute(tail_tc_kernel<NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,                       \
+                             (int)tail_tc_smem_bytes<NR>());                                                        \
+    if (e == cudaSuccess)                                                                                           \
+      e = launch_pdl(tail_tc_kernel<NR>, grid, block, tail_tc_smem_bytes<NR>(), s, dev, l0, q, tail_k, tail_v,       \
+                     tail_len, tail_cap, n_split, part);                                                            \
+  } while (0)
+  static const bool cuda_core = [] { const char* v = getenv("XKV_TAIL_IMPL"); return v && v[0] == 'c'; }();
+  if (dev.d_h == 128 && !cuda_core) {
+    if (dev.n_rep <= 4) XKV_TAIL_TC(4); else if (dev.n_rep <= 8) XKV_TAIL_TC(8); else XKV_TAIL_TC(16);
+  } else if (dev.d_h == 128) {
     if (dev.n_rep <= 4) XKV_TAIL(128, 4); else if (dev.n_rep <= 8) XKV_TAIL(128, 8); else XKV_TAIL(128, 16);
   } else {
     if (dev.n_rep <= 4) XKV_TAIL(64, 4); else if (dev.n_rep <= 8) XKV_TAIL(64, 8); else XKV_TAIL(64, 16);
   }
 #undef XKV_TAIL
+#undef XKV_TAIL_TC
   count_launch();
   return e;
 }
