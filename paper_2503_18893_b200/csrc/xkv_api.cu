@@ -203,6 +203,8 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     {
       const char* e = getenv("XKV_ATTEND_IMPL");
       g->attend_impl = (e && e[0] == 't') ? 1 : 0;
+      const char* te = getenv("XKV_TAIL_IMPL");
+      g->tail_impl = (te && te[0] == 'c') ? 1 : 0;
       const char* pe = getenv("XKV_FUSED_PROF");
       if (pe && pe[0] == '1') {
         XKV_TRY_CUDA(cudaMalloc(&p, (size_t)g->sm_count * 64 * sizeof(unsigned long long)));

@@ -58,6 +58,7 @@ struct xkv_group {
   int has_b_tmap;
   unsigned long long* prof;         // diagnostic cycle counters of the fused kernel, or nullptr
   int attend_impl;                  // 0: tensor-core fused kernel, 1: plain tile kernel
+  int tail_impl;                    // 0: tensor-core tail partials where they apply (d_h = 128), 1: CUDA-core kernel
 };
 
 namespace xkv {

@@ -1,11 +1,11 @@
 // Dense attention partials over the uncompressed tail (Sec. 4 "Implementation details": tokens generated
-// during decoding are not compressed).  The tail is short next to the factorised context, so this is a plain
-// CUDA-core kernel: one CTA per (128-row split of the tail, problem), thread = tail row for the logits,
-// thread = output column for the weighted sum of value rows.
-// Each CTA writes, per query head, (acc[d_h], m, l): the unnormalised output, the running maximum of the scaled
-// logits in log2 units and the sum of 2^(z - m).  The segment merge of the fused kernel folds these in.
+// during decoding are not compressed).  One CTA per (128-row split of the tail, problem) writes, per query head,
+// (acc[d_h], m, l): the unnormalised output, the running maximum of the scaled logits in log2 units and the sum
+// of 2^(z - m).  The segment merge of the fused kernel folds these in.  Two kernels: `tail_tc_kernel` (d_h = 128)
+// forms the tile's logits and value sums on the tensor core; `tail_partial_kernel` is the CUDA-core version
+// (thread = tail row for the logits, thread = output column for the weighted sum of value rows), used for
+// d_h = 64 and when the handle was created with XKV_TAIL_IMPL=c.
 #include <math.h>
-#include <stdlib.h>
 
 #include "xkv_internal.cuh"
 #include "xkv_ptx.cuh"
@@ -437,8 +437,7 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
       e = launch_pdl(tail_tc_kernel<NR>, grid, block, tail_tc_smem_bytes<NR>(), s, dev, l0, q, tail_k, tail_v,       \
                      tail_len, tail_cap, n_split, part);                                                            \
   } while (0)
-  static const bool cuda_core = [] { const char* v = getenv("XKV_TAIL_IMPL"); return v && v[0] == 'c'; }();
-  if (dev.d_h == 128 && !cuda_core) {
+  if (dev.d_h == 128 && !grp->tail_impl) {
     if (dev.n_rep <= 4) XKV_TAIL_TC(4); else if (dev.n_rep <= 8) XKV_TAIL_TC(8); else XKV_TAIL_TC(16);
   } else if (dev.d_h == 128) {
     if (dev.n_rep <= 4) XKV_TAIL(128, 4); else if (dev.n_rep <= 8) XKV_TAIL(128, 8); else XKV_TAIL(128, 16);

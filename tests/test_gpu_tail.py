@@ -34,8 +34,14 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("impl", ["tensor", "cuda"])
 @pytest.mark.parametrize("name,over,cap,lens", CASES, ids=[c[0] for c in CASES])
-def test_tail_parity(name, over, cap, lens):
+def test_tail_parity(name, over, cap, lens, impl, monkeypatch):
+    # d_h = 128 runs the tensor-core tail kernel unless the handle is created with XKV_TAIL_IMPL=c
+    if impl == "cuda":
+        if over.get("d_h", 128) != 128:
+            pytest.skip("d_h = 64 always takes the CUDA-core kernel")
+        monkeypatch.setenv("XKV_TAIL_IMPL", "c")
     s = synth.config(1, **over)
     inp = C.case_from_factors(s)
     rms = _key_rms(s, inp)
