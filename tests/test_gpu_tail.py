@@ -31,6 +31,8 @@ CASES = [
     ("per_sequence_lengths", dict(T=1024, k=128, batch=3), 600, [600, 0, 129]),
     ("d64_heads_16", dict(T=1024, k=128, H_kv=1, H_q=16, d_h=64, r_k=64, r_v=72), 300, [257]),
     ("qwen_like_rep7", dict(T=1024, k=128, H_kv=2, H_q=14, r_k=96, r_v=160), 1500, [1400]),
+    ("d128_heads_16", dict(T=1024, k=128, H_kv=1, H_q=16, r_k=64, r_v=72), 300, [257]),
+    ("full_tiles_only", dict(T=1024, k=128), 512, [512]),
 ]
 
 
