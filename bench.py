@@ -169,18 +169,34 @@ def oracle_sample(shape, inp, n_problems):
     return dt, len(probs), threads
 
 
+def reference_inputs(shape, n_problems):
+    """Inputs of the reference arm, prepared on the host without the CUDA library: factors from the generator,
+    landmarks by the oracle's Algorithm 1 from the keys the factors stand for -- only for the (layer, sequence,
+    head) problems the sample covers (the others stay zero and are never read)."""
+    import numpy as np
+    import torch
+    from oracle import xkv_oracle as O
+    from paper_2503_18893_b200 import synth, workload
+    f32 = lambda t: t.detach().float().cpu().numpy()
+    A_k, A_v, B_k, B_v = synth.make_factors(shape, 0, "cpu")
+    lm = np.zeros((shape.batch, shape.G, shape.H_kv, shape.n_c, shape.d_h), dtype=np.float32)
+    allp = [(l, b, g) for l in range(shape.G) for b in range(shape.batch) for g in range(shape.H_kv)]
+    for (l, b, g) in allp[:n_problems]:
+        K = O.bf16_round(f32(A_k[b]) @ f32(B_k[b, l][:, g * shape.d_h:(g + 1) * shape.d_h]))      # (T, d_h)
+        lm[b, l, g] = O.build_landmarks(K[None], shape.c, shape.rope_base)[0]
+    return workload.GroupInputs(A_k, A_v, B_k, B_v, torch.from_numpy(lm).to(torch.bfloat16),
+                                synth.make_queries(shape, 1, 0))
+
+
 def run_reference(args):
     """The reference arm: the CPU oracle on the host cores, a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    from paper_2503_18893_b200 import workload
-    import torch
     shape = make_shape(args)
-    torch.manual_seed(0)
-    inp = workload.make_group_inputs(shape, 0, 1, "cpu" if not torch.cuda.is_available() else "cuda")
     problems_per_group = shape.G * shape.batch * shape.H_kv
     n = args.cpu_problems or 2
+    inp = reference_inputs(shape, n)
     times = []
     for i in range(args.warmup + args.steps):
         dt, np_, threads = oracle_sample(shape, inp, n)

@@ -231,6 +231,37 @@ XKV_API int xkv_last_cuda_error(void);
 XKV_API uint64_t xkv_kernel_launch_count(void);
 
 /*
+ * The same count split by kernel family: counts[f] = launches of family f since load (host array of
+ * XKV_KERNEL_FAMILIES words).  Tests use it to tell which of two implementations of a step ran.
+ */
+#define XKV_KERNEL_SCAN 0      /* landmark scores + pooling (Algorithm 2 lines 2-3) */
+#define XKV_KERNEL_TOPK 1      /* top-k chunks (Algorithm 2 lines 1, 4, 5) */
+#define XKV_KERNEL_FUSED 2     /* gather + reconstruct + attention on the tensor core (Eq. 3) */
+#define XKV_KERNEL_MERGE 3     /* log-sum-exp merge of attention partials, value projection */
+#define XKV_KERNEL_TILE 4      /* the plain (CUDA-core) reconstruct + attention kernels */
+#define XKV_KERNEL_TAIL_TC 5   /* uncompressed-tail / dense attention partials on the tensor core */
+#define XKV_KERNEL_TAIL_CUDA 6 /* the same partials on CUDA cores */
+#define XKV_KERNEL_LANDMARKS 7 /* Algorithm 1 */
+#define XKV_KERNEL_PREP 8      /* handle set-up: repacking, rotary tables */
+#define XKV_KERNEL_DENSE 9     /* merge of dense-attention partials (xkv_dense_attend) */
+#define XKV_KERNEL_FAMILIES 10
+XKV_API int xkv_debug_launch_counts(uint64_t* counts);
+
+/*
+ * Host-side fault injection for tests of the give-up path (nothing here faults, traps or hangs the GPU: a wait
+ * that can never be satisfied runs into its limit, the kernel raises XKV_FLAG_TIMEOUT and returns).
+ *   XKV_INJECT_SCAN_NO_LOAD   the landmark scan does not issue its loads and waits only briefly for them; the
+ *                             pooled scores keep whatever they held, so the selection that follows is arbitrary
+ *                             (but in range).
+ *   XKV_INJECT_FUSED_NO_B     the reconstruct+attend kernel does not load the reconstruction matrices and
+ *                             waits only briefly; its output for that call is unspecified.
+ * mask = 0 restores normal operation; later calls on the handle are then correct again.
+ */
+#define XKV_INJECT_SCAN_NO_LOAD 1u
+#define XKV_INJECT_FUSED_NO_B 2u
+XKV_API int xkv_debug_set_fault_injection(xkv_group* grp, uint32_t mask);
+
+/*
  * Chunk selection for callers that must not allocate device memory.  (The paper has no counterpart: this is a
  * packaging variant of xkv_sr_select, same arithmetic, same outputs.)
  *

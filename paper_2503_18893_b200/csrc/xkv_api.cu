@@ -12,10 +12,10 @@
 namespace xkv {
 
 static thread_local int g_last_cuda_error = 0;
-static std::atomic<uint64_t> g_launches{0};
+static std::atomic<uint64_t> g_launches[kFamCount];
 
 void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
-void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+void count_launch(KernelFamily family, int n) { g_launches[family].fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 static int check_config(const xkv_group_config* c, bool need_ptrs) {
   if (!c) return XKV_ERR_INVALID_ARG;
@@ -28,6 +28,17 @@ static int check_config(const xkv_group_config* c, bool need_ptrs) {
   if (c->r_k > 8192 || c->r_v > 8192) return XKV_ERR_INVALID_ARG;
   if (c->chunk < 0 || c->chunk > 4096) return XKV_ERR_INVALID_ARG;
   if (c->k_max < 1) return XKV_ERR_INVALID_ARG;
+  {
+    // everything derived from k_max (row strides, tile counts, scratch sizes) has to stay in 32-bit range:
+    // a budget beyond the context selects every row, so nothing larger than T rounded up to chunks is useful
+    const int64_t ch = c->chunk ? c->chunk : 8;
+    const int64_t k_cap = ((int64_t)c->k_max + ch - 1) / ch * ch;
+    if (k_cap + (int64_t)XKV_MAX_OUTLIERS * ch >= ((int64_t)1 << 30)) return XKV_ERR_INVALID_ARG;
+    // landmark rows are addressed by a 32-bit TMA coordinate; problems of a call are a grid dimension
+    const int64_t n_c = ((int64_t)c->T + ch - 1) / ch;
+    if ((int64_t)c->batch * c->G * c->H_kv * n_c >= ((int64_t)1 << 31)) return XKV_ERR_UNSUPPORTED;
+    if ((int64_t)c->batch * c->G * c->H_kv > 65535) return XKV_ERR_UNSUPPORTED;
+  }
   if (!(c->softmax_scale >= 0.0f) || isinf(c->softmax_scale)) return XKV_ERR_INVALID_ARG;
   if (isnan(c->rope_base) || isinf(c->rope_base)) return XKV_ERR_INVALID_ARG;
   if (need_ptrs) {
@@ -107,7 +118,21 @@ const char* xkv_strerror(int s) {
 }
 
 int xkv_last_cuda_error(void) { return g_last_cuda_error; }
-uint64_t xkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+uint64_t xkv_kernel_launch_count(void) {
+  uint64_t n = 0;
+  for (int f = 0; f < kFamCount; ++f) n += g_launches[f].load(std::memory_order_relaxed);
+  return n;
+}
+int xkv_debug_launch_counts(uint64_t* counts) {
+  if (!counts) return XKV_ERR_INVALID_ARG;
+  for (int f = 0; f < kFamCount; ++f) counts[f] = g_launches[f].load(std::memory_order_relaxed);
+  return XKV_OK;
+}
+int xkv_debug_set_fault_injection(xkv_group* g, uint32_t mask) {
+  if (!g || (mask & ~(XKV_INJECT_SCAN_NO_LOAD | XKV_INJECT_FUSED_NO_B))) return XKV_ERR_INVALID_ARG;
+  g->dev.inject = mask;
+  return XKV_OK;
+}
 
 int xkv_group_bytes(const xkv_group_config* cfg, uint64_t* factor_bytes, uint64_t* landmark_bytes) {
   int st = check_config(cfg, false);
@@ -137,6 +162,7 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     XKV_TRY_CUDA(cudaGetDeviceProperties(&prop, g->device));
     if (prop.major != 10) { st = XKV_ERR_ARCH; goto fail; }
     g->sm_count = prop.multiProcessorCount;
+    if (!fused_sm_count_ok(g->sm_count)) { st = XKV_ERR_UNSUPPORTED; goto fail; }   // the segment merge's table size
   }
   {
     GroupDev& d = g->dev;

@@ -221,16 +221,15 @@ cudaError_t launch_t(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* 
   const size_t smem = sizeof(float) * (kSlab * (kTileRows + 4) + kSlab * (DH + 4) + kTileRows * (DH + 1) +
                                        kMaxRep * DH + kMaxRep * kTileRows + 2 * kMaxRep) +
                       sizeof(int) * 2 * kTileRows;
-  cudaError_t e = cudaFuncSetAttribute(recon_attend_tile_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
+  cudaError_t e = ensure_dyn_smem<recon_attend_tile_kernel<DH>>(smem, grp->device);
   if (e != cudaSuccess) return e;
   recon_attend_tile_kernel<DH><<<dim3(tiles, problems), kThreads, smem, s>>>(dev, l0, q, sel_idx, sel_cnt, k_cap,
                                                                             n_tiles);
-  count_launch();
+  count_launch(kFamTile);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   merge_kernel<DH><<<problems * dev.n_rep, DH, 0, s>>>(dev, l0, sel_cnt, k_cap, n_tiles, kTileRows, out, lse);
-  count_launch();
+  count_launch(kFamTile);
   return cudaGetLastError();
 }
 

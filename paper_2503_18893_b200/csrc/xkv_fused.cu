@@ -61,7 +61,7 @@ struct Sched {
 };
 
 struct Bars {        // offsets (in 8-byte words) into the barrier array
-  int full, fullv, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, vfree, grp, total;
+  int full, fullv, emptyk, emptyv, bfull, kfull, kempty, wfull, wempty, pfull, rfree, posfull, vfree, grp, drain, total;
 };
 __host__ __device__ constexpr Bars bar_layout(int na) {
   Bars b{};
@@ -69,7 +69,7 @@ __host__ __device__ constexpr Bars bar_layout(int na) {
   // the kind it waits for is never confused by the other kind's completions
   b.full = 0; b.fullv = na; b.emptyk = 2 * na; b.emptyv = 2 * na + na / 2; b.bfull = 3 * na; b.kfull = b.bfull + kNB;
   b.kempty = b.kfull + 2; b.wfull = b.kempty + 2; b.wempty = b.wfull + 2; b.pfull = b.wempty + 2;
-  b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.vfree = b.posfull + 4; b.grp = b.vfree + 4; b.total = b.grp + 1;
+  b.rfree = b.pfull + 2; b.posfull = b.rfree + 2; b.vfree = b.posfull + 4; b.grp = b.vfree + 4; b.drain = b.grp + 1; b.total = b.drain + 2;
   return b;
 }
 
@@ -101,11 +101,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // small (the warps of a scheduler share its instruction cache).
 __device__ __noinline__ bool wait_bar_slow(volatile int* abort_flag, unsigned int* flags, uint32_t bar, uint32_t parity) {
   const unsigned long long t0 = global_ns();
+  // abort_flag[1] holds the limit in units of 2^16 ns (0: the default)
+  const unsigned long long limit = abort_flag[1] ? ((unsigned long long)abort_flag[1] << 16) : kWaitLimitNs;
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
+      if (global_ns() - t0 > limit) break;
     }
   }
   *abort_flag = 1;
@@ -268,7 +270,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     }
     for (int b = 0; b < 4; ++b) { mbar_init(BAR(bl.posfull + b), 64); mbar_init(BAR(bl.vfree + b), 64); }
     mbar_init(BAR(bl.grp), 128);
-    *abort_flag = 0;
+    mbar_init(BAR(bl.drain), 1); mbar_init(BAR(bl.drain + 1), 1);
+    abort_flag[0] = 0;
+    abort_flag[1] = (dev.inject & XKV_INJECT_FUSED_NO_B) ? 16 : 0;   // injected fault: give up after about a millisecond
     fence_mbar_init();
   }
   if (rope_smem) {
@@ -581,6 +585,13 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
       ++it;
     }
     if (ctx.prof && lane == 0) ctx.prof[ps] = (unsigned long long)(clock64() - role_t0);
+    if (!ok && lane == 0) {
+      // giving up: the tensor-core operations this thread has issued may still be running and the CTA is about to
+      // free its tensor memory; wait (again with a limit) until they have retired
+      const uint32_t db = BAR(bl.drain + (kside ? 0 : 1));
+      tc_commit(db);
+      for (uint32_t i = 0; i < (1u << 22); ++i) if (mbar_try_wait(db, 0)) break;
+    }
     __syncwarp();
   } else if (warp == 13) {
     // =============================== B_k slab loader (TMA) ===============================
@@ -593,6 +604,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
     // tile (the pair after next in the same ring position needs the slab being loaded): then the first slabs of a
     // tile do not have to wait for the end of the previous tile's key phase.
     const bool by_pair = nks_k == nst_k && nks_k >= kNB && kNB <= SK;
+    // fault injection (tests of the give-up path): the slabs are never loaded, so the key-phase warp's wait for
+    // them runs into its limit and the CTA winds down
+    const bool no_b = (dev.inject & XKV_INJECT_FUSED_NO_B) != 0u;
     int bslot = 0, it = 0, slot = 0;
     uint32_t cnt_k = 0;                  // per slot pair: parity of the number of pairs that used it
     uint32_t fifo = 0;                   // per B slot, 4 bits: slot pair (3) and phase parity (1) of the slab it holds
@@ -618,8 +632,10 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
           if (!wait_bar(ctx, BAR(bl.kfull + ((it - 1) & 1)), (uint32_t)(((it - 1) >> 1) & 1), 18)) { ok = false; break; }
         }
         fifo = (fifo & ~(15u << (4 * bslot))) | (my << (4 * bslot));
-        mbar_expect_tx(BAR(bl.bfull + bslot), kSlabBytes);
-        tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, &bk_map, ks * 64, head_row, BAR(bl.bfull + bslot));
+        if (!no_b) {
+          mbar_expect_tx(BAR(bl.bfull + bslot), kSlabBytes);
+          tma_load_2d(bring + (uint32_t)bslot * kSlabBytes, &bk_map, ks * 64, head_row, BAR(bl.bfull + bslot));
+        }
         if (++bslot == kNB) bslot = 0;
       }
       // (a padding slab after an odd number of real slabs sits in the pair that was entered for the last real one)
@@ -989,26 +1005,29 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   memcpy(&mk, grp->bk_tmap, sizeof(mk));
   cudaError_t e;
   if (grp->prof) {     // the variant with the diagnostic counters compiled in
-    e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, true>>(smem, grp->device);
     if (e != cudaSuccess) return e;
     e = launch_pdl(sr_fused_kernel<DH, NR, WB, true>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   } else {
-    e = cudaFuncSetAttribute(sr_fused_kernel<DH, NR, WB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false>>(smem, grp->device);
     if (e != cudaSuccess) return e;
     e = launch_pdl(sr_fused_kernel<DH, NR, WB, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   }
-  count_launch();
+  count_launch(kFamFused);
   if (e != cudaSuccess) return e;
   const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
-  e = cudaFuncSetAttribute(merge_segments_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
+  e = ensure_dyn_smem<merge_segments_kernel<DH>>(msmem, grp->device);
   if (e != cudaSuccess) return e;
   e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, tail, out, lse);
   if (e != cudaSuccess) return e;
-  count_launch();
+  count_launch(kFamMerge);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+// A problem never has more segments than there are CTAs + 1; the merge kernel's tables hold kMergeMaxSeg of them.
+bool fused_sm_count_ok(int sm_count) { return sm_count >= 1 && sm_count + 1 <= kMergeMaxSeg; }
 
 int fused_slots(const xkv_group* grp) {
   const int tpp_max = (grp->k_cap_max + kTile - 1) / kTile;

@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "xkv.h"
 
 namespace xkv {
@@ -38,6 +40,7 @@ struct GroupDev {
   unsigned int* flags;              // device flag word
   const int32_t* outliers;          // [G][batch][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
   int n_out;
+  unsigned int inject;              // XKV_INJECT_* bits (xkv_debug_set_fault_injection); 0 in normal use
 };
 
 }  // namespace xkv
@@ -81,7 +84,28 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
-void count_launch(int n = 1);
+// Kernel families of the launch accounting (xkv_debug_launch_counts reports one counter per family).
+enum KernelFamily {
+  kFamScan = XKV_KERNEL_SCAN, kFamTopk = XKV_KERNEL_TOPK, kFamFused = XKV_KERNEL_FUSED, kFamMerge = XKV_KERNEL_MERGE,
+  kFamTile = XKV_KERNEL_TILE, kFamTailTc = XKV_KERNEL_TAIL_TC, kFamTailCuda = XKV_KERNEL_TAIL_CUDA,
+  kFamLandmarks = XKV_KERNEL_LANDMARKS, kFamPrep = XKV_KERNEL_PREP, kFamDense = XKV_KERNEL_DENSE, kFamCount = XKV_KERNEL_FAMILIES
+};
+void count_launch(KernelFamily family, int n = 1);
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize of one kernel, set once per device instead of on every launch (the
+// attribute is sticky; re-issuing it costs host time on the launch path).  `Kernel` is the kernel's address, so
+// every instantiation keeps its own record.
+constexpr int kMaxDevices = 64;
+template <auto Kernel>
+inline cudaError_t ensure_dyn_smem(size_t bytes, int device) {
+  static std::atomic<size_t> have[kMaxDevices];
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (have[device].load(std::memory_order_acquire) >= bytes && bytes > 0) return cudaSuccess;
+  if (bytes <= 48 * 1024) return cudaSuccess;          // the default limit covers it
+  cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) have[device].store(bytes, std::memory_order_release);
+  return e;
+}
 
 // xkv_prep.cu
 cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch, int G, int r, int H_kv,
@@ -99,6 +123,7 @@ cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, fl
 cudaError_t launch_landmarks(const __nv_bfloat16* keys, __nv_bfloat16* landmarks, float* min_cos, int G, int batch, int T,
                              int H_kv, int d_h, int c, float rope_base, cudaStream_t s);
 
+bool select_stride_ok(int64_t k, int c, int n_out);
 int select_static(const xkv_select_static_config* c, int l0, int l1, const void* q, int32_t k, int32_t* sel_idx,
                   int32_t* sel_cnt, cudaStream_t s);
 // xkv_api.cu: tensor map over [rows][cols] bf16 landmarks, kLandmarkBoxRows-row boxes of 64 columns, 128-byte swizzle
@@ -125,6 +150,7 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
 int fused_slots(const xkv_group* grp);
 size_t fused_part_floats(const xkv_group* grp);
 bool fused_supported(const xkv_group* grp);
+bool fused_sm_count_ok(int sm_count);
 cudaError_t launch_fused(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const int32_t* sel_idx,
                          const int32_t* sel_cnt, int k_cap, __nv_bfloat16* out, float* lse, cudaStream_t s,
                          TailParts tail = TailParts{nullptr, 0});

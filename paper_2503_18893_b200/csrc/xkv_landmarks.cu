@@ -241,7 +241,7 @@ cudaError_t launch_landmarks(const __nv_bfloat16* keys, __nv_bfloat16* landmarks
   else
     landmark_kernel<64><<<grid, kLmThreads, 0, s>>>(keys, landmarks, min_cos, G, batch, T, H_kv, c, n_c, cpc,
                                                     (double)rope_base, use_rope);
-  count_launch();
+  count_launch(kFamLandmarks);
   return cudaGetLastError();
 }
 

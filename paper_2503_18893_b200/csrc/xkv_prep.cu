@@ -30,7 +30,7 @@ cudaError_t launch_repack_b(const __nv_bfloat16* B, __nv_bfloat16* Bt, int batch
                             int d_h, cudaStream_t s) {
   dim3 grid((r + 31) / 32, H_kv * (kDP / 32), batch * G);
   repack_b_kernel<<<grid, dim3(32, 8), 0, s>>>(B, Bt, r, H_kv, d_h);
-  count_launch();
+  count_launch(kFamPrep);
   return cudaGetLastError();
 }
 
@@ -57,7 +57,7 @@ cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift,
   const int half = d_h / 2;
   const long long total = (long long)(n_hi + (1 << rope_shift)) * half;
   rope_tables_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(hi, lo, n_hi, rope_shift, half, base);
-  count_launch();
+  count_launch(kFamPrep);
   return cudaGetLastError();
 }
 

@@ -22,9 +22,9 @@ constexpr uint32_t kWaitLimit = 1u << 22;
 
 using namespace ptx;
 
-// Bounded wait: returns false if the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+// Bounded wait: returns false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;
@@ -92,14 +92,18 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
   const long long prob_lm = ((long long)b * dev.G + l) * dev.H_kv + g;       // landmark order
   const long long prob_out = ((long long)l * dev.batch + b) * dev.H_kv + g;  // [G][batch][H_kv] order
 
+  // fault injection (tests of the give-up path): no load is issued, so the wait below must run into its limit
+  const bool no_load = (dev.inject & XKV_INJECT_SCAN_NO_LOAD) != 0u;
   grid_dependency_wait();          // the queries may come from the kernel launched before this one
   if (threadIdx.x == 0) {          // the thread that initialises the barrier also issues the loads: nothing to wait for
     mbar_init(bar, 1);
     fence_mbar_init();
-    mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
-    const int y = (int)(prob_lm * dev.n_c + j0);
+    if (!no_load) {
+      mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
+      const int y = (int)(prob_lm * dev.n_c + j0);
 #pragma unroll
-    for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar);
+      for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar);
+    }
   }
   grid_dependency_launch();
   // queries of this KV head, widened to fp32 while the landmarks are in flight
@@ -107,8 +111,11 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
   for (int i = threadIdx.x; i < dev.n_rep * DH; i += kScoreThreads) qs[i] = __bfloat162float(qg[i]);
   __syncthreads();
 
-  if (!mbar_wait_bounded(bar, 0)) {
+  if (!mbar_wait_bounded(bar, 0, no_load ? 1024u : kWaitLimit)) {
     if (threadIdx.x == 0) atomicOr(dev.flags, XKV_FLAG_TIMEOUT);
+    // The boxes may still be on their way into this CTA's shared memory, which the next CTA on the SM would
+    // inherit: stay for a second (again bounded) wait before giving the memory up.
+    if (!no_load) (void)mbar_wait_bounded(bar, 0);
     return;
   }
   float best0 = -INFINITY, best1 = -INFINITY;
@@ -460,27 +467,28 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 }  // namespace
 
 // Both kernels of the selection for the problems of layers [l0, l1); `tmap` describes dev.landmarks.
-static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tmap, int l0, int l1,
+// The caller has checked that the row stride (ceil(k/c) + n_out) * c fits 32 bits (select_stride_ok).
+static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tmap, int device, int l0, int l1,
                                      const __nv_bfloat16* q, int k, int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
   const int problems = (l1 - l0) * dev.batch * dev.H_kv;
   const int tiles = (dev.n_c + kScoreRows - 1) / kScoreRows;
   const int c = dev.c;
-  const int k_ch_raw = (k + c - 1) / c;
+  const int k_ch_raw = (int)(((int64_t)k + c - 1) / c);
   const int k_ch = k_ch_raw < dev.n_c ? k_ch_raw : dev.n_c;
   const int k_cap = (k_ch_raw + dev.n_out) * c;      // room for the union with the outlier chunks
   const size_t smem = 1024 + (size_t)(dev.d_h / 64) * kScoreRows * 128 + (size_t)dev.n_rep * dev.d_h * 4;
   dim3 grid(tiles, problems);
   cudaError_t e;
   if (dev.d_h == 128) {
-    e = cudaFuncSetAttribute(score_pool_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dyn_smem<score_pool_kernel<128>>(smem, device);
     if (e != cudaSuccess) return e;
     e = launch_pdl(score_pool_kernel<128>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
   } else {
-    e = cudaFuncSetAttribute(score_pool_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dyn_smem<score_pool_kernel<64>>(smem, device);
     if (e != cudaSuccess) return e;
     e = launch_pdl(score_pool_kernel<64>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
   }
-  count_launch();
+  count_launch(kFamScan);
   if (e != cudaSuccess) return e;
   if (dev.n_c <= kTopkThreads * kTopkItems)
     e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
@@ -488,8 +496,13 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   else
     e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
                    dev.n_out, 1.0f, sel_idx, sel_cnt);
-  count_launch();
+  count_launch(kFamTopk);
   return e;
+}
+
+// (ceil(k/c) + n_out) * c, the row stride of sel_idx, must fit the 32-bit arithmetic of the kernels.
+bool select_stride_ok(int64_t k, int c, int n_out) {
+  return k >= 1 && ((k + c - 1) / c + n_out) * (int64_t)c < ((int64_t)1 << 30);
 }
 
 // The k entries with the largest sign * scores[p][j] of each of `problems` score rows of length n, ids ascending
@@ -506,7 +519,7 @@ cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, fl
   else
     e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, 0, k_ch, k, (const int32_t*)nullptr, 0,
                    sign, out, (int32_t*)nullptr);
-  count_launch();
+  count_launch(kFamTopk);
   return e;
 }
 
@@ -514,7 +527,7 @@ cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloa
                           int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
   CUtensorMap tmap;
   memcpy(&tmap, grp->lm_tmap, sizeof(tmap));
-  return launch_select_dev(grp->dev, tmap, l0, l1, q, k, sel_idx, sel_cnt, s);
+  return launch_select_dev(grp->dev, tmap, grp->device, l0, l1, q, k, sel_idx, sel_cnt, s);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -548,6 +561,9 @@ int select_static(const xkv_select_static_config* c, int l0, int l1, const void*
       ((uintptr_t)sel_idx & 3u) || ((uintptr_t)sel_cnt & 3u))
     return XKV_ERR_INVALID_ARG;
   if (l0 < 0 || l1 > c->G || l0 >= l1 || k < 1) return XKV_ERR_INVALID_ARG;
+  // a budget beyond the context means "every row"; the row stride the caller allocated follows from k, so a k whose
+  // stride leaves 32-bit range is rejected here, before anything is launched
+  if (!select_stride_ok(k, c->chunk ? c->chunk : 8, 0)) return XKV_ERR_INVALID_ARG;
   GroupDev dev{};
   dev.G = c->G; dev.batch = c->batch; dev.T = c->T; dev.H_kv = c->H_kv; dev.H_q = c->H_q; dev.d_h = c->d_h;
   dev.c = c->chunk ? c->chunk : 8;
@@ -557,17 +573,19 @@ int select_static(const xkv_select_static_config* c, int l0, int l1, const void*
   dev.landmarks = (const __nv_bfloat16*)c->landmarks;
   const size_t scores = (size_t)c->G * c->batch * c->H_kv * dev.n_c;   // indexed by absolute layer, like the handle's
   if (scores > (size_t)XKV_STATIC_SELECT_MAX_SCORES) return XKV_ERR_TOO_LARGE;
+  if ((size_t)c->G * c->batch * c->H_kv > 65535) return XKV_ERR_TOO_LARGE;   // problems of a call are a grid dimension
   int device = 0;
   cudaError_t e = cudaGetDevice(&device);
   if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
-  cudaDeviceProp prop;
-  static int cc_major[64] = {};
-  if (device >= 0 && device < 64 && cc_major[device] == 0) {
-    e = cudaGetDeviceProperties(&prop, device);
+  static std::atomic<int> cc_major[kMaxDevices];          // 0: not looked up yet
+  if (device < 0 || device >= kMaxDevices) return XKV_ERR_ARCH;
+  int major = cc_major[device].load(std::memory_order_relaxed);
+  if (major == 0) {
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
     if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
-    cc_major[device] = prop.major;
+    cc_major[device].store(major, std::memory_order_relaxed);
   }
-  if (device < 0 || device >= 64 || cc_major[device] != 10) return XKV_ERR_ARCH;
+  if (major != 10) return XKV_ERR_ARCH;
   float* scratch = static_scratch_ptr(device, &e);
   if (!scratch) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   dev.flags = reinterpret_cast<unsigned int*>(scratch);
@@ -576,7 +594,7 @@ int select_static(const xkv_select_static_config* c, int l0, int l1, const void*
   if (!encode_landmark_map(&tmap, c->landmarks, (uint64_t)c->batch * c->G * c->H_kv * dev.n_c, (uint64_t)c->d_h))
     return XKV_ERR_CUDA;
   e = cudaMemsetAsync(scratch, 0, 64 * sizeof(float), s);              // the flag words start at zero
-  if (e == cudaSuccess) e = launch_select_dev(dev, tmap, l0, l1, (const __nv_bfloat16*)q, k, sel_idx, sel_cnt, s);
+  if (e == cudaSuccess) e = launch_select_dev(dev, tmap, device, l0, l1, (const __nv_bfloat16*)q, k, sel_idx, sel_cnt, s);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }

@@ -310,7 +310,8 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
     }
     tc_commit(bar_s);
   }
-  bool ok = tc_wait_bounded(bar_s, 0);
+  // the outcome of a wait is made CTA-uniform (one thread's poll may run out a moment before another's succeeds)
+  bool ok = __syncthreads_and(tc_wait_bounded(bar_s, 0) ? 1 : 0) != 0;
   tc_fence_after();
   const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
   const bool valid = tid < rows;
@@ -370,7 +371,9 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
     }
     tc_commit(bar_o);
   }
+  const bool ok_s = ok;
   if (ok) ok = tc_wait_bounded(bar_o, 0);
+  ok = __syncthreads_and(ok ? 1 : 0) != 0;
   tc_fence_after();
   float acc[NR];
   if (ok) {
@@ -395,6 +398,11 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
         dst[(size_t)h * (DH + 2) + DH + 1] = ls;
       }
     }
+  }
+  if (!ok && tid == 0) {
+    // giving up: the MMAs issued above may still be running; wait once more (bounded) for the barrier that their
+    // commit arrives on before the tensor memory is freed
+    (void)tc_wait_bounded(ok_s ? bar_o : bar_s, 0);
   }
   tc_fence_before();
   __syncthreads();
@@ -423,16 +431,14 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
   const dim3 grid(problems, n_split), block(kTailThreads);
 #define XKV_TAIL(DH, NR)                                                                                            \
   do {                                                                                                              \
-    e = cudaFuncSetAttribute(tail_partial_kernel<DH, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,              \
-                             (int)tail_smem_bytes<DH, NR>());                                                       \
+    e = ensure_dyn_smem<tail_partial_kernel<DH, NR>>(tail_smem_bytes<DH, NR>(), grp->device);                       \
     if (e == cudaSuccess)                                                                                           \
       e = launch_pdl(tail_partial_kernel<DH, NR>, grid, block, tail_smem_bytes<DH, NR>(), s, dev, l0, q, tail_k,     \
                      tail_v, tail_len, tail_cap, n_split, part);                                                    \
   } while (0)
 #define XKV_TAIL_TC(NR)                                                                                            \
   do {                                                                                                              \
-    e = cudaFuncSetAttribute(tail_tc_kernel<NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,                       \
-                             (int)tail_tc_smem_bytes<NR>());                                                        \
+    e = ensure_dyn_smem<tail_tc_kernel<NR>>(tail_tc_smem_bytes<NR>(), grp->device);                                 \
     if (e == cudaSuccess)                                                                                           \
       e = launch_pdl(tail_tc_kernel<NR>, grid, block, tail_tc_smem_bytes<NR>(), s, dev, l0, q, tail_k, tail_v,       \
                      tail_len, tail_cap, n_split, part);                                                            \
@@ -446,7 +452,7 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
   }
 #undef XKV_TAIL
 #undef XKV_TAIL_TC
-  count_launch();
+  count_launch((dev.d_h == 128 && !grp->tail_impl) ? kFamTailTc : kFamTailCuda);
   return e;
 }
 

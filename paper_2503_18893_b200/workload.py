@@ -1,70 +1,38 @@
-"""Synthetic long-context workloads for tests and the benchmark.
+"""Synthetic long-context workloads for the benchmark and the full-size tests.
 
-Everything here prepares INPUTS of the decode path (it plays the role of the prefill side, which
-is outside the library): factors drawn by `synth.make_factors`, and chunk landmarks computed from
-the keys those factors represent (App. B.1, Algorithm 1 lines 1-3) with plain torch ops on
-whatever device the factors live on.  The decode step itself is only ever run through the
-C ABI (`xkv.py`).
+Everything here prepares INPUTS of the decode path: factors drawn by `synth.make_factors`, and chunk
+landmarks of the keys those factors represent, computed by the library's own prefill entry point
+(`xkv_build_landmarks`, App. B.1, Algorithm 1 lines 1-3).  None of the method's arithmetic is restated in
+Python here; the decode step and the landmarks are only ever run through the C ABI (`xkv.py`).
 """
 from __future__ import annotations
 
 import dataclasses
-import math
 
 import torch
 
 from . import synth
 
 
-def rope_angles(T: int, d_h: int, base: float, device, start: int = 0):
-    """cos/sin of p*theta_i (fp64 angles, returned as fp32), p in [start, start+T), i < d_h/2."""
-    half = d_h // 2
-    theta = torch.pow(torch.tensor(float(base), dtype=torch.float64, device=device),
-                      -torch.arange(half, dtype=torch.float64, device=device) / half)
-    phi = torch.arange(start, start + T, dtype=torch.float64, device=device)[:, None] * theta[None, :]
-    return torch.cos(phi).float(), torch.sin(phi).float()
+def landmarks_from_factors(A_k: torch.Tensor, B_k: torch.Tensor, shape: synth.SRShape) -> torch.Tensor:
+    """Landmarks of the keys the factors stand for, made by the library's own prefill step.
 
-
-def landmarks_from_factors(A_k: torch.Tensor, B_k: torch.Tensor, H_kv: int, c: int, rope_base: float,
-                           rows_per_pass: int = 16384) -> torch.Tensor:
-    """Chunk means of the post-RoPE keys K_l = rope(A_k @ B_k[l]) of every layer and sequence.
-
-    A_k (batch,T,r) bf16, B_k (batch,G,r,d) bf16  ->  bf16 (batch,G,H_kv,n_c,d_h).
-    The mean of a ragged last chunk runs over the rows present.  fp32 arithmetic.
+    The synthetic "original" pre-RoPE keys of layer l are K_l = bf16(A_k @ B_k[l]) (one library matmul per layer:
+    this only manufactures an input); `xkv_build_landmarks` (Algorithm 1) then rotates them and takes the chunk
+    means.  A_k (batch,T,r) bf16, B_k (batch,G,r,d) bf16 on a CUDA device  ->  bf16 (batch,G,H_kv,n_c,d_h).
     """
-    batch, T, r = A_k.shape
-    G, d = B_k.shape[1], B_k.shape[3]
-    d_h = d // H_kv
-    half = d_h // 2
-    n_c = -(-T // c)
-    dev = A_k.device
-    out = torch.empty((batch, G, H_kv, n_c, d_h), dtype=torch.bfloat16, device=dev)
-    step = max(c, (rows_per_pass // c) * c)
-    prev = torch.backends.cuda.matmul.allow_tf32
-    torch.backends.cuda.matmul.allow_tf32 = False
-    try:
-        for b in range(batch):
-            for l in range(G):
-                Bl = B_k[b, l].float()
-                for t0 in range(0, T, step):
-                    t1 = min(T, t0 + step)
-                    K = (A_k[b, t0:t1].float() @ Bl).view(t1 - t0, H_kv, d_h)
-                    if rope_base > 0:
-                        cs, sn = rope_angles(t1 - t0, d_h, rope_base, dev, start=t0)
-                        x1, x2 = K[..., :half], K[..., half:]
-                        K = torch.cat([x1 * cs[:, None, :] - x2 * sn[:, None, :],
-                                       x2 * cs[:, None, :] + x1 * sn[:, None, :]], dim=-1)
-                    n_full = (t1 - t0) // c
-                    j0 = t0 // c
-                    if n_full:
-                        m = K[:n_full * c].view(n_full, c, H_kv, d_h).mean(dim=1)
-                        out[b, l, :, j0:j0 + n_full] = m.permute(1, 0, 2).to(torch.bfloat16)
-                    if n_full * c < t1 - t0:
-                        m = K[n_full * c:].mean(dim=0)
-                        out[b, l, :, j0 + n_full] = m.to(torch.bfloat16)
-    finally:
-        torch.backends.cuda.matmul.allow_tf32 = prev
-    return out
+    from . import xkv
+    if not A_k.is_cuda:
+        raise RuntimeError("workload inputs are prepared with the CUDA library: pass device='cuda'")
+    s = shape
+    lm = torch.empty((s.batch, s.G, s.H_kv, s.n_c, s.d_h), dtype=torch.bfloat16, device=A_k.device)
+    for b in range(s.batch):
+        keys = torch.stack([A_k[b] @ B_k[b, l] for l in range(s.G)]).unsqueeze(0).contiguous()   # (1,G,T,d)
+        xkv.xkv_build_landmarks(keys, lm[b:b + 1], G=s.G, batch=1, T=s.T, H_kv=s.H_kv, d_h=s.d_h, chunk=s.c,
+                                rope_base=s.rope_base)
+        torch.cuda.synchronize()
+        del keys
+    return lm
 
 
 @dataclasses.dataclass
@@ -77,10 +45,10 @@ class GroupInputs:
     q: torch.Tensor          # (n_steps, G, batch, H_q, d_h)
 
 
-def make_group_inputs(shape: synth.SRShape, group: int = 0, n_steps: int = 1, device="cpu") -> GroupInputs:
-    """Factors, landmarks and queries of one window, drawn directly (no factorisation is run)."""
+def make_group_inputs(shape: synth.SRShape, group: int = 0, n_steps: int = 1, device="cuda") -> GroupInputs:
+    """Factors, landmarks and queries of one window on a CUDA device, drawn directly (no factorisation is run)."""
     A_k, A_v, B_k, B_v = synth.make_factors(shape, group, device)
-    lm = landmarks_from_factors(A_k, B_k, shape.H_kv, shape.c, shape.rope_base)
+    lm = landmarks_from_factors(A_k, B_k, shape)
     q = synth.make_queries(shape, n_steps, group, device)
     return GroupInputs(A_k, A_v, B_k, B_v, lm, q)
 

@@ -100,6 +100,14 @@ _lib.xkv_strerror.argtypes = [ctypes.c_int]
 _lib.xkv_strerror.restype = ctypes.c_char_p
 _lib.xkv_last_cuda_error.restype = ctypes.c_int
 _lib.xkv_kernel_launch_count.restype = ctypes.c_uint64
+_lib.xkv_debug_launch_counts.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_debug_launch_counts.restype = ctypes.c_int
+_lib.xkv_debug_set_fault_injection.argtypes = [_P, ctypes.c_uint32]
+_lib.xkv_debug_set_fault_injection.restype = ctypes.c_int
+
+XKV_KERNEL_FAMILIES = ("scan", "topk", "fused", "merge", "tile", "tail_tc", "tail_cuda", "landmarks", "prep", "dense")
+XKV_INJECT_SCAN_NO_LOAD = 1
+XKV_INJECT_FUSED_NO_B = 2
 
 
 class XKVError(RuntimeError):
@@ -118,6 +126,21 @@ def xkv_last_cuda_error() -> int:
 
 def xkv_kernel_launch_count() -> int:
     return int(_lib.xkv_kernel_launch_count())
+
+
+def xkv_debug_launch_counts() -> dict:
+    """Launches since load, by kernel family (names in XKV_KERNEL_FAMILIES)."""
+    a = (ctypes.c_uint64 * len(XKV_KERNEL_FAMILIES))()
+    st = _lib.xkv_debug_launch_counts(a)
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_debug_launch_counts")
+    return {n: int(a[i]) for i, n in enumerate(XKV_KERNEL_FAMILIES)}
+
+
+def xkv_debug_set_fault_injection(grp, mask: int) -> None:
+    st = _lib.xkv_debug_set_fault_injection(grp.handle, mask)
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_debug_set_fault_injection")
 
 
 def _stream(stream) -> int:

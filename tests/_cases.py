@@ -28,8 +28,18 @@ def case_from_clf(shape: synth.SRShape):
     return inp, (K, V)
 
 
-def case_from_factors(shape: synth.SRShape, n_steps=1, device="cpu"):
-    return workload.make_group_inputs(shape, 0, n_steps, device)
+def case_from_factors(shape: synth.SRShape, n_steps=1, group=0):
+    """Factors drawn directly (CPU), landmarks by the oracle's Algorithm 1 from the keys those factors stand for:
+    K_l = bf16(A_k B_k[l]), the synthetic "original" pre-RoPE cache.  CPU tensors (bf16)."""
+    A_k, A_v, B_k, B_v = synth.make_factors(shape, group, "cpu")
+    lm = np.empty((shape.batch, shape.G, shape.H_kv, shape.n_c, shape.d_h), dtype=np.float32)
+    for b in range(shape.batch):
+        for l in range(shape.G):
+            K = O.bf16_round(f32(A_k[b]) @ f32(B_k[b, l]))                       # (T, d)
+            lm[b, l] = O.build_landmarks(K.reshape(shape.T, shape.H_kv, shape.d_h).transpose(1, 0, 2), shape.c,
+                                         shape.rope_base)
+    return workload.GroupInputs(A_k, A_v, B_k, B_v, torch.from_numpy(lm).to(torch.bfloat16),
+                                synth.make_queries(shape, n_steps, group))
 
 
 def oracle_step(shape, inp, step=0, sel_idx=None, sel_cnt=None, problems=None, k=None):

@@ -87,3 +87,28 @@ def test_create_without_gpu_reports_cuda_error_not_a_crash(xkv):
     with pytest.raises(xkv.XKVError) as e:
         xkv.xkv_group_create(cfg, stream=0)
     assert e.value.status in (xkv.XKV_ERR_CUDA, xkv.XKV_ERR_ARCH)
+
+
+def test_budgets_that_overflow_32_bit_strides_are_rejected_on_the_host(xkv):
+    # a caller may pass a huge k to mean "every row": the row stride ceil(k/c)*c must not wrap
+    cfg = xkv.make_config(G=4, batch=1, T=4096, H_kv=8, H_q=32, d_h=128, r_k=64, r_v=64, k_max=2**31 - 1)
+    with pytest.raises(xkv.XKVError) as e:
+        xkv.xkv_group_bytes(cfg)
+    assert e.value.status == xkv.XKV_ERR_INVALID_ARG
+    # the allocation-free entry point checks k before it touches the device (fake, aligned, never dereferenced pointers)
+    sc = xkv.xkv_select_static_config()
+    sc.struct_size = ctypes.sizeof(xkv.xkv_select_static_config)
+    sc.G, sc.batch, sc.T, sc.H_kv, sc.H_q, sc.d_h, sc.chunk = 1, 1, 4096, 2, 8, 64, 8
+    sc.landmarks = 0x10000
+    st = xkv._lib.xkv_sr_select_static(ctypes.byref(sc), 0, 1, 0x20000, 2**31 - 1, 0x30000, 0x40000, None)
+    assert st == xkv.XKV_ERR_INVALID_ARG
+    # sizes whose landmark rows do not fit a 32-bit coordinate are refused, not wrapped
+    big = xkv.make_config(G=64, batch=64, T=(1 << 24) - 1, H_kv=8, H_q=8, d_h=64, r_k=8, r_v=8, k_max=8)
+    with pytest.raises(xkv.XKVError) as e:
+        xkv.xkv_group_bytes(big)
+    assert e.value.status == xkv.XKV_ERR_UNSUPPORTED
+
+
+def test_launch_counters_by_family(xkv):
+    c = xkv.xkv_debug_launch_counts()
+    assert set(c) == set(xkv.XKV_KERNEL_FAMILIES) and sum(c.values()) == xkv.xkv_kernel_launch_count()

@@ -25,25 +25,38 @@ def _fixed_selection(s, n_rows):
     return idx, cnt
 
 
+# (name, shape overrides on top of config 1, tail capacity, per-sequence tail lengths).  d_h = 128 is the head width
+# of every benchmark configuration and the only one the tensor-core tail kernel serves; d_h = 64 always takes the
+# CUDA-core kernel.
+D128 = dict(d_h=128, r_k=64, r_v=64)
 CASES = [
-    ("two_splits_ragged", dict(T=2048, k=256), 700, [700]),
-    ("one_row", dict(T=1024, k=128), 1, [1]),
-    ("per_sequence_lengths", dict(T=1024, k=128, batch=3), 600, [600, 0, 129]),
-    ("d64_heads_16", dict(T=1024, k=128, H_kv=1, H_q=16, d_h=64, r_k=64, r_v=72), 300, [257]),
-    ("qwen_like_rep7", dict(T=1024, k=128, H_kv=2, H_q=14, r_k=96, r_v=160), 1500, [1400]),
-    ("d128_heads_16", dict(T=1024, k=128, H_kv=1, H_q=16, r_k=64, r_v=72), 300, [257]),
-    ("full_tiles_only", dict(T=1024, k=128), 512, [512]),
+    ("d128_two_splits_ragged", dict(T=2048, k=256, **D128), 700, [700]),
+    ("d128_five_splits_ragged", dict(T=1024, k=128, **D128), 640, [515]),
+    ("d128_one_row", dict(T=1024, k=128, **D128), 1, [1]),
+    ("d128_per_sequence_lengths", dict(T=1024, k=128, batch=3, **D128), 600, [600, 0, 129]),
+    ("d128_whole_tiles", dict(T=1024, k=128, **D128), 512, [512]),
+    ("d128_rep7", dict(T=1024, k=128, H_kv=2, H_q=14, d_h=128, r_k=96, r_v=160), 1500, [1400]),
+    ("d128_rep16", dict(T=1024, k=128, H_kv=1, H_q=16, d_h=128, r_k=64, r_v=72), 300, [257]),
+    ("d64_two_splits_ragged", dict(T=2048, k=256), 700, [700]),
+    ("d64_per_sequence_lengths", dict(T=1024, k=128, batch=3), 600, [600, 0, 129]),
+    ("d64_rep16", dict(T=1024, k=128, H_kv=1, H_q=16, d_h=64, r_k=64, r_v=72), 300, [257]),
+    ("d64_rep7", dict(T=1024, k=128, H_kv=2, H_q=14, r_k=96, r_v=160), 1500, [1400]),
 ]
 
 
 @pytest.mark.parametrize("impl", ["tensor", "cuda"])
 @pytest.mark.parametrize("name,over,cap,lens", CASES, ids=[c[0] for c in CASES])
 def test_tail_parity(name, over, cap, lens, impl, monkeypatch):
+    from paper_2503_18893_b200 import xkv
+    s = synth.config(1, **over)
+    assert s.d_h == (128 if name.startswith("d128") else 64)
     # d_h = 128 runs the tensor-core tail kernel unless the handle is created with XKV_TAIL_IMPL=c
     if impl == "cuda":
-        if over.get("d_h", 128) != 128:
-            pytest.skip("d_h = 64 always takes the CUDA-core kernel")
+        if s.d_h != 128:
+            pytest.skip("d_h = 64 always takes the CUDA-core kernel: covered by the other parametrisation")
         monkeypatch.setenv("XKV_TAIL_IMPL", "c")
+    expect_family = "tail_tc" if (impl == "tensor" and s.d_h == 128) else "tail_cuda"
+    before = xkv.xkv_debug_launch_counts()
     s = synth.config(1, **over)
     inp = C.case_from_factors(s)
     rms = _key_rms(s, inp)
@@ -52,6 +65,9 @@ def test_tail_parity(name, over, cap, lens, impl, monkeypatch):
     cnt[0, 0, 0] = 0                                   # one problem attends to the tail only
     g = C.GpuCase(s, inp)
     gout, glse = g.attend_tail(idx, cnt, tk, tv, lens)
+    after = xkv.xkv_debug_launch_counts()
+    ran = {f for f in ("tail_tc", "tail_cuda") if after[f] > before[f]}
+    assert ran == {expect_family}, (name, impl, ran)     # the kernel under test is the one that ran
     oout, olse = C.oracle_step_with_tail(s, inp, idx, cnt, tk, tv, lens)
     assert g.status() == (0, 0)
     # empty problems (no selected rows and no tail rows) give 0 and -inf on both sides

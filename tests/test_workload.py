@@ -1,5 +1,5 @@
-"""Input preparation (no GPU): the generator is deterministic and the torch landmark builder used for
-large workloads agrees with the oracle's Algorithm 1."""
+"""Input preparation (no GPU): the generator is deterministic, the recipes have the structure they claim, and
+the test cases take their landmarks from the oracle's Algorithm 1."""
 import numpy as np
 import torch
 
@@ -44,15 +44,15 @@ def test_direct_factors_are_in_factorised_form():
     assert not torch.equal(idx[0, 0, 0], idx[0, 0, 0].sort().values)       # left unsorted
 
 
-def test_torch_landmark_builder_matches_oracle_algorithm_1():
+def test_test_cases_take_landmarks_from_the_oracle():
+    from tests import _cases as C
     s = synth.config(1, T=203, r_k=16, r_v=16)                             # ragged last chunk (203 = 25*8 + 3)
-    A_k, A_v, B_k, B_v = synth.make_factors(s)
-    lm = workload.landmarks_from_factors(A_k, B_k, s.H_kv, s.c, s.rope_base, rows_per_pass=64)
-    assert lm.shape == (1, s.G, s.H_kv, 26, s.d_h)
-    for l in range(s.G):
-        K = (A_k[0].double() @ B_k[0, l].double()).numpy().reshape(s.T, s.H_kv, s.d_h).transpose(1, 0, 2)
-        ref = O.build_landmarks(K, s.c, s.rope_base)
-        np.testing.assert_allclose(lm[0, l].float().numpy(), ref, rtol=2e-2, atol=2e-3)
+    inp = C.case_from_factors(s)
+    assert inp.landmarks.shape == (1, s.G, s.H_kv, 26, s.d_h) and inp.landmarks.dtype == torch.bfloat16
+    # the last landmark is the mean of the three rows present, of the rotated bf16 keys A_k B_k
+    K = O.bf16_round(C.f32(inp.A_k[0]) @ C.f32(inp.B_k[0, 1]))[:, s.d_h:2 * s.d_h]
+    tail = O.rope_rotate(K[200:203], np.arange(200, 203), s.rope_base).mean(axis=0)
+    np.testing.assert_allclose(C.f32(inp.landmarks[0, 1, 1, 25]), tail, rtol=1e-2, atol=1e-3)
 
 
 def test_byte_and_flop_model():
