@@ -348,7 +348,7 @@ int xkv_build_landmarks(const xkv_landmark_config* c, const void* keys, void* la
   e = launch_landmarks((const __nv_bfloat16*)keys, (__nv_bfloat16*)landmarks, min_cos, c->G, c->batch, c->T, c->H_kv,
                        c->d_h, ch, c->rope_base, s);
   if (e == cudaSuccess && n_outliers > 0)
-    e = launch_topk_rows(min_cos, c->G * c->batch * c->H_kv, n_c, n_outliers, -1.0f, outliers, s);
+    e = launch_topk_rows(min_cos, c->G * c->batch * c->H_kv, n_c, n_outliers, -1.0f, outliers, device, s);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }

@@ -117,7 +117,8 @@ cudaError_t launch_rope_tables(float2* hi, float2* lo, int n_hi, int rope_shift,
 cudaError_t launch_select(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, int k,
                           int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
 
-cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, cudaStream_t s);
+cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, int device,
+                             cudaStream_t s);
 
 // xkv_landmarks.cu
 cudaError_t launch_landmarks(const __nv_bfloat16* keys, __nv_bfloat16* landmarks, float* min_cos, int G, int batch, int T,

@@ -35,6 +35,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
+// Order-preserving map float -> uint32 (larger float = larger key), with -0 folded onto +0.
+__device__ __forceinline__ uint32_t score_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  if (u == 0x80000000u) u = 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 // One pass over the staged tile for HB query heads; returns per-row max of the scaled scores.
 template <int DH, int HB>
 __device__ __forceinline__ void score_pass(uint32_t tile, const float* __restrict__ qs, int row0, float s,
@@ -128,9 +135,10 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
     else if (hb == 2) score_pass<DH, 2>(tile, qh, row0, dev.sel_scale, best0, best1);
     else score_pass<DH, 1>(tile, qh, row0, dev.sel_scale, best0, best1);
   }
-  float* dst = dev.pooled + prob_out * dev.n_c;
-  if (j0 + row0 < dev.n_c) dst[j0 + row0] = best0;
-  if (j0 + row0 + kScoreThreads < dev.n_c) dst[j0 + row0 + kScoreThreads] = best1;
+  // the pooled scores are handed on as order-preserving integer keys (what the top-k compares)
+  uint32_t* dst = reinterpret_cast<uint32_t*>(dev.pooled) + prob_out * dev.n_c;
+  if (j0 + row0 < dev.n_c) dst[j0 + row0] = score_key(best0);
+  if (j0 + row0 + kScoreThreads < dev.n_c) dst[j0 + row0 + kScoreThreads] = score_key(best1);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -140,26 +148,26 @@ constexpr int kTopkItems = 16;    // consecutive chunks per thread and super-blo
 constexpr int kTopkBins = 2048;   // histogram bins per radix pass
 constexpr int kTopkCand = 256;    // at most this many keys are ranked against one another directly
 
-// Order-preserving map float -> uint32 (larger float = larger key), with -0 folded onto +0.
-__device__ __forceinline__ uint32_t score_key(float f) {
-  uint32_t u = __float_as_uint(f);
-  if (u == 0x80000000u) u = 0u;
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 // Keys of this thread's 16 consecutive chunks of one super-block (0 beyond n_c; callers mask by index).
+// sign == 0: the array already holds keys (the landmark scan writes them); else it holds floats and the key is
+// that of sign * value.
 __device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, float sign, uint32_t (&key)[kTopkItems]) {
+  const bool keyed = sign == 0.0f;
   if (j0 + kTopkItems <= n_c && ((n_c & 3) == 0)) {
     const float4* p = reinterpret_cast<const float4*>(S + j0);
 #pragma unroll
     for (int i = 0; i < kTopkItems / 4; ++i) {
       const float4 v = p[i];
-      key[4 * i] = score_key(v.x * sign); key[4 * i + 1] = score_key(v.y * sign);
-      key[4 * i + 2] = score_key(v.z * sign); key[4 * i + 3] = score_key(v.w * sign);
+      const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) key[4 * i + e] = keyed ? __float_as_uint(f[e]) : score_key(f[e] * sign);
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < kTopkItems; ++i) key[i] = (j0 + i < n_c) ? score_key(S[j0 + i] * sign) : 0u;
+    for (int i = 0; i < kTopkItems; ++i) {
+      const float f = (j0 + i < n_c) ? S[j0 + i] : 0.0f;
+      key[i] = (j0 + i < n_c) ? (keyed ? __float_as_uint(f) : score_key(f * sign)) : 0u;
+    }
   }
 }
 
@@ -171,7 +179,7 @@ template <bool CACHED>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out, float sign,
             int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
-  __shared__ uint32_t hist[kTopkBins];
+  __shared__ __align__(16) uint32_t hist[kTopkBins];
   __shared__ uint32_t warp_tot[kTopkThreads / 32];
   __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
   __shared__ uint32_t sh_a, sh_b, sh_c;
@@ -294,9 +302,28 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
           } else {
             load_keys(S, j0, n_c, sign, key);
           }
+          // this thread's candidates as a bit mask; the warp reserves room for all of its candidates with one atomic
+          uint32_t cm = 0;
 #pragma unroll
           for (int i = 0; i < kTopkItems; ++i) {
-            if (j0 + i < n_c && key[i] >= lo && key[i] - lo <= span) cand[atomicAdd(&sh_a, 1u)] = key[i];
+            if (j0 + i < n_c && key[i] >= lo && key[i] - lo <= span) cm |= 1u << i;
+          }
+          const uint32_t mine_c = (uint32_t)__popc(cm);
+          if (__any_sync(0xffffffffu, cm != 0u)) {
+            uint32_t inc = mine_c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+              if (lane >= o) inc += v;
+            }
+            uint32_t wbase = 0;
+            if (lane == 31) wbase = atomicAdd(&sh_a, inc);
+            wbase = __shfl_sync(0xffffffffu, wbase, 31);
+            uint32_t at = wbase + inc - mine_c;
+#pragma unroll
+            for (int i = 0; i < kTopkItems; ++i) {
+              if ((cm >> i) & 1u) cand[at++] = key[i];
+            }
           }
         }
         __syncthreads();
@@ -305,7 +332,15 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
         if ((uint32_t)tid < n_cand) {
           const uint32_t mykey = cand[tid];
           uint32_t gt = 0, eq = 0;
-          for (uint32_t i = 0; i < n_cand; ++i) {
+          const uint32_t n4 = n_cand & ~3u;
+          const uint4* c4 = reinterpret_cast<const uint4*>(cand);
+#pragma unroll 4
+          for (uint32_t i = 0; i < n4; i += 4) {
+            const uint4 v = c4[i >> 2];
+            gt += (v.x > mykey ? 1u : 0u) + (v.y > mykey ? 1u : 0u) + (v.z > mykey ? 1u : 0u) + (v.w > mykey ? 1u : 0u);
+            eq += (v.x == mykey ? 1u : 0u) + (v.y == mykey ? 1u : 0u) + (v.z == mykey ? 1u : 0u) + (v.w == mykey ? 1u : 0u);
+          }
+          for (uint32_t i = n4; i < n_cand; ++i) {
             const uint32_t c2 = cand[i];
             gt += c2 > mykey ? 1u : 0u;
             eq += c2 == mykey ? 1u : 0u;
@@ -397,7 +432,15 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
     uint32_t gt_before = run_gt + (excl & 0xffffu);
     uint32_t eq_before = run_eq + (excl >> 16);
     if (n_out == 0) {
-      // only a few percent of the chunks are taken: walk the set bits instead of all items
+      // Only a few percent of the chunks are taken.  Output position of a taken chunk = taken chunks before it.
+      // If the super-block's taken chunks fit the list (the histogram's memory, free by now), their ids go there
+      // first and the whole CTA then writes the rows, consecutive threads to consecutive words; else every thread
+      // writes the rows of its own chunks.
+      const uint32_t blk_gt = tot1 & 0xffffu, blk_eq = tot1 >> 16;
+      const uint32_t eq_room = need_eq > run_eq ? need_eq - run_eq : 0u;        // equal keys this super-block may still take
+      const uint32_t blk_taken = blk_gt + min(blk_eq, eq_room);
+      const uint32_t pos0 = run_gt + min(run_eq, need_eq);                       // chunks written by earlier super-blocks
+      const bool listed = blk_taken <= (uint32_t)kTopkBins;
       uint32_t m = gtm | eqm;
       while (m) {
         const int i = __ffs(m) - 1;
@@ -405,7 +448,25 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
         const uint32_t below = (1u << i) - 1u;
         const uint32_t g_b = gt_before + (uint32_t)__popc(gtm & below), e_b = eq_before + (uint32_t)__popc(eqm & below);
         const bool is_gt = (gtm >> i) & 1u;
-        if (is_gt || e_b < need_eq) write_chunk(g_b + min(e_b, need_eq), j0 + i);
+        if (is_gt || e_b < need_eq) {
+          const uint32_t pos = g_b + min(e_b, need_eq);
+          if (listed) hist[pos - pos0] = (uint32_t)(j0 + i); else write_chunk(pos, j0 + i);
+        }
+      }
+      if (listed) {
+        __syncthreads();
+        if (c == 8) {
+          for (uint32_t w = (uint32_t)tid; w < blk_taken * 8u; w += kTopkThreads) {
+            const int row = (int)hist[w >> 3] * 8 + (int)(w & 7u);
+            if (row < T) out[(size_t)pos0 * 8 + w] = row;
+          }
+        } else {
+          for (uint32_t w = (uint32_t)tid; w < blk_taken * (uint32_t)c; w += kTopkThreads) {
+            const uint32_t e = w / (uint32_t)c, t = w - e * (uint32_t)c;
+            const int row = (int)hist[e] * c + (int)t;
+            if (row < T) out[(size_t)pos0 * c + w] = row;
+          }
+        }
       }
     } else {
       // membership in the top-k first, then the union with the outlier chunks, then positions over the union
@@ -464,7 +525,327 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
   if (tid == 0 && sel_cnt) sel_cnt[prob] = cnt;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The same selection for n_c <= 16384 chunks (one super-block), organised so that almost all of the work is done
+// on a short list instead of on every key.  Each thread holds 16 consecutive keys, split into GPT groups; the
+// k_ch-th largest of the group maxima is a lower bound P of the k_ch-th largest key (at least k_ch keys -- those
+// maxima -- are >= it), and with k_ch a few percent of n_c only a few percent of the keys pass it.  The keys >= P
+// go to a list in shared memory (key, chunk index); the exact k_ch-th largest key is then found on the list by
+// the radix select of topk_kernel; membership goes to a bitmap over the chunks (united with the head's outlier
+// chunks), whose prefix popcounts give the ascending output positions.  GPT = 16 disables the filter (P = the
+// smallest key): chosen by the host when there are fewer groups than k_ch.  The result is identical to
+// topk_kernel's for every input; only the amount of work differs.
+constexpr int kPivotListMax = kTopkThreads * kTopkItems;    // every key may pass (all keys equal)
+
+// Bin (counted from the top) that holds the `need`-th largest of the keys counted in hist[0..kTopkBins), by a
+// suffix sum over the bins; thread t owns bins 2t, 2t+1.  Results in sh[0] = bin, sh[1] = rank wanted inside the
+// bin, sh[2] = keys in the bin.  Contains barriers: call it from all threads.
+__device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, uint32_t* warp_tot, uint32_t* sh, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  const uint32_t h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+  const uint32_t mine = h0 + h1;
+  uint32_t suf = mine;                                     // inclusive over higher lanes of the warp
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_down_sync(0xffffffffu, suf, o);
+    if (lane + o < 32) suf += v;
+  }
+  if (lane == 0) warp_tot[warp] = suf;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t t = warp_tot[lane];
+    uint32_t ws = t;                                       // inclusive over higher warps
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_down_sync(0xffffffffu, ws, o);
+      if (lane + o < 32) ws += v;
+    }
+    warp_tot[lane] = ws - t;                               // keys in bins of higher warps
+  }
+  __syncthreads();
+  const uint32_t above = warp_tot[warp] + (suf - mine);    // keys in bins above 2t+1
+  if (above < need && above + mine >= need) {              // exactly one thread
+    if (above + h1 >= need) { sh[0] = 2 * tid + 1; sh[1] = need - above; sh[2] = h1; }
+    else { sh[0] = 2 * tid; sh[1] = need - above - h1; sh[2] = h0; }
+  }
+  __syncthreads();
+}
+
+template <int GPT>
+__global__ void __launch_bounds__(kTopkThreads, 1)
+topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out, float sign,
+                  int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
+  extern __shared__ __align__(16) uint8_t pivot_smem[];
+  uint32_t* list_key = reinterpret_cast<uint32_t*>(pivot_smem);                    // [kPivotListMax]; later the chunk list
+  uint16_t* list_idx = reinterpret_cast<uint16_t*>(list_key + kPivotListMax);      // [kPivotListMax]
+  __shared__ __align__(16) uint32_t hist[kTopkBins];
+  __shared__ uint32_t take_w[kPivotListMax / 32], eq_w[kPivotListMax / 32];        // bitmaps over the chunks
+  __shared__ uint32_t warp_tot[kTopkThreads / 32];
+  __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
+  __shared__ uint32_t sh[4];
+  __shared__ uint32_t sh_n;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_layer = dev.batch * dev.H_kv;
+  const long long prob = (long long)l0 * per_layer + blockIdx.x;     // [G][batch][H_kv] order
+  const float* __restrict__ S = dev.pooled + prob * dev.n_c;
+  int32_t* __restrict__ out = sel_idx + prob * k_cap;
+  const int n_c = dev.n_c, c = dev.c, T = dev.T;
+  constexpr int NW = kPivotListMax / 32;                               // words of a bitmap (512)
+  constexpr int NG = GPT == 16 ? 1 : GPT;                              // group maxima kept per thread
+  constexpr int GS = kTopkItems / NG;                                  // keys per group
+
+  grid_dependency_wait();                      // the pooled scores come from the kernel launched before
+  grid_dependency_launch();
+  const int j0 = tid * kTopkItems;
+  const bool all = (k_ch >= n_c);
+  uint32_t thr = 0, need_eq = 0;
+  for (int w = tid; w < NW; w += kTopkThreads) { take_w[w] = 0u; eq_w[w] = 0u; }
+  if (tid == 0) sh_n = 0;
+  if (!all) {
+    uint32_t key[kTopkItems];
+    load_keys(S, j0, n_c, sign, key);
+    // ---- extrema of this thread's keys and of its groups
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    uint32_t gmax[NG];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) gmax[g] = 0u;
+#pragma unroll
+    for (int i = 0; i < kTopkItems; ++i) {
+      if (j0 + i < n_c) {
+        kmin = min(kmin, key[i]); kmax = max(kmax, key[i]);
+        if (GPT != 16) gmax[i / GS] = max(gmax[i / GS], key[i]);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    if (lane == 0) { warp_min[warp] = kmin; warp_max[warp] = kmax; }
+    for (int i = tid; i < kTopkBins; i += kTopkThreads) hist[i] = 0;
+    __syncthreads();
+    kmin = warp_min[lane]; kmax = warp_max[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    // ---- pivot: lower edge of the bin that holds the k_ch-th largest group maximum
+    uint32_t P = kmin;
+    if (GPT != 16) {
+      const uint32_t span1 = kmax - kmin;
+      const int bits1 = 32 - __clz(span1);
+      const int sh1 = bits1 > 11 ? bits1 - 11 : 0;
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        if (j0 + g * GS < n_c) atomicAdd(&hist[(gmax[g] - kmin) >> sh1], 1u);    // the group has at least one key
+      }
+      __syncthreads();
+      find_bin(hist, (uint32_t)k_ch, warp_tot, sh, tid);
+      P = kmin + (sh[0] << sh1);
+      __syncthreads();
+    }
+    // ---- the keys >= P, with their chunk index, to the list (one shared-memory atomic per warp)
+    {
+      uint32_t cm = 0;
+#pragma unroll
+      for (int i = 0; i < kTopkItems; ++i) {
+        if (j0 + i < n_c && key[i] >= P) cm |= 1u << i;
+      }
+      const uint32_t mine_c = (uint32_t)__popc(cm);
+      if (__any_sync(0xffffffffu, cm != 0u)) {
+        uint32_t inc = mine_c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += v;
+        }
+        uint32_t wbase = 0;
+        if (lane == 31) wbase = atomicAdd(&sh_n, inc);
+        wbase = __shfl_sync(0xffffffffu, wbase, 31);
+        uint32_t at = wbase + inc - mine_c;
+#pragma unroll
+        for (int i = 0; i < kTopkItems; ++i) {
+          if ((cm >> i) & 1u) { list_key[at] = key[i]; list_idx[at] = (uint16_t)(j0 + i); ++at; }
+        }
+      }
+    }
+    __syncthreads();
+    const int n_list = (int)sh_n;                                      // >= k_ch
+    // ---- radix select of the k_ch-th largest key on the list: bins subdivide the window [lo, lo + span]
+    uint32_t lo = P, span = kmax - P, need = (uint32_t)k_ch;
+    for (;;) {
+      const int bits = 32 - __clz(span);                               // span < 2^bits
+      const int shb = bits > 11 ? bits - 11 : 0;
+      for (int i = tid; i < kTopkBins; i += kTopkThreads) hist[i] = 0;
+      __syncthreads();
+      for (int e = tid; e < n_list; e += kTopkThreads) {
+        const uint32_t rel = list_key[e] - lo;                         // keys below lo wrap to huge values
+        if (rel <= span) atomicAdd(&hist[rel >> shb], 1u);
+      }
+      __syncthreads();
+      find_bin(hist, need, warp_tot, sh, tid);
+      const uint32_t bsel = sh[0], in_bin = sh[2];
+      need = sh[1];
+      lo += bsel << shb;
+      span = min(span - (bsel << shb), (shb ? (1u << shb) : 1u) - 1u);
+      __syncthreads();
+      if (shb == 0) { thr = lo; need_eq = need; break; }
+      if (in_bin <= (uint32_t)kTopkCand) {
+        // few keys are left in the window: collect them and rank them against one another
+        uint32_t* cand = hist;
+        if (tid == 0) sh[3] = 0;
+        __syncthreads();
+        for (int e = tid; e < n_list; e += kTopkThreads) {
+          const uint32_t kk = list_key[e];
+          if (kk - lo <= span) cand[atomicAdd(&sh[3], 1u)] = kk;
+        }
+        __syncthreads();
+        const uint32_t n_cand = sh[3];                                 // == in_bin
+        __syncthreads();
+        if ((uint32_t)tid < n_cand) {
+          const uint32_t mykey = cand[tid];
+          uint32_t gt = 0, eq = 0;
+          const uint32_t n4 = n_cand & ~3u;
+          const uint4* c4 = reinterpret_cast<const uint4*>(cand);
+#pragma unroll 4
+          for (uint32_t i = 0; i < n4; i += 4) {
+            const uint4 v = c4[i >> 2];
+            gt += (v.x > mykey ? 1u : 0u) + (v.y > mykey ? 1u : 0u) + (v.z > mykey ? 1u : 0u) + (v.w > mykey ? 1u : 0u);
+            eq += (v.x == mykey ? 1u : 0u) + (v.y == mykey ? 1u : 0u) + (v.z == mykey ? 1u : 0u) + (v.w == mykey ? 1u : 0u);
+          }
+          for (uint32_t i = n4; i < n_cand; ++i) {
+            const uint32_t c2 = cand[i];
+            gt += c2 > mykey ? 1u : 0u;
+            eq += c2 == mykey ? 1u : 0u;
+          }
+          if (gt < need && need <= gt + eq) { sh[0] = mykey; sh[1] = need - gt; }   // equal keys write the same pair
+        }
+        __syncthreads();
+        thr = sh[0];
+        need_eq = sh[1];
+        __syncthreads();
+        break;
+      }
+    }
+    // ---- membership: keys above the threshold, and (separately) keys equal to it
+    for (int e = tid; e < n_list; e += kTopkThreads) {
+      const uint32_t kk = list_key[e];
+      const uint32_t j = list_idx[e];
+      if (kk > thr) atomicOr(&take_w[j >> 5], 1u << (j & 31u));
+      else if (kk == thr) atomicOr(&eq_w[j >> 5], 1u << (j & 31u));
+    }
+  } else {
+    __syncthreads();                                                   // the bitmaps are zeroed
+    for (int w = tid; w < NW; w += kTopkThreads) {
+      const int first = w * 32;
+      take_w[w] = first + 32 <= n_c ? 0xffffffffu : (first < n_c ? ((1u << (n_c - first)) - 1u) : 0u);
+    }
+  }
+  // Algorithm 2 line 5: the head's static outlier chunks join the set
+  if (n_out > 0) {
+    __syncthreads();
+    const int32_t* outl = outliers + (size_t)prob * (size_t)n_out;     // [G][batch][H_kv][n_out], like sel_idx
+    for (int o = tid; o < n_out; o += kTopkThreads) {
+      const int jo = outl[o];
+      if (jo >= 0 && jo < n_c) atomicOr(&take_w[jo >> 5], 1u << (jo & 31));
+    }
+  }
+  __syncthreads();
+  // ---- exclusive prefix over the CTA in thread order; the total goes to sh[3]
+  auto block_scan = [&](uint32_t mine) -> uint32_t {
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t t = warp_tot[lane];
+      uint32_t ti = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, ti, o);
+        if (lane >= o) ti += v;
+      }
+      warp_tot[lane] = ti - t;
+      if (lane == 31) sh[3] = ti;
+    }
+    __syncthreads();
+    return inc - mine + warp_tot[warp];
+  };
+  // keys equal to the threshold: the need_eq with the lowest chunk index are taken (thread w owns word w)
+  static_assert(NW <= kTopkThreads, "one bitmap word per thread");
+  uint32_t fw = tid < NW ? take_w[tid] : 0u;
+  {
+    const uint32_t ew = tid < NW ? eq_w[tid] : 0u;
+    const uint32_t eq_before = block_scan((uint32_t)__popc(ew));
+    uint32_t room = need_eq > eq_before ? need_eq - eq_before : 0u;
+    uint32_t rest = ew;
+    while (rest && room) { fw |= rest & (0u - rest); rest &= rest - 1u; --room; }   // lowest set bits first
+    __syncthreads();                                                   // sh[3] and warp_tot are reused below
+  }
+  // ---- positions over the union, chunk ids to the chunk list (ascending), rows written by the whole CTA
+  const uint32_t before = block_scan((uint32_t)__popc(fw));
+  const uint32_t taken = sh[3];
+  {
+    uint32_t pos = before, rest = fw;
+    while (rest) {
+      list_key[pos++] = (uint32_t)(tid * 32 + __ffs(rest) - 1);
+      rest &= rest - 1u;
+    }
+  }
+  __syncthreads();
+  if (c == 8) {
+    for (uint32_t w = (uint32_t)tid; w < taken * 8u; w += kTopkThreads) {
+      const int row = (int)list_key[w >> 3] * 8 + (int)(w & 7u);
+      if (row < T) out[w] = row;
+    }
+  } else {
+    for (uint32_t w = (uint32_t)tid; w < taken * (uint32_t)c; w += kTopkThreads) {
+      const uint32_t e = w / (uint32_t)c, t = w - e * (uint32_t)c;
+      const int row = (int)list_key[e] * c + (int)t;
+      if (row < T) out[w] = row;
+    }
+  }
+  // whole chunks unless the ragged last chunk was taken (it is then the last one)
+  int cnt = (int)taken * c;
+  if (taken > 0 && list_key[taken - 1] == (uint32_t)(n_c - 1)) cnt -= (n_c * c - T);
+  for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
+  if (tid == 0 && sel_cnt) sel_cnt[prob] = cnt;
+}
+
 }  // namespace
+
+// Top-k of `problems` rows of dev.pooled (sign == 0: keys; else floats compared as sign * value).
+static cudaError_t launch_topk(const GroupDev& dev, int device, int problems, int l0, int k_ch, int k_cap,
+                               const int32_t* outliers, int n_out, float sign, int32_t* sel_idx, int32_t* sel_cnt,
+                               cudaStream_t s) {
+  if (dev.n_c > kTopkThreads * kTopkItems)
+    return launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, outliers, n_out,
+                      sign, sel_idx, sel_cnt);
+  // groups per thread: the fewest with at least k_ch groups in all (16 = no filter)
+  const size_t smem = (size_t)kPivotListMax * (sizeof(uint32_t) + sizeof(uint16_t));
+  cudaError_t e;
+#define XKV_PIVOT(GPT)                                                                                         \
+  do {                                                                                                         \
+    e = ensure_dyn_smem<topk_pivot_kernel<GPT>>(smem, device);                                                 \
+    if (e == cudaSuccess)                                                                                      \
+      e = launch_pdl(topk_pivot_kernel<GPT>, dim3(problems), dim3(kTopkThreads), smem, s, dev, l0, k_ch, k_cap, \
+                     outliers, n_out, sign, sel_idx, sel_cnt);                                                 \
+  } while (0)
+  auto groups = [&](int gpt) { return (dev.n_c + kTopkItems / gpt - 1) / (kTopkItems / gpt); };
+  if (groups(1) >= k_ch) XKV_PIVOT(1);
+  else if (groups(2) >= k_ch) XKV_PIVOT(2);
+  else if (groups(4) >= k_ch) XKV_PIVOT(4);
+  else XKV_PIVOT(16);
+#undef XKV_PIVOT
+  return e;
+}
 
 // Both kernels of the selection for the problems of layers [l0, l1); `tmap` describes dev.landmarks.
 // The caller has checked that the row stride (ceil(k/c) + n_out) * c fits 32 bits (select_stride_ok).
@@ -490,12 +871,7 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   }
   count_launch(kFamScan);
   if (e != cudaSuccess) return e;
-  if (dev.n_c <= kTopkThreads * kTopkItems)
-    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
-                   dev.n_out, 1.0f, sel_idx, sel_cnt);
-  else
-    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, dev.outliers,
-                   dev.n_out, 1.0f, sel_idx, sel_cnt);
+  e = launch_topk(dev, device, problems, l0, k_ch, k_cap, dev.outliers, dev.n_out, 0.0f, sel_idx, sel_cnt, s);
   count_launch(kFamTopk);
   return e;
 }
@@ -507,18 +883,13 @@ bool select_stride_ok(int64_t k, int c, int n_out) {
 
 // The k entries with the largest sign * scores[p][j] of each of `problems` score rows of length n, ids ascending
 // (ties to the lowest id), padded with -1: out [problems][k].  Used for the static outlier chunks (Algorithm 1 line 5).
-cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, cudaStream_t s) {
+cudaError_t launch_topk_rows(const float* scores, int problems, int n, int k, float sign, int32_t* out, int device,
+                             cudaStream_t s) {
   GroupDev dev{};
   dev.G = 1; dev.batch = problems; dev.H_kv = 1; dev.T = n; dev.c = 1; dev.n_c = n;
   dev.pooled = const_cast<float*>(scores);
   const int k_ch = k < n ? k : n;
-  cudaError_t e;
-  if (n <= kTopkThreads * kTopkItems)
-    e = launch_pdl(topk_kernel<true>, dim3(problems), dim3(kTopkThreads), 0, s, dev, 0, k_ch, k, (const int32_t*)nullptr, 0,
-                   sign, out, (int32_t*)nullptr);
-  else
-    e = launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, 0, k_ch, k, (const int32_t*)nullptr, 0,
-                   sign, out, (int32_t*)nullptr);
+  cudaError_t e = launch_topk(dev, device, problems, 0, k_ch, k, nullptr, 0, sign, out, nullptr, s);
   count_launch(kFamTopk);
   return e;
 }
