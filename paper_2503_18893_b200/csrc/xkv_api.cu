@@ -177,6 +177,7 @@ int xkv_group_create(const xkv_group_config* cfg, void* stream, xkv_group** out)
     d.sel_scale = 1.0f / sqrtf((float)c.d_h);
     d.att_scale = c.softmax_scale > 0.0f ? c.softmax_scale : 1.0f / sqrtf((float)c.d_h);
     d.use_rope = c.rope_base > 0.0f;
+    d.lm_const = 1;
     d.A_k = (const __nv_bfloat16*)c.A_k; d.A_v = (const __nv_bfloat16*)c.A_v;
     d.landmarks = (const __nv_bfloat16*)c.landmarks;
     g->k_cap_max = (int)(((int64_t)c.k_max + c.chunk - 1) / c.chunk) * c.chunk;

@@ -40,6 +40,7 @@ struct GroupDev {
   unsigned int* flags;              // device flag word
   const int32_t* outliers;          // [G][batch][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
   int n_out;
+  int lm_const;                     // 1: the landmarks do not change while the handle lives (loads may run ahead of the stream)
   unsigned int inject;              // XKV_INJECT_* bits (xkv_debug_set_fault_injection); 0 in normal use
 };
 

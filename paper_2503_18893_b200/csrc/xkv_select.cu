@@ -101,17 +101,26 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
 
   // fault injection (tests of the give-up path): no load is issued, so the wait below must run into its limit
   const bool no_load = (dev.inject & XKV_INJECT_SCAN_NO_LOAD) != 0u;
-  grid_dependency_wait();          // the queries may come from the kernel launched before this one
+  // A handle's landmarks are constant while the handle is used (the caller's contract), so their loads may start
+  // before the kernel launched before this one has finished; the queries may come from that kernel and are
+  // read after the dependency wait.  Without a handle (the allocation-free entry point) nothing is known about
+  // the landmarks, and the loads wait too.
+  const bool early = dev.lm_const != 0;
+  if (!early) grid_dependency_wait();
   if (threadIdx.x == 0) {          // the thread that initialises the barrier also issues the loads: nothing to wait for
     mbar_init(bar, 1);
     fence_mbar_init();
     if (!no_load) {
       mbar_expect_tx(bar, (uint32_t)((DH / 64) * kScoreRows * 128));
       const int y = (int)(prob_lm * dev.n_c + j0);
+      // every landmark is read once per call: first in line for eviction, so that the stream does not push the
+      // pooled scores (written below, read by the top-k) and the gathered basis rows out of L2
+      const uint64_t pol = l2_policy_evict_first();
 #pragma unroll
-      for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar);
+      for (int bx = 0; bx < DH / 64; ++bx) tma_load_2d_hint(tile + bx * kScoreRows * 128, &tmap, bx * 64, y, bar, pol);
     }
   }
+  if (early) grid_dependency_wait();
   grid_dependency_launch();
   // queries of this KV head, widened to fp32 while the landmarks are in flight
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * dev.n_rep) * DH;
