@@ -172,6 +172,24 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
                                            void* out, float* lse, void* stream);
 
 /*
+ * Plain decode attention over an UNCOMPRESSED bf16 cache: out_h = softmax(scale * q_h K^T) V for the query heads of
+ * every (layer, sequence, KV head).  This is the baseline that selective reconstruction is measured against (Sec. 5,
+ * "Efficiency Studies": full attention reads the whole cache, SR removes the term that grows with the context); it
+ * runs the kernels of the uncompressed tail with several tiles per CTA and a merge of its own.
+ * K, V       bf16 [G][batch][H_kv][cap][d_h], device, borrowed for the call; keys as the model stores them (rotated).
+ * len        int32 [batch], device, or NULL for cap rows in every sequence (clamped to cap, flag raised, as for the tail).
+ * cap        1 <= cap <= XKV_DENSE_MAX_ROWS; beyond XKV_TAIL_MAX_ROWS only d_h = 128 is served (else UNSUPPORTED).
+ * workspace  device scratch of at least xkv_dense_workspace_bytes(grp, cap) bytes, 16-byte aligned, caller-owned.
+ * The handle supplies the shapes (G, batch, heads, d_h) and the softmax scale; its factors are not read.
+ * With len = 0 a head's output is 0 and its lse is -inf.  Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+#define XKV_DENSE_MAX_ROWS (1 << 22)
+XKV_API int xkv_dense_workspace_bytes(const xkv_group* grp, int32_t cap, uint64_t* bytes);
+XKV_API int xkv_dense_attend(xkv_group* grp, int layer_begin, int layer_end, const void* q, const void* K, const void* V,
+                             const int32_t* len, int32_t cap, void* workspace, uint64_t workspace_bytes, void* out,
+                             float* lse, void* stream);
+
+/*
  * Algorithm 1 (App. B.1), the prefill side of the selector, for every sequence, layer and KV head g:
  *   landmark[j]  = mean over the rows x of chunk j of rope(K[x]),  chunk j = rows c*j .. min(c*j+c, T)-1   (lines 1-3)
  *   min_cos[j]   = min over those rows of cos(rope(K[x]), landmark[j])  (fp32, the unrounded mean; a zero vector

@@ -417,4 +417,31 @@ int xkv_sr_reconstruct_attend_tail(xkv_group* g, int layer_begin, int layer_end,
   return XKV_OK;
 }
 
+int xkv_dense_workspace_bytes(const xkv_group* g, int32_t cap, uint64_t* bytes) {
+  if (!g || !bytes || cap < 1 || cap > XKV_DENSE_MAX_ROWS) return XKV_ERR_INVALID_ARG;
+  if (!dense_supported(g, cap)) return XKV_ERR_UNSUPPORTED;
+  *bytes = (uint64_t)tail_part_floats(g, cap) * sizeof(float);
+  return XKV_OK;
+}
+
+int xkv_dense_attend(xkv_group* g, int layer_begin, int layer_end, const void* q, const void* K, const void* V,
+                     const int32_t* len, int32_t cap, void* workspace, uint64_t workspace_bytes, void* out, float* lse,
+                     void* stream) {
+  if (!g || !q || !K || !V || !workspace || !out) return XKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
+  if (cap < 1 || cap > XKV_DENSE_MAX_ROWS) return XKV_ERR_INVALID_ARG;
+  if (!dense_supported(g, cap)) return XKV_ERR_UNSUPPORTED;
+  if (workspace_bytes < (uint64_t)tail_part_floats(g, cap) * sizeof(float)) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)lse & 3u) || ((uintptr_t)K & 15u) ||
+      ((uintptr_t)V & 15u) || ((uintptr_t)len & 3u) || ((uintptr_t)workspace & 15u))
+    return XKV_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = launch_tail_partials(g, layer_begin, layer_end, (const __nv_bfloat16*)q, (const __nv_bfloat16*)K,
+                                       (const __nv_bfloat16*)V, len, cap, (float*)workspace, s);
+  if (e == cudaSuccess)
+    e = launch_dense_merge(g, layer_begin, layer_end, (const float*)workspace, cap, (__nv_bfloat16*)out, lse, s);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
 }  // extern "C"

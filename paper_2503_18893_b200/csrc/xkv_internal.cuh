@@ -143,6 +143,10 @@ struct TailParts {
   int n_split;
 };
 int tail_splits(int tail_cap);
+int tail_tiles_per_split(int tail_cap);
+bool dense_supported(const xkv_group* grp, int cap);
+cudaError_t launch_dense_merge(const xkv_group* grp, int l0, int l1, const float* part, int cap, __nv_bfloat16* out,
+                               float* lse, cudaStream_t s);
 size_t tail_part_floats(const xkv_group* grp, int tail_cap);
 cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const __nv_bfloat16* tail_k,
                                  const __nv_bfloat16* tail_v, const int32_t* tail_len, int tail_cap, float* part,

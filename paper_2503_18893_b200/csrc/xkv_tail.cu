@@ -224,12 +224,12 @@ template <int NR>
 __global__ void __launch_bounds__(kTailThreads)
 tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ tail_k,
                const __nv_bfloat16* __restrict__ tail_v, const int32_t* __restrict__ tail_len, int tail_cap,
-               int n_split, float* __restrict__ part) {
+               int n_split, int tiles_per_split, float* __restrict__ part) {
   using namespace ptx;
   constexpr int DH = 128;
   extern __shared__ uint8_t tc_smem[];
   __shared__ float red_s[NR * (kTailThreads / 32)];
-  __shared__ float m_s[NR];
+  __shared__ float m_s[2][NR];                         // running maximum per head, before and after the current tile
   const uint32_t base = (smem_u32(tc_smem) + 1023u) & ~1023u;
   uint8_t* gen = tc_smem + (base - smem_u32(tc_smem));
   const uint32_t k_addr = base, v_addr = base + 2 * kTcSlab, q_addr = base + 4 * kTcSlab, p_addr = q_addr + 4096;
@@ -251,6 +251,7 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
   }
   // operands that stay zero: heads that do not exist (q rows, weight rows)
   for (int i = tid; i < 8192 / 4; i += kTailThreads) reinterpret_cast<uint32_t*>(q_gen)[i] = 0u;
+  if (tid < NR) { m_s[0][tid] = -INFINITY; m_s[1][tid] = -INFINITY; }
   if (warp == 0) {
     tmem_alloc(smem_u32(tmem_slot), 32);
     tmem_relinquish();
@@ -267,124 +268,156 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
     if (tid == 0 && split == 0) atomicOr(dev.flags, XKV_FLAG_INDEX_RANGE);
     len = len < 0 ? 0 : tail_cap;
   }
-  const int r_begin = split * kTailSplitRows;
-  const int rows = max(0, min(len - r_begin, kTailSplitRows));
-
-  // ---- stage K and V in the tensor core's layout: 64-column slabs, 128-byte rows, 16-byte units swizzled by the
-  // row; rows beyond `rows` are zero-filled (a weight of zero times garbage would still be garbage)
-  const size_t head_rows = (((size_t)l * dev.batch + b) * dev.H_kv + g) * (size_t)tail_cap + r_begin;
-  const __nv_bfloat16* Kh = tail_k + head_rows * DH;
-  const __nv_bfloat16* Vh = tail_v + head_rows * DH;
-  for (int i = tid; i < kTailThreads * 16; i += kTailThreads) {
-    const int r = i >> 4, c = i & 15;                  // row, 16-byte piece of the 256-byte row
-    const uint32_t off = (uint32_t)(c >> 3) * kTcSlab + (uint32_t)r * 128u + ((((uint32_t)c & 7u) ^ ((uint32_t)r & 7u)) << 4);
-    const uint32_t nb = r < rows ? 16u : 0u;
-    const size_t src = (size_t)(r < rows ? r : 0) * DH + c * 8;
-    cp_async16(k_addr + off, Kh + src, nb);
-    cp_async16(v_addr + off, Vh + src, nb);
-  }
-  cp_async_commit();
-  // q as the B operand of the logits: [16 heads][128 dims], K-major, same slab/swizzle scheme
+  // q as the B operand of the logits: [16 heads][128 dims], K-major, 64-column slabs, 128-byte swizzle
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep) * DH;
   for (int i = tid; i < n_rep * 16; i += kTailThreads) {
     const int h = i >> 4, c = i & 15;
     const uint4 v = *reinterpret_cast<const uint4*>(qg + h * DH + c * 8);
     *reinterpret_cast<uint4*>(q_gen + (c >> 3) * 2048 + h * 128 + (((c & 7) ^ (h & 7)) << 4)) = v;
   }
-  cp_async_wait<0>();
-  fence_proxy_async();                                 // the tensor core reads what this thread wrote or copied
-  __syncthreads();
-
   const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
   constexpr uint32_t idesc_s = idesc_bf16_f32(128, 16);
   constexpr uint32_t idesc_o = idesc_bf16_f32(128, 16) | (1u << 15);          // A read along its rows (MN-major)
-  // ---- logits
-  if (tid == 0) {
-    const uint32_t k_lo = (uint32_t)(smem_desc_sw128(k_addr, 0) & 0xFFFFFFFFull);
-    const uint32_t q_lo = (uint32_t)(smem_desc_sw128(q_addr, 0) & 0xFFFFFFFFull);
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {                   // 16 dims per step: 32 bytes along the row, next slab after four
-      const uint32_t a = k_lo + (uint32_t)(kk >> 2) * (kTcSlab >> 4) + (uint32_t)(kk & 3) * 2u;
-      const uint32_t bq = q_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
-      tc_mma_bf16(tmem, desc_hi | a, desc_hi | bq, idesc_s, kk ? 1u : 0u);
-    }
-    tc_commit(bar_s);
-  }
-  // the outcome of a wait is made CTA-uniform (one thread's poll may run out a moment before another's succeeds)
-  bool ok = __syncthreads_and(tc_wait_bounded(bar_s, 0) ? 1 : 0) != 0;
-  tc_fence_after();
   const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-  const bool valid = tid < rows;
-  float z[NR];
-  if (ok) {
+  const size_t head_rows = (((size_t)l * dev.batch + b) * dev.H_kv + g) * (size_t)tail_cap;
+
+  // running results of the split: thread = output column d for acc, thread = row for the weight sums
+  float acc[NR], l_thr[NR];
+#pragma unroll
+  for (int h = 0; h < NR; ++h) { acc[h] = 0.0f; l_thr[h] = 0.0f; }
+  bool ok = true;
+  int issued = 0;                                      // MMA group committed and not yet known to have retired: 0 none, 1 logits, 2 values
+  uint32_t issued_par = 0;                             // barrier phase that group completes
+  // A split is `tiles_per_split` consecutive 128-row tiles, walked with a running softmax (one tile for tails up
+  // to XKV_TAIL_MAX_ROWS; more for the long caches of xkv_dense_attend, so that the merge sees a bounded number
+  // of partial results).
+  for (int t = 0; t < tiles_per_split; ++t) {
+    const int r_begin = (split * tiles_per_split + t) * kTailSplitRows;
+    const int rows = max(0, min(len - r_begin, kTailSplitRows));
+    if (rows == 0 && t > 0) break;                     // CTA-uniform: the split ends inside the cache
+    const int cur = t & 1, nxt = cur ^ 1;
+    const uint32_t par = (uint32_t)(t & 1);
+    // ---- stage K and V in the tensor core's layout: 64-column slabs, 128-byte rows, 16-byte units swizzled by
+    // the row; rows beyond `rows` are zero-filled (a weight of zero times garbage would still be garbage)
+    const __nv_bfloat16* Kh = tail_k + (head_rows + r_begin) * DH;
+    const __nv_bfloat16* Vh = tail_v + (head_rows + r_begin) * DH;
+    for (int i = tid; i < kTailThreads * 16; i += kTailThreads) {
+      const int r = i >> 4, c = i & 15;                // row, 16-byte piece of the 256-byte row
+      const uint32_t off = (uint32_t)(c >> 3) * kTcSlab + (uint32_t)r * 128u + ((((uint32_t)c & 7u) ^ ((uint32_t)r & 7u)) << 4);
+      const uint32_t nb = r < rows ? 16u : 0u;
+      const size_t src = (size_t)(r < rows ? r : 0) * DH + c * 8;
+      cp_async16(k_addr + off, Kh + src, nb);
+      cp_async16(v_addr + off, Vh + src, nb);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    fence_proxy_async();                               // the tensor core reads what this thread wrote or copied
+    __syncthreads();
+    // ---- logits
+    if (tid == 0) {
+      const uint32_t k_lo = (uint32_t)(smem_desc_sw128(k_addr, 0) & 0xFFFFFFFFull);
+      const uint32_t q_lo = (uint32_t)(smem_desc_sw128(q_addr, 0) & 0xFFFFFFFFull);
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {                 // 16 dims per step: 32 bytes along the row, next slab after four
+        const uint32_t a = k_lo + (uint32_t)(kk >> 2) * (kTcSlab >> 4) + (uint32_t)(kk & 3) * 2u;
+        const uint32_t bq = q_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
+        tc_mma_bf16(tmem, desc_hi | a, desc_hi | bq, idesc_s, kk ? 1u : 0u);
+      }
+      tc_commit(bar_s);
+    }
+    issued = 1; issued_par = par;
+    // the outcome of a wait is made CTA-uniform (one thread's poll may run out a moment before another's succeeds)
+    ok = __syncthreads_and(tc_wait_bounded(bar_s, par) ? 1 : 0) != 0;
+    if (!ok) break;
+    issued = 0;
+    tc_fence_after();
+    const bool valid = tid < rows;
+    float z[NR];
     tmem_ld<NR>(tmem + lane_base, z);
     tc_wait_ld();
-  } else {
+    // ---- tile maximum per head, folded into the running maximum
 #pragma unroll
-    for (int h = 0; h < NR; ++h) z[h] = 0.0f;
+    for (int h = 0; h < NR; ++h) {
+      z[h] = valid ? z[h] * scale2 : -INFINITY;
+      float v = z[h];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;
+    }
+    __syncthreads();
+    if (tid < NR) {
+      float tm = red_s[tid * (kTailThreads / 32)];
+#pragma unroll
+      for (int w = 1; w < kTailThreads / 32; ++w) tm = fmaxf(tm, red_s[tid * (kTailThreads / 32) + w]);
+      m_s[nxt][tid] = fmaxf(m_s[cur][tid], tm);
+    }
+    __syncthreads();
+    // ---- weights as the bf16 B operand [row block][head][64 rows]; the denominator sums the rounded values
+    float alpha[NR];
+    {
+      uint8_t* Pw = p_gen + (tid >> 6) * 2048 + (tid & 7) * 2;
+      const uint32_t p_unit = (uint32_t)((tid & 63) >> 3);
+#pragma unroll
+      for (int h = 0; h < NR; ++h) {
+        const float mo = m_s[cur][h], mn = m_s[nxt][h];
+        alpha[h] = (mo == -INFINITY) ? 0.0f : ex2_approx(mo - mn);
+        const float p = (valid && mn != -INFINITY) ? ex2_approx(z[h] - mn) : 0.0f;
+        const __nv_bfloat16 pb = __float2bfloat16(p);
+        if (h < n_rep) *reinterpret_cast<__nv_bfloat16*>(Pw + h * 128 + ((p_unit ^ (uint32_t)(h & 7)) << 4)) = pb;
+        l_thr[h] = l_thr[h] * alpha[h] + __bfloat162float(pb);
+      }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // ---- values: O^T[d][head] = V^T P^T
+    if (tid == 0) {
+      const uint32_t v_lo = ((uint32_t)(smem_desc_sw128(v_addr, 0) & 0xFFFFull)) | ((uint32_t)(kTcSlab >> 4) << 16);
+      const uint32_t p_lo = (uint32_t)(smem_desc_sw128(p_addr, 0) & 0xFFFFFFFFull);
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {                 // 16 tile rows per step: 2048 bytes down the slab, 32 bytes along P
+        const uint32_t bp = p_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
+        tc_mma_bf16(tmem + 16u, desc_hi | (v_lo + (uint32_t)kk * (2048u >> 4)), desc_hi | bp, idesc_o, kk ? 1u : 0u);
+      }
+      tc_commit(bar_o);
+    }
+    issued = 2; issued_par = par;
+    ok = __syncthreads_and(tc_wait_bounded(bar_o, par) ? 1 : 0) != 0;
+    if (!ok) break;
+    issued = 0;
+    tc_fence_after();
+    float o[NR];
+    tmem_ld<NR>(tmem + lane_base + 16u, o);
+    tc_wait_ld();
+#pragma unroll
+    for (int h = 0; h < NR; ++h) acc[h] = fmaf(acc[h], alpha[h], o[h]);
+    tc_fence_before();
+    __syncthreads();                                   // the tile's memory and both accumulators may be reused
+    tc_fence_after();
   }
-  // ---- tile maximum per head
+  if (!ok) {
+    if (tid == 0) {
+      atomicOr(dev.flags, XKV_FLAG_TIMEOUT);
+      // giving up: the MMAs issued above may still be running; wait once more (bounded) for the barrier that
+      // their commit arrives on before the tensor memory is freed
+      if (issued) (void)tc_wait_bounded(issued == 1 ? bar_s : bar_o, issued_par);
+    }
+#pragma unroll
+    for (int h = 0; h < NR; ++h) { acc[h] = 0.0f; l_thr[h] = 0.0f; }
+  }
+  // ---- per head: sum of the weights over the rows (thread = row)
+  __syncthreads();
 #pragma unroll
   for (int h = 0; h < NR; ++h) {
-    z[h] = valid ? z[h] * scale2 : -INFINITY;
-    float v = z[h];
+    float v = l_thr[h];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;
   }
   __syncthreads();
-  if (tid < NR) {
-    float tm = red_s[tid * (kTailThreads / 32)];
-#pragma unroll
-    for (int w = 1; w < kTailThreads / 32; ++w) tm = fmaxf(tm, red_s[tid * (kTailThreads / 32) + w]);
-    m_s[tid] = tm;
-  }
-  __syncthreads();
-  // ---- weights as the bf16 B operand [row block][head][64 rows] and their sums (of the rounded values)
-  {
-    uint8_t* Pw = p_gen + (tid >> 6) * 2048 + (tid & 7) * 2;
-    const uint32_t p_unit = (uint32_t)((tid & 63) >> 3);
-#pragma unroll
-    for (int h = 0; h < NR; ++h) {
-      const float mn = m_s[h];
-      const float p = (valid && mn != -INFINITY) ? ex2_approx(z[h] - mn) : 0.0f;
-      const __nv_bfloat16 pb = __float2bfloat16(p);
-      if (h < n_rep) *reinterpret_cast<__nv_bfloat16*>(Pw + h * 128 + ((p_unit ^ (uint32_t)(h & 7)) << 4)) = pb;
-      float v = __bfloat162float(pb);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) red_s[h * (kTailThreads / 32) + warp] = v;    // (the maxima were consumed before the last barrier)
-    }
-  }
-  fence_proxy_async();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  // ---- values: O^T[d][head] = V^T P^T
-  if (tid == 0 && ok) {
-    const uint32_t v_lo = ((uint32_t)(smem_desc_sw128(v_addr, 0) & 0xFFFFull)) | ((uint32_t)(kTcSlab >> 4) << 16);
-    const uint32_t p_lo = (uint32_t)(smem_desc_sw128(p_addr, 0) & 0xFFFFFFFFull);
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {                   // 16 tile rows per step: 2048 bytes down the slab, 32 bytes along P
-      const uint32_t bp = p_lo + (uint32_t)(kk >> 2) * (2048u >> 4) + (uint32_t)(kk & 3) * 2u;
-      tc_mma_bf16(tmem + 16u, desc_hi | (v_lo + (uint32_t)kk * (2048u >> 4)), desc_hi | bp, idesc_o, kk ? 1u : 0u);
-    }
-    tc_commit(bar_o);
-  }
-  const bool ok_s = ok;
-  if (ok) ok = tc_wait_bounded(bar_o, 0);
-  ok = __syncthreads_and(ok ? 1 : 0) != 0;
-  tc_fence_after();
-  float acc[NR];
-  if (ok) {
-    tmem_ld<NR>(tmem + lane_base + 16u, acc);
-    tc_wait_ld();
-  } else {
-    if (tid == 0) atomicOr(dev.flags, XKV_FLAG_TIMEOUT);
-#pragma unroll
-    for (int h = 0; h < NR; ++h) acc[h] = 0.0f;
-  }
-  // ---- write the partial: [py][split][head][DH + 2]
+  // ---- write the partial: [py][split][head][DH + 2].  The running maximum alternates between m_s[0] and m_s[1]
+  // and never decreases, so the larger of the two is the final one.
   float* dst = part + (((size_t)py * n_split + split) * n_rep) * (DH + 2);
 #pragma unroll
   for (int h = 0; h < NR; ++h) {
@@ -394,15 +427,10 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
         float ls = 0.0f;
 #pragma unroll
         for (int w = 0; w < kTailThreads / 32; ++w) ls += red_s[h * (kTailThreads / 32) + w];
-        dst[(size_t)h * (DH + 2) + DH] = m_s[h];
+        dst[(size_t)h * (DH + 2) + DH] = ok ? fmaxf(m_s[0][h], m_s[1][h]) : -INFINITY;
         dst[(size_t)h * (DH + 2) + DH + 1] = ls;
       }
     }
-  }
-  if (!ok && tid == 0) {
-    // giving up: the MMAs issued above may still be running; wait once more (bounded) for the barrier that their
-    // commit arrives on before the tensor memory is freed
-    (void)tc_wait_bounded(ok_s ? bar_o : bar_s, 0);
   }
   tc_fence_before();
   __syncthreads();
@@ -412,9 +440,73 @@ tail_tc_kernel(GroupDev dev, int l0, const __nv_bfloat16* __restrict__ q, const 
   }
 }
 
+// Merge of dense-attention partials (xkv_dense_attend): one CTA per (problem, query head); the splits are
+// spread over 1024 / DH groups of DH threads, thread = output column.  m is in log2 units.
+constexpr int kDenseMergeThreads = 1024;
+template <int DH>
+__global__ void __launch_bounds__(kDenseMergeThreads)
+dense_merge_kernel(GroupDev dev, int l0, const float* __restrict__ part, int n_split, __nv_bfloat16* __restrict__ out,
+                   float* __restrict__ lse) {
+  __shared__ float twgt_s[kTailMaxSplit];
+  __shared__ float ML_s[2];
+  __shared__ float red[kDenseMergeThreads];
+  constexpr int FOLD = kDenseMergeThreads / DH;
+  const int tid = threadIdx.x, n_rep = dev.n_rep;
+  const int h = blockIdx.x % n_rep, py = blockIdx.x / n_rep;
+  const int per_layer = dev.batch * dev.H_kv;
+  const int g = py % dev.H_kv, b = (py / dev.H_kv) % dev.batch, l = l0 + py / per_layer;
+  ptx::grid_dependency_wait();                         // the partials come from the kernel launched before this one
+  ptx::grid_dependency_launch();
+  const int nts = min(n_split, kTailMaxSplit);
+  const size_t tstride = (size_t)n_rep * (DH + 2);
+  const float* tpart = part + ((size_t)py * n_split) * tstride + (size_t)h * (DH + 2);
+  if (tid < 32) {
+    float mx = -INFINITY;
+    for (int s = tid; s < nts; s += 32) mx = fmaxf(mx, tpart[s * tstride + DH]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float Ls = 0.0f;
+    for (int s = tid; s < nts; s += 32) {
+      const float ms = tpart[s * tstride + DH];
+      const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
+      twgt_s[s] = w;
+      Ls += w * tpart[s * tstride + DH + 1];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
+    if (tid == 0) { ML_s[0] = mx; ML_s[1] = Ls; }
+  }
+  __syncthreads();
+  const int d = tid % DH, f = tid / DH;
+  float o = 0.0f;
+#pragma unroll 4
+  for (int s = f; s < nts; s += FOLD) o = fmaf(twgt_s[s], tpart[s * tstride + d], o);
+  red[f * DH + d] = o;
+  __syncthreads();
+  if (tid < DH) {
+    float v = 0.0f;
+#pragma unroll
+    for (int i = 0; i < FOLD; ++i) v += red[i * DH + tid];
+    const float M = ML_s[0], L = ML_s[1];
+    const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h;
+    out[qh * DH + tid] = __float2bfloat16(L > 0.0f ? v / L : 0.0f);
+    if (lse && tid == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+  }
+}
+
 }  // namespace
 
-int tail_splits(int tail_cap) { return (tail_cap + kTailSplitRows - 1) / kTailSplitRows; }
+// Tiles walked by one CTA of the tail kernels: one while the merge's table of partial results holds every tile,
+// more for longer caches (dense attention).
+int tail_tiles_per_split(int tail_cap) {
+  const int tiles = (tail_cap + kTailSplitRows - 1) / kTailSplitRows;
+  return (tiles + kTailMaxSplit - 1) / kTailMaxSplit;
+}
+
+int tail_splits(int tail_cap) {
+  const int tiles = (tail_cap + kTailSplitRows - 1) / kTailSplitRows, tps = tail_tiles_per_split(tail_cap);
+  return (tiles + tps - 1) / tps;
+}
 
 size_t tail_part_floats(const xkv_group* grp, int tail_cap) {
   const xkv_group_config& c = grp->cfg;
@@ -426,9 +518,11 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
                                  cudaStream_t s) {
   const GroupDev& dev = grp->dev;
   const int problems = (l1 - l0) * dev.batch * dev.H_kv;
-  const int n_split = tail_splits(tail_cap);
+  const int n_split = tail_splits(tail_cap), tps = tail_tiles_per_split(tail_cap);
   cudaError_t e = cudaSuccess;
   const dim3 grid(problems, n_split), block(kTailThreads);
+  // only the tensor-core kernel walks several tiles per CTA
+  if (tps > 1 && !(dev.d_h == 128 && !grp->tail_impl)) return cudaErrorInvalidValue;
 #define XKV_TAIL(DH, NR)                                                                                            \
   do {                                                                                                              \
     e = ensure_dyn_smem<tail_partial_kernel<DH, NR>>(tail_smem_bytes<DH, NR>(), grp->device);                       \
@@ -441,7 +535,7 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
     e = ensure_dyn_smem<tail_tc_kernel<NR>>(tail_tc_smem_bytes<NR>(), grp->device);                                 \
     if (e == cudaSuccess)                                                                                           \
       e = launch_pdl(tail_tc_kernel<NR>, grid, block, tail_tc_smem_bytes<NR>(), s, dev, l0, q, tail_k, tail_v,       \
-                     tail_len, tail_cap, n_split, part);                                                            \
+                     tail_len, tail_cap, n_split, tps, part);                                                       \
   } while (0)
   if (dev.d_h == 128 && !grp->tail_impl) {
     if (dev.n_rep <= 4) XKV_TAIL_TC(4); else if (dev.n_rep <= 8) XKV_TAIL_TC(8); else XKV_TAIL_TC(16);
@@ -453,6 +547,27 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
 #undef XKV_TAIL
 #undef XKV_TAIL_TC
   count_launch((dev.d_h == 128 && !grp->tail_impl) ? kFamTailTc : kFamTailCuda);
+  return e;
+}
+
+// Can xkv_dense_attend serve `cap` rows with this handle?  Longer caches than the tail limit need the multi-tile
+// (tensor-core, d_h = 128) kernel.
+bool dense_supported(const xkv_group* grp, int cap) {
+  return tail_tiles_per_split(cap) == 1 || (grp->dev.d_h == 128 && !grp->tail_impl);
+}
+
+cudaError_t launch_dense_merge(const xkv_group* grp, int l0, int l1, const float* part, int cap, __nv_bfloat16* out,
+                               float* lse, cudaStream_t s) {
+  const GroupDev& dev = grp->dev;
+  const int problems = (l1 - l0) * dev.batch * dev.H_kv;
+  cudaError_t e;
+  if (dev.d_h == 128)
+    e = launch_pdl(dense_merge_kernel<128>, dim3(problems * dev.n_rep), dim3(kDenseMergeThreads), 0, s, dev, l0, part,
+                   tail_splits(cap), out, lse);
+  else
+    e = launch_pdl(dense_merge_kernel<64>, dim3(problems * dev.n_rep), dim3(kDenseMergeThreads), 0, s, dev, l0, part,
+                   tail_splits(cap), out, lse);
+  count_launch(kFamDense);
   return e;
 }
 

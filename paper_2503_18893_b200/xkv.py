@@ -77,6 +77,15 @@ _lib.xkv_sr_reconstruct_attend_tail.argtypes = [_P, ctypes.c_int, ctypes.c_int, 
 _lib.xkv_sr_reconstruct_attend_tail.restype = ctypes.c_int
 
 
+_lib.xkv_dense_workspace_bytes.argtypes = [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_dense_workspace_bytes.restype = ctypes.c_int
+_lib.xkv_dense_attend.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, ctypes.c_int32, _P, ctypes.c_uint64,
+                                  _P, _P, _P]
+_lib.xkv_dense_attend.restype = ctypes.c_int
+XKV_DENSE_MAX_ROWS = 1 << 22
+XKV_TAIL_MAX_ROWS = 32768
+
+
 class xkv_landmark_config(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("G", ctypes.c_int32), ("batch", ctypes.c_int32),
                 ("T", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("d_h", ctypes.c_int32), ("chunk", ctypes.c_int32),
@@ -273,6 +282,24 @@ def xkv_sr_reconstruct_attend_tail(grp: Group, layer_begin: int, layer_end: int,
                                              _ptr(out), _ptr(lse), _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_sr_reconstruct_attend_tail")
+
+
+def xkv_dense_workspace_bytes(grp: Group, cap: int) -> int:
+    b = ctypes.c_uint64()
+    st = _lib.xkv_dense_workspace_bytes(grp.handle, cap, ctypes.byref(b))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_dense_workspace_bytes")
+    return b.value
+
+
+def xkv_dense_attend(grp: Group, layer_begin: int, layer_end: int, q, K, V, length, cap: int, workspace, out, lse=None,
+                     stream=None) -> None:
+    """Plain decode attention over an uncompressed cache K, V [G][batch][H_kv][cap][d_h] (the dense baseline)."""
+    st = _lib.xkv_dense_attend(grp.handle, layer_begin, layer_end, _ptr(q), _ptr(K), _ptr(V), _ptr(length), cap,
+                               _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(out), _ptr(lse),
+                               _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_dense_attend")
 
 
 def xkv_group_status(grp: Group, stream=None):
