@@ -27,9 +27,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, sr_fused_kernel (95.46 + 3.38 MB) + merge_segments_kernel
-# (5.65 MB), one window of config 3
-NCU_ATTEND_DRAM_BYTES = 104.5e6
 METRIC = "SR decode steps/sec per layer group at 128K ctx"
 UNIT = "group-steps/s"
 
@@ -54,6 +51,15 @@ def parse_args():
     ap.add_argument("--op", default="decode", choices=["decode", "landmarks"],
                     help="decode: the hot path (default).  landmarks: the prefill-side Algorithm 1 kernel alone "
                          "(not the headline metric; prints its own JSON line)")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="times the `steps`-step region is repeated (0: as many as make about a second of timed work)")
+    ap.add_argument("--dense", action="store_true",
+                    help="also time plain decode attention over an uncompressed bf16 cache of the same shape")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the other benchmark configurations and the corner points of the stress sweep, one JSON "
+                         "line per point (each with the dense-attention arm and a parity check)")
+    ap.add_argument("--sweep-out", default=None, help="with --sweep: also write a markdown table to this file")
+    ap.add_argument("--sweep-filter", default=None, help="with --sweep: only the points whose label contains this text")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-problems", type=int, default=None, help="oracle sample size in (layer,head) problems")
     return ap.parse_args()
@@ -73,11 +79,10 @@ def make_shape(args):
     return synth.config(args.config, **over)
 
 
-def shard_units(n_units: int, rank: int, world: int):
-    """Contiguous share of n_units independent units for `rank` (sizes differ by at most one)."""
-    lo = (n_units * rank) // world
-    hi = (n_units * (rank + 1)) // world
-    return list(range(lo, hi))
+def replica_units(n_windows: int, rank: int):
+    """Ids of the synthetic windows that rank `rank` serves: every rank holds a full replica of the workload made of
+    its own sequences (fixed work per GPU: weak scaling), so the ids of different ranks never overlap."""
+    return list(range(rank * n_windows, (rank + 1) * n_windows))
 
 
 def reduce_max(value: float, dist=None) -> float:
@@ -148,25 +153,70 @@ def peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def oracle_sample(shape, inp, n_problems):
-    """Time the CPU oracle (as it stands) on the first n_problems (layer, sequence, head) problems of a window.
-    Returns (seconds, problems, threads)."""
+def oracle_sample(shape, inp, n_problems, spread=False):
+    """Time the CPU oracle (as it stands) on n_problems (layer, sequence, head) problems of a window: the first
+    ones, or (spread) ones spread evenly over the window.  Returns (seconds, problems, cores, results) where cores is
+    the CPU time the call used divided by its wall time (the oracle's scoring loop is serial numpy; only its
+    BLAS calls use several threads) and results = (problem list, sel_idx, sel_cnt, out, lse) of the oracle."""
     import numpy as np
     from oracle import xkv_oracle as O
     f32 = lambda t: t.detach().float().cpu().numpy()
-    A_k, A_v, B_k, B_v, lm, q = (f32(t) for t in (inp.A_k, inp.A_v, inp.B_k, inp.B_v, inp.landmarks, inp.q[0]))
     allp = [(l, b, g) for l in range(shape.G) for b in range(shape.batch) for g in range(shape.H_kv)]
-    probs = allp[:n_problems]
-    t0 = time.perf_counter()
-    O.sr_decode_step(A_k, A_v, B_k, B_v, lm, q, k=shape.k, c=shape.c, H_kv=shape.H_kv, rope_base=shape.rope_base,
-                     problems=probs)
-    dt = time.perf_counter() - t0
+    n_problems = min(n_problems, len(allp))
+    probs = [allp[(i * len(allp)) // n_problems] for i in range(n_problems)] if spread else allp[:n_problems]
+    # only the sequences the sample touches are widened to fp32 on the host
+    seqs = sorted({b for (_, b, _) in probs})
+    pos = {b: i for i, b in enumerate(seqs)}
+    A_k, A_v, B_k, B_v, lm = (f32(t[seqs]) for t in (inp.A_k, inp.A_v, inp.B_k, inp.B_v, inp.landmarks))
+    q = f32(inp.q[0][:, seqs])
+    sub = [(l, pos[b], g) for (l, b, g) in probs]
+    c0, t0 = time.process_time(), time.perf_counter()
+    res = O.sr_decode_step(A_k, A_v, B_k, B_v, lm, q, k=shape.k, c=shape.c, H_kv=shape.H_kv, rope_base=shape.rope_base,
+                           problems=sub)
+    dt, cpu = time.perf_counter() - t0, time.process_time() - c0
+    # back to the full batch numbering
+    full = []
+    for a in res:
+        z = np.zeros(a.shape[:1] + (shape.batch,) + a.shape[2:], dtype=a.dtype)
+        z[:, seqs] = a
+        full.append(z)
+    return dt, len(probs), round(max(1.0, cpu / max(dt, 1e-9)), 1), (probs,) + tuple(full)
+
+
+def parity_against(shape, oracle_results, gidx, gcnt, gout, glse):
+    """Compare the library's results of one window-step with the oracle's on the problems the oracle evaluated:
+    number of index-set mismatches, worst relative error per output vector, worst absolute LSE error."""
+    import numpy as np
+    probs, oidx, ocnt, oout, olse = oracle_results
+    bad, err, lerr = 0, 0.0, 0.0
+    for (l, b, g) in probs:
+        if int(gcnt[l, b, g]) != int(ocnt[l, b, g]) or not np.array_equal(gidx[l, b, g], oidx[l, b, g]):
+            bad += 1
+        hs = slice(g * shape.n_rep, (g + 1) * shape.n_rep)
+        num = np.abs(gout[l, b, hs].astype(np.float64) - oout[l, b, hs]).max(axis=-1)
+        den = np.maximum(np.abs(oout[l, b, hs]).max(axis=-1), 1e-30)
+        err = max(err, float((num / den).max()))
+        lerr = max(lerr, float(np.abs(glse[l, b, hs] - olse[l, b, hs]).max()))
+    return {"problems_checked": len(probs), "idx_mismatch": bad, "max_rel_err": err, "max_lse_abs_err": lerr,
+            "tolerance": 2e-2}
+
+
+def captured_traffic(kernel_file: str):
+    """DRAM bytes per reconstruct_attend call from the ncu capture summarised under profiles/, if that capture was
+    taken from the kernel source as it is now (the summary records the source file's hash); else None."""
+    import glob
+    import hashlib
+    import re
     try:
-        from threadpoolctl import threadpool_info
-        threads = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
-    except Exception:
-        threads = os.cpu_count() or 1
-    return dt, len(probs), threads
+        with open(os.path.join(ROOT, "paper_2503_18893_b200", "csrc", kernel_file), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+    for path in glob.glob(os.path.join(ROOT, "profiles", "*.md")):
+        for m in re.finditer(r"capture-of: (\S+) sha256=(\w+) attend_dram_bytes_per_launch=([0-9.e+]+)", open(path).read()):
+            if m.group(1) == kernel_file and m.group(2) == digest:
+                return float(m.group(3))
+    return None
 
 
 def reference_inputs(shape, n_problems):
@@ -199,7 +249,7 @@ def run_reference(args):
     inp = reference_inputs(shape, n)
     times = []
     for i in range(args.warmup + args.steps):
-        dt, np_, threads = oracle_sample(shape, inp, n)
+        dt, np_, threads, _ = oracle_sample(shape, inp, n)
         if i >= args.warmup:
             times.append(dt)
     sec = sum(times)
@@ -266,35 +316,20 @@ def run_landmarks(args):
     return 0
 
 
-def main():
-    args = parse_args()
-    if args.op == "landmarks":
-        return run_landmarks(args)
-    if args.impl == "reference":
-        return run_reference(args)
-
+def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, with_dense=False, cpu_problems=None):
+    """Time the decode step of one workload on this rank's GPU and return the JSON line (a dict)."""
+    import numpy as np
     import torch
-    import torch.distributed as dist
-    from paper_2503_18893_b200 import workload
+    from paper_2503_18893_b200 import workload, xkv
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    from paper_2503_18893_b200 import xkv
-
-    shape = make_shape(args)
-    # Each rank owns one full replica of the workload (its own sequence): per-GPU work is fixed.
-    n_q = 8
-    wl = workload.DeviceWorkload(shape, n_steps=n_q, device="cuda", tail_rows=args.tail)
-    n_groups = len(wl.groups)
     s = shape
+    n_q = 8
+    wl = workload.DeviceWorkload(shape, n_steps=n_q, device="cuda", groups=replica_units(shape.n_groups, rank),
+                                 tail_rows=args.tail)
+    n_groups = len(wl.groups)
     q_bytes = n_groups * s.G * s.batch * s.H_q * s.d_h * 2
     out_bytes = q_bytes
+    ddist = dist if world > 1 else None
 
     def barrier():
         if world > 1:
@@ -302,6 +337,7 @@ def main():
         torch.cuda.synchronize()
 
     stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
     for i in range(args.warmup):
         wl.step(i)
         if i == 0:
@@ -309,28 +345,42 @@ def main():
             if st0 != 0:   # a kernel gave up on a bounded wait or saw a bad index: do not time a broken run
                 raise SystemExit(f"device status {st0} (flags {fl0}) after the first step: {xkv.xkv_strerror(st0)}")
     barrier()
+    # how often the `steps`-step region is repeated: about a second of timed work, so that the clock sampler sees
+    # the load and a slow outlier shows; one probe region decides
+    e0 = ev(); e0.record(stream)
+    for i in range(args.steps):
+        wl.step(i)
+    e1 = ev(); e1.record(stream)
+    barrier()
+    probe_ms = e0.elapsed_time(e1)
+    repeats = args.repeats if args.repeats > 0 else int(min(200, max(3, round(1000.0 / max(probe_ms, 1e-3)))))
+    if world > 1:       # every rank must run the same number of regions
+        repeats = int(reduce_max(float(repeats), dist))
 
-    # ---- timed region 1: inputs resident in HBM, exactly `steps` steps between two events
+    # ---- timed region 1: inputs resident in HBM; `repeats` regions of exactly `steps` steps, each between two
+    # events with a barrier on both sides; the reported region is the median one (max over ranks per region)
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    ev = lambda: torch.cuda.Event(enable_timing=True)
     launches0 = xkv.xkv_kernel_launch_count()
-    barrier()
     t_wall0 = time.time()
-    e_start = ev(); e_start.record(stream)
-    for i in range(args.steps):
-        wl.step(args.warmup + i)
-    e_stop = ev(); e_stop.record(stream)
-    barrier()
-    launches = xkv.xkv_kernel_launch_count() - launches0
-    ms_total = reduce_max(e_start.elapsed_time(e_stop), dist if world > 1 else None)
+    regions = []
+    for r in range(repeats):
+        barrier()
+        a = ev(); a.record(stream)
+        for i in range(args.steps):
+            wl.step(args.warmup + r * args.steps + i)
+        b = ev(); b.record(stream)
+        barrier()
+        regions.append(reduce_max(a.elapsed_time(b), ddist))
+    launches = (xkv.xkv_kernel_launch_count() - launches0) // repeats
+    ms_total = statistics.median(regions)
 
     # ---- timed region 1b: the same steps again with an event around every ABI call, for the per-kernel roofline
     # (kept out of region 1: an event between two calls keeps the second call's kernels from starting under
     # programmatic dependent launch while the first call's kernels drain)
     marks = []
-    for i in range(args.steps):
+    for i in range(max(args.steps, 10)):
         for gi, grp in enumerate(wl.groups):
             q = wl.inputs[gi].q[(args.warmup + i) % n_q]
             a = ev(); a.record(stream)
@@ -354,14 +404,15 @@ def main():
             uniq += int(torch.unique(rows[rows >= 0]).numel())
     uniq_per_group = uniq / n_groups
     bytes_model = workload.algorithmic_bytes(s, unique_rows=uniq_per_group)
-    flops = workload.algorithmic_flops(s)
+    flops_paper = workload.algorithmic_flops(s)
+    flops_exec = workload.executed_flops(s)
     pk = peaks()
 
     # ---- timed region 2: end to end through the C ABI with host buffers (pinned), copies inside
     q_host = [torch.stack([wl.inputs[gi].q[j] for gi in range(n_groups)]).cpu().pin_memory() for j in range(n_q)]
     q_dev = torch.empty_like(q_host[0], device="cuda")
     out_host = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
-    e2e_steps = max(3, args.steps // 2)
+    e2e_steps = max(3, min(args.steps * repeats, 200) // 2)
     barrier()
     e0 = ev(); e0.record(stream)
     for i in range(e2e_steps):
@@ -371,38 +422,48 @@ def main():
         stream.synchronize()                      # the caller consumes the result before the next token
     e1 = ev(); e1.record(stream)
     barrier()
-    e2e_ms = reduce_max(e0.elapsed_time(e1), dist if world > 1 else None)
+    e2e_ms = reduce_max(e0.elapsed_time(e1), ddist)
 
     total_group_steps = world * n_groups * args.steps
     value = total_group_steps / (ms_total * 1e-3)
     e2e_value = world * n_groups * e2e_steps / (e2e_ms * 1e-3)
+    us_window = (ms_total / args.steps / n_groups) * 1e3
 
-    # dominant kernel: reconstruct+attend (gather, contraction, attention); HBM bound at this shape
+    # ---- dominant kernel: the reconstruct+attend call (gather, contraction, attention).  Its bound is the larger
+    # of the byte term (unique gathered rows + B, at the measured HBM peak) and the tensor term of the flops the
+    # kernel executes (the value side is re-associated); the paper's cost formula is kept as a labelled side field.
     att_s = statistics.mean(att_ms) * 1e-3
     sel_s = statistics.mean(sel_ms) * 1e-3
     att_bytes = bytes_model["rows_unique"] + bytes_model["B"] + bytes_model["small"]
     sel_bytes = bytes_model["landmarks"]
     hbm_t = att_bytes / (pk["hbm_gbs"] * 1e9)
-    tc_t = flops / (pk["bf16_tflops_sustained"] * 1e12)
+    tc_t = flops_exec / (pk["bf16_tflops_sustained"] * 1e12)
     if hbm_t >= tc_t:
         roof = {"bound": "hbm", "achieved": att_bytes / att_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
     else:
-        roof = {"bound": "tensor", "achieved": flops / att_s / 1e12, "peak": pk["bf16_tflops_sustained"],
+        roof = {"bound": "tensor", "achieved": flops_exec / att_s / 1e12, "peak": pk["bf16_tflops_sustained"],
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    # DRAM bytes of one reconstruct_attend call (fused kernel + segment merge) from the ncu capture of one window of
-    # this workload (profiles/kernels_one_window_cfg3.md); it only applies to the unmodified headline shape.
-    traffic = None
-    if shape.name == "cfg3_llama_128k" and (s.T, s.r_k, s.r_v, s.k, s.batch) == (131072, 512, 512, 4096, 1):
-        traffic = NCU_ATTEND_DRAM_BYTES
-    roof.update({"traffic": traffic, "kernel": "xkv_sr_reconstruct_attend (gather + reconstruct + attention)",
+    headline_shape = (shape.name == "cfg3_llama_128k" and args.tail == 0 and
+                      (s.T, s.r_k, s.r_v, s.k, s.batch) == (131072, 512, 512, 4096, 1))
+    roof.update({"traffic": captured_traffic("xkv_fused.cu") if headline_shape else None,
+                 "kernel": "xkv_sr_reconstruct_attend (gather + reconstruct + attention)",
                  "peak_source": pk["source"], "us_per_launch": att_s * 1e6,
-                 "algorithmic_bytes_per_launch": att_bytes, "algorithmic_flops_per_launch": flops})
+                 "algorithmic_bytes_per_launch": att_bytes,
+                 "hbm_frac": att_bytes / att_s / 1e9 / pk["hbm_gbs"],
+                 "executed_flops_per_launch": flops_exec,
+                 "executed_tflops": flops_exec / att_s / 1e12,
+                 "executed_frac_of_bf16_peak": flops_exec / att_s / 1e12 / pk["bf16_tflops_sustained"],
+                 "paper_formula_flops_per_launch": flops_paper,
+                 "paper_formula_tflops": flops_paper / att_s / 1e12})
     step_t = max(bytes_model["bytes_min"] / (pk["hbm_gbs"] * 1e9), tc_t)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, world),
+        "repeats": {"regions": repeats, "steps_per_region": args.steps, "region_ms_median": ms_total,
+                    "region_ms_min": min(regions), "region_ms_max": max(regions),
+                    "value_from": "median region, max over ranks"},
         "tokens_per_s": world * s.batch * args.steps / (ms_total * 1e-3),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": q_bytes, "d2h_bytes_per_step": out_bytes,
                 "steps": e2e_steps},
@@ -413,30 +474,203 @@ def main():
                           "achieved_gbs": sel_bytes / sel_s / 1e9, "frac": sel_bytes / sel_s / 1e9 / pk["hbm_gbs"]},
         "step_roofline": {"bytes_min_per_group_step": bytes_model["bytes_min"],
                           "bytes_issued_per_group_step": bytes_model["bytes_issued"],
-                          "flops_per_group_step": flops, "unique_rows_per_group_step": uniq_per_group,
-                          "ideal_us": step_t * 1e6, "achieved_us": (ms_total / args.steps / n_groups) * 1e3,
-                          "frac": step_t / ((ms_total / args.steps / n_groups) * 1e-3),
-                          "frac_of_nominal_8TBs": (bytes_model["bytes_min"] / 8e12) /
-                                                  ((ms_total / args.steps / n_groups) * 1e-3)},
+                          "executed_flops_per_group_step": flops_exec, "unique_rows_per_group_step": uniq_per_group,
+                          "bound": "hbm" if bytes_model["bytes_min"] / (pk["hbm_gbs"] * 1e9) >= tc_t else "tensor",
+                          "ideal_us": step_t * 1e6, "achieved_us": us_window, "frac": step_t * 1e6 / us_window,
+                          "frac_of_nominal_8TBs": (bytes_model["bytes_min"] / 8e12) * 1e6 / us_window},
         "device_status": {"status": st, "flags": flags},
     }
     if args.tail > 0:       # not the headline workload: the step also attends to uncompressed generated tokens
         line["config"]["tail_rows"] = args.tail
         line["config"]["workload"] += f", plus {args.tail} uncompressed tail rows per sequence"
-        line["roofline"]["traffic"] = None
-    if rank == 0 and not args.no_cpu_baseline:
-        n = args.cpu_problems or min(s.G * s.batch * s.H_kv, 32)
-        dt, np_, threads = oracle_sample(shape, wl.inputs[0], n)
-        line["cpu_baseline"] = {"value": (np_ / (s.G * s.batch * s.H_kv)) / dt, "unit": UNIT, "cores": threads,
-                                "kind": "oracle", "seconds": dt,
-                                "sample": f"{np_} of {s.G * s.batch * s.H_kv} (layer,head) problems of window 0, one step"}
+
+    # ---- the dense arm: plain decode attention over an uncompressed bf16 cache of the same shape (what SR replaces)
+    if with_dense:
+        try:
+            line["dense_attention"] = dense_arm(shape, wl, us_window, pk)
+        except Exception as e:      # the arm is a side measurement: a failure there is reported, not fatal
+            line["dense_attention"] = {"skipped": repr(e)[:200]}
+            torch.cuda.empty_cache()
+
+    # ---- the CPU oracle on the host cores (rank 0), timed on a bounded sample of window 0; the same oracle run also
+    # serves as the parity check of what was just timed (window 0, query set 0)
+    if rank == 0 and with_cpu:
+        n_all = s.G * s.batch * s.H_kv
+        n = cpu_problems or args.cpu_problems or min(n_all, 32)
+        dt, np_, cores, ores = oracle_sample(shape, wl.inputs[0], n, spread=(n < n_all))
+        line["cpu_baseline"] = {"value": (np_ / n_all) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "seconds": dt,
+                                "sample": f"{np_} of {n_all} (layer,head) problems of window 0, one step"}
+        q0 = wl.inputs[0].q[0]
+        xkv.xkv_sr_select(wl.groups[0], 0, s.G, q0, s.k, wl.sel_idx[0], wl.sel_cnt[0])
+        wl.attend(0, q0)
+        torch.cuda.synchronize()
+        line["parity"] = parity_against(shape, ores, wl.sel_idx[0].cpu().numpy(), wl.sel_cnt[0].cpu().numpy(),
+                                        wl.out[0].float().cpu().numpy(), wl.lse[0].cpu().numpy())
     wl.close()
+    del wl
+    torch.cuda.empty_cache()
+    return line
+
+
+def dense_arm(shape, wl, sr_us_window, pk):
+    """Time xkv_dense_attend (and torch's scaled_dot_product_attention beside it, as a cross-check only) on window 0's
+    shape with a synthetic uncompressed cache [G][batch][H_kv][T][d_h] for K and for V."""
+    import torch
+    from paper_2503_18893_b200 import synth, xkv
+    s = shape
+    cache_bytes = 2 * s.G * s.batch * s.H_kv * s.T * s.d_h * 2
+    free, _ = torch.cuda.mem_get_info()
+    if cache_bytes * 1.15 + (4 << 30) > free:
+        return {"skipped": f"the uncompressed cache of one window is {cache_bytes / 1e9:.1f} GB; {free / 1e9:.1f} GB are free"}
+    grp = wl.groups[0]
+    try:
+        need = xkv.xkv_dense_workspace_bytes(grp, s.T)
+    except xkv.XKVError as e:
+        return {"skipped": str(e)}
+    # the cache is drawn layer by layer and sequence by sequence (the generator works in fp32: drawing 69 GB at once
+    # would need twice that)
+    K = torch.empty((s.G, s.batch, s.H_kv, s.T, s.d_h), dtype=torch.bfloat16, device="cuda")
+    V = torch.empty_like(K)
+    for l in range(s.G):
+        for b in range(s.batch):
+            for which, dst in ((21, K), (22, V)):
+                dst[l, b] = synth.normal(synth.stream_key(s.seed, which, l, b), (s.H_kv, s.T, s.d_h), "cuda").to(torch.bfloat16)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    out = torch.empty((s.G, s.batch, s.H_q, s.d_h), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((s.G, s.batch, s.H_q), dtype=torch.float32, device="cuda")
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda") if cache_bytes < (512 << 20) else None
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    n_q = wl.n_steps
+
+    def timed(fn, n_warm=3, n=10):
+        ts = []
+        for i in range(n_warm + n):
+            if flush is not None:
+                flush.zero_()                        # caches smaller than a few L2s: flush between calls
+            a, b = ev(), ev()
+            a.record(); fn(i); b.record()
+            torch.cuda.synchronize()
+            if i >= n_warm:
+                ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts)
+
+    ours = timed(lambda i: xkv.xkv_dense_attend(grp, 0, s.G, wl.inputs[0].q[i % n_q], K, V, None, s.T, ws, out, lse))
+    res = {"kernel": "xkv_dense_attend", "us_per_window_step": ours, "cache_bytes": cache_bytes,
+           "achieved_gbs": cache_bytes / (ours * 1e-6) / 1e9, "frac_of_hbm_peak": cache_bytes / (ours * 1e-6) / 1e9 / pk["hbm_gbs"],
+           "sr_us_per_window_step": sr_us_window, "sr_speedup_over_dense": ours / sr_us_window,
+           "l2": "flushed between calls" if flush is not None else "cache larger than L2"}
+    try:
+        import torch.nn.functional as F
+
+        def sdpa(i):
+            q = wl.inputs[0].q[i % n_q]
+            for l in range(s.G):
+                F.scaled_dot_product_attention(q[l].unsqueeze(2), K[l], V[l], enable_gqa=True)
+        res["torch_sdpa_us_per_window_step"] = timed(sdpa)
+    except Exception as e:      # a cross-check only
+        res["torch_sdpa_us_per_window_step"] = None
+        res["torch_sdpa_note"] = repr(e)[:120]
+    del K, V, ws
+    torch.cuda.empty_cache()
+    return res
+
+
+def sweep_points():
+    """(label, shape) of the benchmark configurations besides the headline one and of the corner points of the
+    stress sweep (config 5: T x r x k x batch on the Llama-shaped window).  Small points get several windows, visited
+    round-robin, so that a step's inputs are several times the L2 and nothing survives in it between steps."""
+    from paper_2503_18893_b200 import synth
+    pts = [("cfg2 T=32K r=512 k=2048 B=1", synth.config(2, n_groups=4)),
+           ("cfg3 T=128K r=512 k=4096 B=1 (headline)", synth.config(3, n_groups=8)),
+           ("cfg3 T=128K r=512 k=4096 B=4", synth.config(3, batch=4, n_groups=2)),
+           ("cfg4 Qwen-shaped T=64K r=256 k=2048 B=8 n_rep=7", synth.config(4, n_groups=2)),
+           ("cfg5 T=64K r=512 k=4096 B=1 (centre)", synth.config(5, n_groups=4))]
+    for T in (16384, 262144):
+        for r in (256, 1024):
+            for k in (1024, 16384):
+                for B in (1, 16):
+                    window_bytes = B * (T * 2 * r * 2 + 4 * (T // 8) * 1024 * 2)
+                    n_groups = int(max(1, min(16, -(-(512 << 20) // window_bytes))))
+                    pts.append((f"cfg5 T={T // 1024}K r={r} k={k} B={B}",
+                                synth.config(5, T=T, r_k=r, r_v=r, k=k, batch=B, n_groups=n_groups,
+                                             seed=1005 + (T // 1024) * 7 + r * 3 + k + B)))
+    return pts
+
+
+def run_sweep(args, world, rank, local_rank, dist):
+    rows = []
+    for label, shape in sweep_points():
+        if args.sweep_filter and args.sweep_filter not in label:
+            continue
+        a = argparse.Namespace(**vars(args))
+        a.steps, a.warmup, a.repeats, a.tail = 5, 3, 0, 0
+        try:
+            line = measure_point(shape, a, world, rank, local_rank, dist, with_cpu=True, with_dense=True, cpu_problems=2)
+        except Exception as e:      # a point that does not fit or is not supported is reported, not fatal
+            line = {"config": {"workload": label}, "skipped": repr(e)[:300]}
+            import torch
+            torch.cuda.empty_cache()
+        line["point"] = label
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+        rows.append(line)
+    if rank == 0 and args.sweep_out:
+        with open(args.sweep_out, "w") as f:
+            f.write(sweep_table(rows))
+    return 0
+
+
+def sweep_table(rows) -> str:
+    out = ["| point | windows | SR us / window-step | window-steps/s | tokens/s | bytes_min MB | bound | roofline frac | "
+           "select us | attend us | dense us (ours) | dense GB/s | torch SDPA us | SR speed-up over dense | parity (idx "
+           "mismatch / max rel err) |", "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+    for r in rows:
+        if "skipped" in r:
+            out.append(f"| {r['point']} | skipped: {r['skipped']} |" + " |" * 13)
+            continue
+        sr, d = r["step_roofline"], r.get("dense_attention", {})
+        par = r.get("parity", {})
+        dense = (f"{d['us_per_window_step']:.0f} | {d['achieved_gbs']:.0f} | "
+                 f"{(d.get('torch_sdpa_us_per_window_step') or float('nan')):.0f} | {d['sr_speedup_over_dense']:.2f}"
+                 if "us_per_window_step" in d else f"{d.get('skipped', 'n/a')} | | | ")
+        out.append(f"| {r['point']} | {r['config']['windows']} | {sr['achieved_us']:.1f} | {r['value']:.0f} | "
+                   f"{r['tokens_per_s']:.0f} | {sr['bytes_min_per_group_step'] / 1e6:.1f} | {sr['bound']} | "
+                   f"{sr['frac']:.3f} | {r['select_kernel']['us_per_launch']:.1f} | {r['roofline']['us_per_launch']:.1f} | "
+                   f"{dense} | {par.get('idx_mismatch', 'n/a')} / {par.get('max_rel_err', float('nan')):.1e} |")
+    return "\n".join(out) + "\n"
+
+
+def main():
+    args = parse_args()
+    if args.op == "landmarks":
+        return run_landmarks(args)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if args.sweep:
+        rc = run_sweep(args, world, rank, local_rank, dist)
+    else:
+        line = measure_point(make_shape(args), args, world, rank, local_rank, dist,
+                             with_cpu=not args.no_cpu_baseline, with_dense=args.dense)
+        if rank == 0:
+            print(json.dumps(line))
+        rc = 0
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
-    if rank == 0:
-        print(json.dumps(line))
-    return 0
+    return rc
 
 
 if __name__ == "__main__":

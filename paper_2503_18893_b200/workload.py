@@ -80,6 +80,15 @@ def algorithmic_flops(shape: synth.SRShape) -> float:
     return 2.0 * problems * M * shape.d_h * (shape.r_k + shape.r_v)
 
 
+def executed_flops(shape: synth.SRShape) -> float:
+    """Flops the tensor-core path issues for one window-step: keys as in the paper's formula, values re-associated
+    (sum_j p_j (A_v[S_j] B_v) = (sum_j p_j A_v[S_j]) B_v): 2 M r_V n_pad for the weighted basis rows (n_pad = the
+    query heads of a KV head padded to the smallest MMA width, 16) plus 2 r_V d_h per query head for the projection."""
+    problems = shape.G * shape.H_kv * shape.batch
+    M = min(shape.k_cap, shape.T)
+    return problems * (2.0 * M * shape.d_h * shape.r_k + 2.0 * M * shape.r_v * 16 + 2.0 * shape.r_v * shape.d_h * shape.n_rep)
+
+
 class DeviceWorkload:
     """All windows of a configuration resident on one GPU, with their handles and output buffers."""
 
