@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--groups", type=int, default=None, help="number of windows (default: the config's)")
     ap.add_argument("--tail", type=int, default=0,
                     help="rows of uncompressed generated tokens attended to besides the selected rows (default none)")
+    ap.add_argument("--quant", type=int, default=0, choices=[0, 4],
+                    help="gather the token bases from b-bit round-to-nearest codes (0: bf16 bases, the headline)")
     ap.add_argument("--op", default="decode", choices=["decode", "landmarks"],
                     help="decode: the hot path (default).  landmarks: the prefill-side Algorithm 1 kernel alone "
                          "(not the headline metric; prints its own JSON line)")
@@ -325,7 +327,7 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
     s = shape
     n_q = 8
     wl = workload.DeviceWorkload(shape, n_steps=n_q, device="cuda", groups=replica_units(shape.n_groups, rank),
-                                 tail_rows=args.tail)
+                                 tail_rows=args.tail, quant_bits=getattr(args, "quant", 0))
     n_groups = len(wl.groups)
     q_bytes = n_groups * s.G * s.batch * s.H_q * s.d_h * 2
     out_bytes = q_bytes
@@ -403,7 +405,7 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
             rows = wl.sel_idx[gi][:, b_].reshape(-1)
             uniq += int(torch.unique(rows[rows >= 0]).numel())
     uniq_per_group = uniq / n_groups
-    bytes_model = workload.algorithmic_bytes(s, unique_rows=uniq_per_group)
+    bytes_model = workload.algorithmic_bytes(s, unique_rows=uniq_per_group, quant_bits=getattr(args, "quant", 0))
     flops_paper = workload.algorithmic_flops(s)
     flops_exec = workload.executed_flops(s)
     pk = peaks()
@@ -444,7 +446,7 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
         roof = {"bound": "tensor", "achieved": flops_exec / att_s / 1e12, "peak": pk["bf16_tflops_sustained"],
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    headline_shape = (shape.name == "cfg3_llama_128k" and args.tail == 0 and
+    headline_shape = (shape.name == "cfg3_llama_128k" and args.tail == 0 and not getattr(args, "quant", 0) and
                       (s.T, s.r_k, s.r_v, s.k, s.batch) == (131072, 512, 512, 4096, 1))
     roof.update({"traffic": captured_traffic("xkv_fused.cu") if headline_shape else None,
                  "kernel": "xkv_sr_reconstruct_attend (gather + reconstruct + attention)",
@@ -480,6 +482,9 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
                           "frac_of_nominal_8TBs": (bytes_model["bytes_min"] / 8e12) * 1e6 / us_window},
         "device_status": {"status": st, "flags": flags},
     }
+    if getattr(args, "quant", 0):       # not the headline workload: 4-bit bases
+        line["config"]["quant_bits"] = args.quant
+        line["config"]["workload"] += f", token bases as {args.quant}-bit RTN codes (groups of 32)"
     if args.tail > 0:       # not the headline workload: the step also attends to uncompressed generated tokens
         line["config"]["tail_rows"] = args.tail
         line["config"]["workload"] += f", plus {args.tail} uncompressed tail rows per sequence"
@@ -497,7 +502,12 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
     if rank == 0 and with_cpu:
         n_all = s.G * s.batch * s.H_kv
         n = cpu_problems or args.cpu_problems or min(n_all, 32)
-        dt, np_, cores, ores = oracle_sample(shape, wl.inputs[0], n, spread=(n < n_all))
+        oinp = wl.inputs[0]
+        if getattr(args, "quant", 0):       # the oracle works on what the codes stand for
+            oinp = workload.GroupInputs(xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_k, args.quant), args.quant),
+                                        xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_v, args.quant), args.quant),
+                                        oinp.B_k, oinp.B_v, oinp.landmarks, oinp.q)
+        dt, np_, cores, ores = oracle_sample(shape, oinp, n, spread=(n < n_all))
         line["cpu_baseline"] = {"value": (np_ / n_all) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "seconds": dt,
                                 "sample": f"{np_} of {n_all} (layer,head) problems of window 0, one step"}

@@ -172,6 +172,36 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
                                            void* out, float* lse, void* stream);
 
 /*
+ * Round-to-nearest quantisation of factors (App. "Integrate with Quantization": RTN on the compressed cache; the
+ * printed 25.7x at 4 bits is the 8.03x of the 16-bit factors times 16/5, i.e. one bit of overhead per scalar).
+ * Groups of 32 consecutive scalars of a row share a bf16 scale and a bf16 offset:
+ *   zero = bf16(min), scale = bf16((max - min)/15), code = clip(rint((x - zero)/scale), 0, 15)   (fp32, ties to even)
+ *   x_hat = bf16(code*scale + zero), the exact value rounded once.
+ * x      bf16 [rows][cols], device, 16-byte aligned; cols a multiple of 32.
+ * codes  [rows][cols/2] bytes, 16-byte aligned.  Inside every 32-bit word (scalars e0..e7) nibble k of the low half
+ *        is e_2k and nibble k of the high half is e_2k+1.
+ * meta   uint32 [rows][cols/32]: scale in the low 16 bits, offset in the high 16 bits.
+ * bits   4 (the only width with a storage format here; else UNSUPPORTED).
+ * xkv_dequantize_rtn writes x_hat (for the small per-layer matrices B, which a handle takes as bf16).
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+XKV_API int xkv_quantize_rtn(const void* x, int64_t rows, int32_t cols, int32_t bits, void* codes, void* meta, void* stream);
+XKV_API int xkv_dequantize_rtn(const void* codes, const void* meta, int64_t rows, int32_t cols, int32_t bits, void* x,
+                               void* stream);
+
+/*
+ * From now on xkv_sr_reconstruct_attend (and the _tail variant) gathers the token bases from 4-bit codes and
+ * dequantises them on the way into shared memory (Eq. 3 on x_hat); a gathered row costs r/2 + r/8 bytes instead
+ * of 2r.  The handle's A_k / A_v (which xkv_group_create then accepts as NULL) are no longer read.
+ * codes_k, meta_k  quantised A_k: [batch][T][r_k/2] bytes and uint32 [batch][T][r_k/32] (layout of xkv_quantize_rtn
+ *                  with rows = batch*T), device, BORROWED until the handle is destroyed; likewise codes_v, meta_v.
+ * bits             4; r_k and r_v must be multiples of 32.  All-NULL pointers switch back to the bf16 bases.
+ * Errors: INVALID_ARG, UNSUPPORTED (ranks, or a shape the tensor-core path does not cover).
+ */
+XKV_API int xkv_group_set_quantized_bases(xkv_group* grp, const void* codes_k, const void* meta_k, const void* codes_v,
+                                          const void* meta_v, int32_t bits);
+
+/*
  * Plain decode attention over an UNCOMPRESSED bf16 cache: out_h = softmax(scale * q_h K^T) V for the query heads of
  * every (layer, sequence, KV head).  This is the baseline that selective reconstruction is measured against (Sec. 5,
  * "Efficiency Studies": full attention reads the whole cache, SR removes the term that grows with the context); it

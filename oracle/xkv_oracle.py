@@ -435,7 +435,7 @@ def compression_ratios(N: int, W: int, L: int, d: int, r_k: int, r_v: int, c: in
 # Canonical arithmetic (fp32, IEEE, so that the codes are the same integers on every implementation):
 #   lo, hi = min, max of the group;  zero = bf16(lo);  scale = bf16((hi - lo) / (2^b - 1))
 #   code   = clip(rint((x - zero) / scale), 0, 2^b - 1)        (rint: ties to even; scale == 0 -> code 0)
-#   x_hat  = bf16(code * scale + zero)                          (code * scale is exact in fp32)
+#   x_hat  = bf16(code * scale + zero)                          (the exact value, rounded once)
 # --------------------------------------------------------------------------
 
 RTN_GROUP = 32
@@ -462,12 +462,21 @@ def rtn_quantize(X: np.ndarray, bits: int, group: int = RTN_GROUP):
     return codes.reshape(n, m), scale, zero
 
 
+def bf16_round_exact(x: np.ndarray) -> np.ndarray:
+    """Round float64 values to the nearest bf16 (8 significant bits, ties to even) in ONE step; returns float32.
+    (Going through float32 first would round twice.)  Values in the normal range of bf16 only."""
+    x = np.asarray(x, dtype=np.float64)
+    m, e = np.frexp(x)                                   # x = m * 2^e, 0.5 <= |m| < 1
+    return np.ldexp(np.rint(m * 256.0) / 256.0, e).astype(np.float32)
+
+
 def rtn_dequantize(codes: np.ndarray, scale: np.ndarray, zero: np.ndarray, group: int = RTN_GROUP) -> np.ndarray:
-    """x_hat = bf16(code * scale + zero), float32 array holding bf16 values."""
+    """x_hat = bf16(code * scale + zero): the exact value (formed in fp64, where it is exact for any realistic
+    exponent gap) rounded once.  float32 array holding bf16 values."""
     n, m = codes.shape
-    c = codes.reshape(n, m // group, group).astype(np.float32)
-    x = c * scale[:, :, None].astype(np.float32) + zero[:, :, None].astype(np.float32)   # product exact, one rounding
-    return bf16_round(x.reshape(n, m))
+    c = codes.reshape(n, m // group, group).astype(np.float64)
+    x = c * scale[:, :, None].astype(np.float64) + zero[:, :, None].astype(np.float64)
+    return bf16_round_exact(x.reshape(n, m))
 
 
 def quantized_bits_per_scalar(bits: int, group: int = RTN_GROUP, meta_bits: int = 32) -> float:

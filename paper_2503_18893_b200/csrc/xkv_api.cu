@@ -42,7 +42,8 @@ static int check_config(const xkv_group_config* c, bool need_ptrs) {
   if (!(c->softmax_scale >= 0.0f) || isinf(c->softmax_scale)) return XKV_ERR_INVALID_ARG;
   if (isnan(c->rope_base) || isinf(c->rope_base)) return XKV_ERR_INVALID_ARG;
   if (need_ptrs) {
-    if (!c->A_k || !c->A_v || !c->B_k || !c->B_v) return XKV_ERR_INVALID_ARG;
+    // A_k / A_v may be NULL: the handle then serves reconstruct+attend only after xkv_group_set_quantized_bases
+    if (!c->B_k || !c->B_v || (!c->A_k) != (!c->A_v)) return XKV_ERR_INVALID_ARG;
     const uintptr_t m = (uintptr_t)c->A_k | (uintptr_t)c->A_v | (uintptr_t)c->B_k | (uintptr_t)c->B_v |
                         (uintptr_t)c->landmarks;
     if (m & 15u) return XKV_ERR_INVALID_ARG;   // 16-byte vector loads and TMA need this
@@ -315,9 +316,11 @@ int xkv_sr_reconstruct_attend(xkv_group* g, int layer_begin, int layer_end, cons
   if (!g || !q || !sel_idx || !sel_cnt || !out) return XKV_ERR_INVALID_ARG;
   if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
   if (k_cap < 1 || k_cap > g->k_cap_max) return XKV_ERR_INVALID_ARG;
+  if (!g->dev.A_k && !g->dev.Aq_k) return XKV_ERR_INVALID_ARG;      // created without bases and none set since
   if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) ||
       ((uintptr_t)sel_cnt & 3u) || ((uintptr_t)lse & 3u))
     return XKV_ERR_INVALID_ARG;
+  if (g->dev.Aq_k && (g->attend_impl || !fused_supported(g))) return XKV_ERR_UNSUPPORTED;   // codes: tensor-core path only
   cudaError_t e = (g->attend_impl || !fused_supported(g))
                       ? launch_reconstruct_attend(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt,
                                                   k_cap, (__nv_bfloat16*)out, lse, (cudaStream_t)stream)
@@ -401,6 +404,7 @@ int xkv_sr_reconstruct_attend_tail(xkv_group* g, int layer_begin, int layer_end,
   if (layer_begin < 0 || layer_end > g->cfg.G || layer_begin >= layer_end) return XKV_ERR_INVALID_ARG;
   if (k_cap < 1 || k_cap > g->k_cap_max) return XKV_ERR_INVALID_ARG;
   if (tail_cap < 1 || tail_cap > XKV_TAIL_MAX_ROWS) return XKV_ERR_INVALID_ARG;
+  if (!g->dev.A_k && !g->dev.Aq_k) return XKV_ERR_INVALID_ARG;
   if (workspace_bytes < (uint64_t)tail_part_floats(g, tail_cap) * sizeof(float)) return XKV_ERR_INVALID_ARG;
   if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)sel_idx & 3u) || ((uintptr_t)sel_cnt & 3u) ||
       ((uintptr_t)lse & 3u) || ((uintptr_t)tail_k & 15u) || ((uintptr_t)tail_v & 15u) || ((uintptr_t)tail_len & 3u) ||
@@ -414,6 +418,45 @@ int xkv_sr_reconstruct_attend_tail(xkv_group* g, int layer_begin, int layer_end,
     e = launch_fused(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt, k_cap, (__nv_bfloat16*)out,
                      lse, s, TailParts{(const float*)workspace, tail_splits(tail_cap)});
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+static int check_rtn_args(const void* a, const void* b, const void* c3, int64_t rows, int32_t cols, int32_t bits) {
+  if (!a || !b || !c3 || rows < 0 || cols < 32 || cols % 32 != 0) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)a & 15u) || ((uintptr_t)b & 15u) || ((uintptr_t)c3 & 15u)) return XKV_ERR_INVALID_ARG;
+  if (bits != 4) return (bits >= 1 && bits <= 8) ? XKV_ERR_UNSUPPORTED : XKV_ERR_INVALID_ARG;
+  return XKV_OK;
+}
+
+int xkv_quantize_rtn(const void* x, int64_t rows, int32_t cols, int32_t bits, void* codes, void* meta, void* stream) {
+  const int st = check_rtn_args(x, codes, meta, rows, cols, bits);
+  if (st != XKV_OK) return st;
+  cudaError_t e = launch_quantize_rtn4((const __nv_bfloat16*)x, rows, cols, codes, meta, (cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+int xkv_dequantize_rtn(const void* codes, const void* meta, int64_t rows, int32_t cols, int32_t bits, void* x, void* stream) {
+  const int st = check_rtn_args(codes, meta, x, rows, cols, bits);
+  if (st != XKV_OK) return st;
+  cudaError_t e = launch_dequantize_rtn4(codes, meta, rows, cols, (__nv_bfloat16*)x, (cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+int xkv_group_set_quantized_bases(xkv_group* g, const void* codes_k, const void* meta_k, const void* codes_v,
+                                  const void* meta_v, int32_t bits) {
+  if (!g) return XKV_ERR_INVALID_ARG;
+  if (!codes_k && !meta_k && !codes_v && !meta_v) {
+    g->dev.Aq_k = g->dev.Aq_v = nullptr; g->dev.Am_k = g->dev.Am_v = nullptr;
+    return XKV_OK;
+  }
+  if (!codes_k || !meta_k || !codes_v || !meta_v) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)codes_k | (uintptr_t)meta_k | (uintptr_t)codes_v | (uintptr_t)meta_v) & 15u) return XKV_ERR_INVALID_ARG;
+  if (bits != 4) return (bits >= 1 && bits <= 8) ? XKV_ERR_UNSUPPORTED : XKV_ERR_INVALID_ARG;
+  if (g->cfg.r_k % 32 != 0 || g->cfg.r_v % 32 != 0 || !fused_supported(g)) return XKV_ERR_UNSUPPORTED;
+  g->dev.Aq_k = (const uint8_t*)codes_k; g->dev.Am_k = (const uint32_t*)meta_k;
+  g->dev.Aq_v = (const uint8_t*)codes_v; g->dev.Am_v = (const uint32_t*)meta_v;
   return XKV_OK;
 }
 

@@ -216,7 +216,9 @@ __host__ __device__ constexpr int ring_slots() {
 
 // NR: query heads per KV head rounded up to 4, 8 or 16.  WB: most 128-column blocks of r_v (registers of the
 // value epilogue): NR * WB <= 64.
-template <int DH, int NR, int WB, bool PROF>
+// QUANT: the token bases are gathered from 4-bit codes (xkv_group_set_quantized_bases) and dequantised by the
+// producer warps on their way into the rings.
+template <int DH, int NR, int WB, bool PROF, bool QUANT>
 __global__ void __launch_bounds__(kThreads, 1)
 sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched sc, const __nv_bfloat16* __restrict__ q,
                 const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt) {
@@ -400,6 +402,73 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         if (slot == RS) slot = 0;
       }
     };
+    // The same phase from 4-bit codes.  Four consecutive lanes share a tile row: lane q4 fetches the 16 bytes of
+    // codes and the scale/offset word of one 32-column group of the slot pair (64 contiguous bytes per row and
+    // request), turns them into 32 bf16 values (packed arithmetic, one rounding) and stores them as four 16-byte
+    // units of the swizzled slab; a stream's 64 threads cover 16 rows per pass, 8 passes per pair.  The loads of a
+    // pair are issued before the wait for the pair's release, so their latency overlaps it.
+    const uint32_t q4 = (uint32_t)(t64 & 3), rq = (uint32_t)(t64 >> 2);
+    auto issue_phase_q = [&](const uint32_t (&rw)[8], int b) {
+      const uint8_t* Cb = (kstream ? dev.Aq_k : dev.Aq_v) + (size_t)b * dev.T * (size_t)(r >> 1);
+      const uint32_t* Mb = (kstream ? dev.Am_k : dev.Am_v) + (size_t)b * dev.T * (size_t)(r >> 5);
+      const uint32_t ring_q = base + (kstream ? 0u : (uint32_t)SK * kSlabBytes);
+      auto fetch = [&](int ks, uint4 (&cw)[8], uint32_t (&mw)[8]) {
+        const int col0 = ks * 64 + (int)q4 * 32;           // first column of this lane's group
+        const bool in = col0 < r;                          // false in a padding slab: zeros are stored
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          cw[i] = in ? __ldg(reinterpret_cast<const uint4*>(Cb + (size_t)rw[i] * (size_t)(r >> 1) + (col0 >> 1))) : make_uint4(0, 0, 0, 0);
+          mw[i] = in ? __ldg(Mb + (size_t)rw[i] * (size_t)(r >> 5) + (col0 >> 5)) : 0u;
+        }
+      };
+      auto store = [&](const uint4 (&cw)[8], const uint32_t (&mw)[8]) -> bool {
+        const int pr = slot >> 1;
+        const uint32_t bit = 1u << pr;
+        if (used & bit) {             // wait for the release of the pair's previous occupant
+          if (!wait_bar(ctx, BAR(bar_empty + pr), (rel_par >> pr) & 1u, ps + 3)) { ok = false; return false; }
+          rel_par ^= bit;
+        }
+        used |= bit;
+        // this lane's group lies in slab (q4 >> 1) of the pair, 16-byte units 4*(q4 & 1) .. +3 of the 128-byte row
+        const uint32_t st = ring_q + (uint32_t)(slot + (int)(q4 >> 1)) * kSlabBytes;
+        const uint32_t u0 = (q4 & 1u) * 4u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint32_t j = rq + 16u * (uint32_t)i;       // tile row
+          const uint32_t w[4] = {cw[i].x, cw[i].y, cw[i].z, cw[i].w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint32_t o[4];
+            dequant_word(w[u], mw[i], o);
+            const uint32_t a = st + j * 128u + (((u0 + (uint32_t)u) ^ (j & 7u)) << 4);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          }
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");   // the staged rotary rows of this tile (key stream) have landed too
+        fence_proxy_async();                               // the tensor core reads these stores
+        mbar_arrive(BAR(bar_full + slot));                 // both slabs of the pair are complete when all 64 threads are done
+        mbar_arrive(BAR(bar_full + slot + 1));
+        slot += 2;
+        if (slot == RS) slot = 0;
+        return true;
+      };
+      // (a second register set, so that the next pair's loads are in flight while this pair is converted, was
+      // measured and lost: 103 us against 85 us per call at the headline size)
+      uint4 ca[8];
+      uint32_t ma[8];
+#pragma unroll 1
+      for (int ks = 0; ks < nst; ks += 2) {
+        fetch(ks, ca, ma);
+        if (!store(ca, ma)) return;
+      }
+    };
+    auto load_rows_q = [&](uint32_t (&rw)[8]) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int p = pos_s[pb * kTile + (int)rq + 16 * i];
+        rw[i] = p < 0 ? 0u : (uint32_t)p;
+      }
+    };
     auto load_rows = [&](uint32_t (&ro)[16]) {             // rows without a selected token read row 0 (weight 0)
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
@@ -465,10 +534,17 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         mbar_arrive(BAR(bl.posfull + pb));
       }
       if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
-      uint32_t ro[16];
-      load_rows(ro);
-      if (!kstream) mbar_arrive(BAR(bl.vfree + pb));       // this thread is done with the position buffer
-      issue_phase(ro, cur.b);
+      if constexpr (QUANT) {
+        uint32_t rw[8];
+        load_rows_q(rw);
+        if (!kstream) mbar_arrive(BAR(bl.vfree + pb));     // this thread is done with the position buffer
+        issue_phase_q(rw, cur.b);
+      } else {
+        uint32_t ro[16];
+        load_rows(ro);
+        if (!kstream) mbar_arrive(BAR(bl.vfree + pb));     // this thread is done with the position buffer
+        issue_phase(ro, cur.b);
+      }
       ++it;
       if (++pb == 4) pb = 0;
     }
@@ -1005,13 +1081,18 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   memcpy(&mk, grp->bk_tmap, sizeof(mk));
   cudaError_t e;
   if (grp->prof) {     // the variant with the diagnostic counters compiled in
-    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, true>>(smem, grp->device);
+    if (dev.Aq_k) return cudaErrorNotSupported;        // no diagnostic variant of the quantised gather
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, true, false>>(smem, grp->device);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(sr_fused_kernel<DH, NR, WB, true>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, true, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+  } else if (dev.Aq_k) {
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, true>>(smem, grp->device);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, true>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   } else {
-    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false>>(smem, grp->device);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, false>>(smem, grp->device);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   }
   count_launch(kFamFused);
   if (e != cudaSuccess) return e;

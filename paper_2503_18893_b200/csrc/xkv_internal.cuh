@@ -40,6 +40,10 @@ struct GroupDev {
   unsigned int* flags;              // device flag word
   const int32_t* outliers;          // [G][batch][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
   int n_out;
+  const uint8_t* Aq_k;              // 4-bit codes of A_k [batch][T][r_k/2], or nullptr (then the bf16 bases are gathered)
+  const uint8_t* Aq_v;              // [batch][T][r_v/2]
+  const uint32_t* Am_k;             // scale/offset words [batch][T][r_k/32]
+  const uint32_t* Am_v;             // [batch][T][r_v/32]
   int lm_const;                     // 1: the landmarks do not change while the handle lives (loads may run ahead of the stream)
   unsigned int inject;              // XKV_INJECT_* bits (xkv_debug_set_fault_injection); 0 in normal use
 };
@@ -151,6 +155,11 @@ size_t tail_part_floats(const xkv_group* grp, int tail_cap);
 cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __nv_bfloat16* q, const __nv_bfloat16* tail_k,
                                  const __nv_bfloat16* tail_v, const int32_t* tail_len, int tail_cap, float* part,
                                  cudaStream_t s);
+
+// xkv_quant.cu
+cudaError_t launch_quantize_rtn4(const __nv_bfloat16* x, long long rows, int cols, void* codes, void* meta, cudaStream_t s);
+cudaError_t launch_dequantize_rtn4(const void* codes, const void* meta, long long rows, int cols, __nv_bfloat16* x,
+                                   cudaStream_t s);
 
 // xkv_fused.cu
 int fused_slots(const xkv_group* grp);

@@ -169,6 +169,23 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// Eight 4-bit codes of one 32-bit word -> eight bf16 values in four registers of two (the first of a pair in the low
+// half): x = code * scale + zero with ONE rounding of the exact value.  Code layout: (word >> 4k) & 0x000F000F is the
+// pair (e_2k, e_2k+1); meta holds the bf16 scale in its low half and the bf16 offset in its high half.
+// 0x4300 | n is the bf16 number 128 + n; subtracting 128 is exact, and the packed fused multiply-add rounds once.
+__device__ __forceinline__ void dequant_word(uint32_t w, uint32_t meta, uint32_t* out4) {
+  const uint32_t s2 = __byte_perm(meta, meta, 0x1010);
+  const uint32_t z2 = __byte_perm(meta, meta, 0x3232);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t biased = ((w >> (4 * k)) & 0x000F000Fu) | 0x43004300u;
+    uint32_t n, x;
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(n) : "r"(biased), "r"(0x43004300u));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(x) : "r"(n), "r"(s2), "r"(z2));
+    out4[k] = x;
+  }
+}
+
 // Programmatic dependent launch: block until the kernel this one depends on has completed and flushed its writes
 // (a no-op when the kernel was not launched with the programmatic-serialization attribute).
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

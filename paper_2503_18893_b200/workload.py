@@ -53,7 +53,7 @@ def make_group_inputs(shape: synth.SRShape, group: int = 0, n_steps: int = 1, de
     return GroupInputs(A_k, A_v, B_k, B_v, lm, q)
 
 
-def algorithmic_bytes(shape: synth.SRShape, unique_rows=None) -> dict:
+def algorithmic_bytes(shape: synth.SRShape, unique_rows=None, quant_bits: int = 0) -> dict:
     """Bytes one window-step has to move (bf16 storage), per term.
 
     landmarks: every landmark is read once;  rows_issued: every selected row of A_k and A_v;
@@ -63,10 +63,12 @@ def algorithmic_bytes(shape: synth.SRShape, unique_rows=None) -> dict:
     problems = shape.G * shape.H_kv * shape.batch
     M = min(shape.k_cap, shape.T)
     lm = shape.batch * shape.G * shape.n_c * shape.d * 2
-    issued = problems * M * (shape.r_k + shape.r_v) * 2
+    # bytes per stored scalar of a basis row: 2 (bf16), or (b + 1)/8 with b-bit codes and their scale/offset words
+    bps = 2.0 if not quant_bits else (quant_bits + 1) / 8.0
+    issued = problems * M * (shape.r_k + shape.r_v) * bps
     if unique_rows is None:
         unique_rows = shape.batch * min(shape.G * shape.H_kv * M, shape.T)
-    uniq = unique_rows * (shape.r_k + shape.r_v) * 2
+    uniq = unique_rows * (shape.r_k + shape.r_v) * bps
     Bm = shape.batch * shape.G * (shape.r_k + shape.r_v) * shape.d * 2
     small = shape.G * shape.batch * shape.H_q * shape.d_h * 2 * 2 + problems * (M + 1) * 4 * 2
     return {"landmarks": lm, "rows_issued": issued, "rows_unique": uniq, "B": Bm, "small": small,
@@ -92,7 +94,8 @@ def executed_flops(shape: synth.SRShape) -> float:
 class DeviceWorkload:
     """All windows of a configuration resident on one GPU, with their handles and output buffers."""
 
-    def __init__(self, shape: synth.SRShape, n_steps: int = 4, device="cuda", groups=None, tail_rows: int = 0):
+    def __init__(self, shape: synth.SRShape, n_steps: int = 4, device="cuda", groups=None, tail_rows: int = 0,
+                 quant_bits: int = 0):
         from . import xkv  # loads the CUDA library; raises if it is not built
         self.xkv = xkv
         self.shape = shape
@@ -104,6 +107,10 @@ class DeviceWorkload:
             inp = make_group_inputs(shape, gi, n_steps, device)
             grp = xkv.create_from_tensors(inp.A_k, inp.A_v, inp.B_k, inp.B_v, inp.landmarks, H_kv=shape.H_kv,
                                           H_q=shape.H_q, k_max=shape.k, chunk=shape.c, rope_base=shape.rope_base)
+            if quant_bits:      # the token bases as b-bit codes (App. "Integrate with Quantization"), made by the library
+                ck, mk = xkv.xkv_quantize_rtn(inp.A_k, quant_bits)
+                cv, mv = xkv.xkv_quantize_rtn(inp.A_v, quant_bits)
+                xkv.xkv_group_set_quantized_bases(grp, ck, mk, cv, mv, quant_bits)
             self.inputs.append(inp)
             self.groups.append(grp)
         n = len(self.groups)

@@ -82,6 +82,12 @@ _lib.xkv_dense_workspace_bytes.restype = ctypes.c_int
 _lib.xkv_dense_attend.argtypes = [_P, ctypes.c_int, ctypes.c_int, _P, _P, _P, _P, ctypes.c_int32, _P, ctypes.c_uint64,
                                   _P, _P, _P]
 _lib.xkv_dense_attend.restype = ctypes.c_int
+_lib.xkv_quantize_rtn.argtypes = [_P, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _P, _P, _P]
+_lib.xkv_quantize_rtn.restype = ctypes.c_int
+_lib.xkv_dequantize_rtn.argtypes = [_P, _P, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _P, _P]
+_lib.xkv_dequantize_rtn.restype = ctypes.c_int
+_lib.xkv_group_set_quantized_bases.argtypes = [_P, _P, _P, _P, _P, ctypes.c_int32]
+_lib.xkv_group_set_quantized_bases.restype = ctypes.c_int
 XKV_DENSE_MAX_ROWS = 1 << 22
 XKV_TAIL_MAX_ROWS = 32768
 
@@ -282,6 +288,37 @@ def xkv_sr_reconstruct_attend_tail(grp: Group, layer_begin: int, layer_end: int,
                                              _ptr(out), _ptr(lse), _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_sr_reconstruct_attend_tail")
+
+
+def xkv_quantize_rtn(x, bits: int = 4, stream=None):
+    """RTN-quantise a bf16 device tensor [..., cols] along its last axis in groups of 32 (include/xkv.h).
+    Returns (codes uint8 [..., cols/2], meta int32 [..., cols/32]) device tensors."""
+    cols = x.shape[-1]
+    rows = x.numel() // cols
+    codes = torch.empty(x.shape[:-1] + (cols // 2,), dtype=torch.uint8, device=x.device)
+    meta = torch.empty(x.shape[:-1] + (cols // 32,), dtype=torch.int32, device=x.device)
+    st = _lib.xkv_quantize_rtn(_ptr(x), rows, cols, bits, _ptr(codes), _ptr(meta), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_quantize_rtn")
+    return codes, meta
+
+
+def xkv_dequantize_rtn(codes, meta, bits: int = 4, stream=None):
+    """bf16 tensor [..., cols] of the dequantised values x_hat."""
+    cols = codes.shape[-1] * 2
+    rows = codes.numel() // (cols // 2)
+    x = torch.empty(codes.shape[:-1] + (cols,), dtype=torch.bfloat16, device=codes.device)
+    st = _lib.xkv_dequantize_rtn(_ptr(codes), _ptr(meta), rows, cols, bits, _ptr(x), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_dequantize_rtn")
+    return x
+
+
+def xkv_group_set_quantized_bases(grp: Group, codes_k, meta_k, codes_v, meta_v, bits: int = 4) -> None:
+    st = _lib.xkv_group_set_quantized_bases(grp.handle, _ptr(codes_k), _ptr(meta_k), _ptr(codes_v), _ptr(meta_v), bits)
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_group_set_quantized_bases")
+    grp.quantized = (codes_k, meta_k, codes_v, meta_v)      # keep the borrowed tensors alive with the handle
 
 
 def xkv_dense_workspace_bytes(grp: Group, cap: int) -> int:

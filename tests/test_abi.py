@@ -62,6 +62,11 @@ def test_create_rejects_null_and_misaligned_pointers(xkv):
     with pytest.raises(xkv.XKVError) as e:                       # all factor pointers NULL
         xkv.xkv_group_create(cfg, stream=0)
     assert e.value.status == xkv.XKV_ERR_INVALID_ARG
+    cfg.B_k = cfg.B_v = 0x1000
+    cfg.A_k = 0x1000                                             # one basis without the other
+    with pytest.raises(xkv.XKVError) as e:
+        xkv.xkv_group_create(cfg, stream=0)
+    assert e.value.status == xkv.XKV_ERR_INVALID_ARG
     cfg.A_k = cfg.A_v = cfg.B_k = cfg.B_v = 0x1000
     cfg.A_v = 0x1008                                             # not 16-byte aligned
     with pytest.raises(xkv.XKVError) as e:
@@ -112,3 +117,12 @@ def test_budgets_that_overflow_32_bit_strides_are_rejected_on_the_host(xkv):
 def test_launch_counters_by_family(xkv):
     c = xkv.xkv_debug_launch_counts()
     assert set(c) == set(xkv.XKV_KERNEL_FAMILIES) and sum(c.values()) == xkv.xkv_kernel_launch_count()
+
+
+def test_quantisation_entry_points_check_their_arguments_on_the_host(xkv):
+    L = xkv._lib
+    assert L.xkv_quantize_rtn(0x1000, 4, 48, 4, 0x2000, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG      # cols % 32
+    assert L.xkv_quantize_rtn(0x1000, 4, 64, 3, 0x2000, 0x3000, None) == xkv.XKV_ERR_UNSUPPORTED      # no 3-bit format
+    assert L.xkv_quantize_rtn(0x1000, 4, 64, 9, 0x2000, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG
+    assert L.xkv_dequantize_rtn(0x1008, 0x2000, 4, 64, 4, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG    # alignment
+    assert L.xkv_group_set_quantized_bases(None, None, None, None, None, 4) == xkv.XKV_ERR_INVALID_ARG

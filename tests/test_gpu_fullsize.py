@@ -144,3 +144,27 @@ def test_config3_window_with_an_8192_row_uncompressed_tail():
         shares.append(np.exp(lse_sr - lse))
     assert 0.01 < float(np.median(np.concatenate(shares))) < 0.99          # both parts matter
     g.close()
+
+
+def test_config3_window_from_4bit_bases():
+    """The headline window with the token bases as 4-bit round-to-nearest codes (App. "Integrate with
+    Quantization"): sampled problems against the oracle on the dequantised bases."""
+    from paper_2503_18893_b200 import xkv
+    s = synth.config(3, n_groups=1)
+    inp = workload.make_group_inputs(s, 0, 1, "cuda")
+    g = C.GpuCase(s, inp)
+    ck, mk = xkv.xkv_quantize_rtn(g.inp.A_k)
+    cv, mv = xkv.xkv_quantize_rtn(g.inp.A_v)
+    xkv.xkv_group_set_quantized_bases(g.grp, ck, mk, cv, mv)
+    gidx, gcnt = g.select(0)
+    gout, glse = g.attend(gidx, gcnt, 0)
+    assert g.status() == (0, 0)
+    deq = workload.GroupInputs(xkv.xkv_dequantize_rtn(ck, mk), xkv.xkv_dequantize_rtn(cv, mv), inp.B_k, inp.B_v,
+                               inp.landmarks, inp.q)          # bit-equal to the oracle's dequantiser (tests/test_gpu_quant.py)
+    cache = {}
+    for (l, b, hk) in [(0, 0, 1), (2, 0, 6), (3, 0, 3)]:
+        o, lse = _oracle_attend(s, deq, l, b, hk, gidx[l, b, hk, :gcnt[l, b, hk]], 0, cache)
+        hs = slice(hk * s.n_rep, (hk + 1) * s.n_rep)
+        assert C.rel_err(gout[l, b, hs], o) <= TOL, (l, b, hk)
+        np.testing.assert_allclose(glse[l, b, hs], lse, atol=2e-2)
+    g.close()

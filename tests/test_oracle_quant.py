@@ -74,3 +74,13 @@ def test_stored_bits_and_printed_ratios():
     assert O.quantized_bits_per_scalar(4) == 5.0 and O.quantized_bits_per_scalar(3) == 4.0
     assert abs(O.quantized_compression_ratio(8.03, 4) - 25.70) < 0.0075      # the paper's xKV-4bit row
     assert abs(O.quantized_compression_ratio(8.03, 3) - 32.12) < 0.0075      # the paper's xKV-3bit row
+
+
+def test_single_step_bf16_rounding_matches_the_two_step_routine_where_both_are_exact():
+    # on float32 inputs whose low 16 bits hold no sticky information beyond bit 15 the two roundings agree;
+    # on a constructed double-rounding case they differ and the single-step routine is the correct one
+    x = _bf16_matrix(8, 8, 5).astype(np.float64) * (1.0 + 2.0 ** -10)          # not bf16 values any more
+    assert np.array_equal(O.bf16_round_exact(x), O.bf16_round(x.astype(np.float32)))
+    tricky = 1.0 + 2.0 ** -8 + 2.0 ** -40          # just above the tie between 1 and 1 + 2^-7: must round up
+    assert O.bf16_round_exact(np.array([tricky]))[0] == np.float32(1.0 + 2.0 ** -7)
+    assert O.bf16_round(np.array([tricky], dtype=np.float32))[0] == np.float32(1.0)   # float32 first lands on the tie
