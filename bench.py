@@ -50,7 +50,7 @@ def parse_args():
                     help="rows of uncompressed generated tokens attended to besides the selected rows (default none)")
     ap.add_argument("--quant", type=int, default=0, choices=[0, 4],
                     help="gather the token bases from b-bit round-to-nearest codes (0: bf16 bases, the headline)")
-    ap.add_argument("--op", default="decode", choices=["decode", "landmarks"],
+    ap.add_argument("--op", default="decode", choices=["decode", "landmarks", "clf"],
                     help="decode: the hot path (default).  landmarks: the prefill-side Algorithm 1 kernel alone "
                          "(not the headline metric; prints its own JSON line)")
     ap.add_argument("--repeats", type=int, default=0,
@@ -315,6 +315,56 @@ def run_landmarks(args):
                       "achieved_gbs_landmarks_only": key_bytes / (res["landmarks_only"] * 1e-3) / 1e9,
                       "frac_of_hbm_peak": key_bytes / (res["landmarks_only"] * 1e-3) / 1e9 / pk["hbm_gbs"],
                       "peak_source": pk["source"]}))
+    return 0
+
+
+def run_clf(args):
+    """Times xkv_clf_factorize (Eq. 1 by randomised SVD) on the raw key cache of one window and one sequence of the
+    workload's shape, and compares its residual with the optimum (eigenvalues of the fp64 Gram matrix, by torch on
+    the GPU: a harness cross-check).  Not the headline metric; prints its own JSON line."""
+    import torch
+    from paper_2503_18893_b200 import synth, xkv
+    torch.cuda.set_device(0)
+    s = make_shape(args)
+    K, _ = synth.make_kv(s, device="cuda")                                          # (G, T, d) bf16
+    X = torch.cat([K[l] for l in range(s.G)], dim=1).contiguous()
+    del K
+    r, q, p = s.r_k, 2, 32
+    cfg = xkv.make_clf_config(T=s.T, G=s.G, d=s.d, r=r, oversample=p, power_iters=q)
+    l = xkv.xkv_clf_rank_l(cfg)
+    omega = synth.normal(synth.stream_key(s.seed, 31), (s.G * s.d, l), "cuda").to(torch.bfloat16)
+    ws = torch.empty(xkv.xkv_clf_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    A = torch.empty((s.T, r), dtype=torch.bfloat16, device="cuda")
+    B = torch.empty((s.G, r, s.d), dtype=torch.bfloat16, device="cuda")
+    sig = torch.empty(r, dtype=torch.float32, device="cuda")
+    ts = []
+    for i in range(args.warmup + args.steps):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); xkv.xkv_clf_factorize(cfg, X, omega, ws, A, B, sig); e1.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            ts.append(e0.elapsed_time(e1))
+    st, flags = xkv.xkv_clf_status(ws)
+    # residual against the optimum
+    N = s.G * s.d
+    gram = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+    for t0 in range(0, s.T, 16384):
+        xb = X[t0:t0 + 16384].double()
+        gram += xb.T @ xb
+    ev = torch.linalg.eigvalsh(gram).flip(0).clamp_min(0)
+    optimum = float(ev[r:].sum())
+    Vm = torch.cat([B[g] for g in range(s.G)], dim=1).double()                      # (r, N)
+    res = 0.0
+    for t0 in range(0, s.T, 16384):
+        res += float(((X[t0:t0 + 16384].double() - A[t0:t0 + 16384].double() @ Vm) ** 2).sum())
+    ms = statistics.median(ts)
+    tall_flops = (2 * (q + 2) + 1) * 2.0 * s.T * N * l                              # 2 products per iteration + A
+    print(json.dumps({"op": "xkv_clf_factorize", "config": f"T={s.T}, G={s.G}, d={s.d} (X is {s.T} x {N}), r={r}, "
+                      f"oversample={p} (l={l}), power_iters={q}", "ms": ms, "tall_product_tflops": tall_flops / (ms * 1e-3) / 1e12,
+                      "residual_over_optimum": res / optimum, "relative_residual": res / float(ev.sum()),
+                      "orthonormality_max_dev": float((Vm @ Vm.T - torch.eye(r, device="cuda", dtype=torch.float64)).abs().max()),
+                      "sigma_max_rel_err": float(((sig.double() - ev[:r].sqrt()).abs() / ev[0].sqrt()).max()),
+                      "status": st, "flags": flags}))
     return 0
 
 
@@ -655,6 +705,8 @@ def main():
     args = parse_args()
     if args.op == "landmarks":
         return run_landmarks(args)
+    if args.op == "clf":
+        return run_clf(args)
     if args.impl == "reference":
         return run_reference(args)
 

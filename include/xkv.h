@@ -59,6 +59,7 @@ typedef enum {
 /* Bits of the device flag word returned by xkv_group_status. */
 #define XKV_FLAG_INDEX_RANGE 1u
 #define XKV_FLAG_TIMEOUT 2u
+#define XKV_FLAG_CLF_BREAKDOWN 4u /* xkv_clf_factorize: a Cholesky pivot was not positive (reported by xkv_clf_status) */
 
 /*
  * Problem statement for one window (names follow the paper; T is its L, G its W).
@@ -170,6 +171,42 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
                                            const void* tail_k, const void* tail_v, const int32_t* tail_len,
                                            int32_t tail_cap, void* workspace, uint64_t workspace_bytes,
                                            void* out, float* lse, void* stream);
+
+/*
+ * Cross-layer factorisation on the GPU (Sec. 3.1, Eq. 1): for one sequence and one cache (keys or values), the
+ * rank-r factors A = U Sigma (T x r) and B_l (r x d per layer) of X = [X_l0 ... X_l0+G-1] (T x G d), by the
+ * randomised SVD the paper describes for prefill (App. "Custom SVD Kernel": power iterations as 16-bit tensor-core
+ * matrix products, shifted Cholesky QR instead of Householder QR).  Steps: Z <- omega; (power_iters + 1) times
+ * Y = X Z, U = X^T Y, Z = orth(U) (three passes of Cholesky QR with a relative diagonal shift, fp32); then the
+ * Rayleigh-Ritz step on span(Z): M = Z^T X^T X Z = P Lambda P^T (Jacobi), V = Z P_r, B = V^T rounded to bf16,
+ * A = X bf16(V), sigma = sqrt(Lambda).  The result approximates the optimum of Eq. 1 (it is not unique up to signs and
+ * rotations inside equal singular values: compare residuals, never factors).
+ * cfg       host struct: T rows, G layers, d columns per layer (G*d a multiple of 64), rank r (multiple of 8),
+ *           oversample p (0 means 32; l = r + p rounded up to a multiple of 64, at most G*d), power_iters q (0..8).
+ * X         bf16 [T][G*d] (the layers' caches side by side, layer l in columns l*d .. l*d+d-1), device, 16-byte aligned.
+ * omega     bf16 [G*d][l] random test matrix drawn by the caller (standard normal), device; l from xkv_clf_rank_l.
+ * workspace device scratch of at least xkv_clf_workspace_bytes(cfg) bytes, 256-byte aligned, caller-owned.
+ * A         out bf16 [T][r];  B out bf16 [G][r][d] (the layout of xkv_group_config.B_k for one sequence);
+ * sigma     out fp32 [r], optional.
+ * The call allocates nothing and enqueues everything on `stream`.  xkv_clf_status (after the caller has synchronised,
+ * or blocking on `stream`) reads the flag word of the workspace: XKV_FLAG_TIMEOUT, XKV_FLAG_CLF_BREAKDOWN.
+ * Errors: INVALID_ARG, UNSUPPORTED (l too large for the eigen-solver: l <= 2048), ARCH, CUDA.
+ */
+typedef struct {
+  uint32_t struct_size; /* sizeof(xkv_clf_config) */
+  int32_t T, G, d, r;
+  int32_t oversample;   /* p; 0 means 32 */
+  int32_t power_iters;  /* q */
+} xkv_clf_config;
+XKV_API int xkv_clf_rank_l(const xkv_clf_config* cfg, int32_t* l);
+XKV_API int xkv_clf_workspace_bytes(const xkv_clf_config* cfg, uint64_t* bytes);
+XKV_API int xkv_clf_factorize(const xkv_clf_config* cfg, const void* X, const void* omega, void* workspace,
+                              uint64_t workspace_bytes, void* A, void* B, float* sigma, void* stream);
+XKV_API int xkv_clf_status(const void* workspace, uint32_t* flags, void* stream);
+/* Diagnostic: the tensor-core product of the factorisation alone, C (M x N, fp32) = A B^T for A bf16 [K][M] and
+ * B bf16 [N][K] (M, K multiples of 8); flags: one device word (XKV_FLAG_TIMEOUT). */
+XKV_API int xkv_debug_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, float* C, uint32_t* flags,
+                           void* stream);
 
 /*
  * Round-to-nearest quantisation of factors (App. "Integrate with Quantization": RTN on the compressed cache; the
@@ -292,7 +329,8 @@ XKV_API uint64_t xkv_kernel_launch_count(void);
 #define XKV_KERNEL_LANDMARKS 7 /* Algorithm 1 */
 #define XKV_KERNEL_PREP 8      /* handle set-up: repacking, rotary tables */
 #define XKV_KERNEL_DENSE 9     /* merge of dense-attention partials (xkv_dense_attend) */
-#define XKV_KERNEL_FAMILIES 10
+#define XKV_KERNEL_CLF 10      /* cross-layer factorisation (xkv_clf_factorize) */
+#define XKV_KERNEL_FAMILIES 11
 XKV_API int xkv_debug_launch_counts(uint64_t* counts);
 
 /*

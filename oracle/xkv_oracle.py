@@ -487,3 +487,54 @@ def quantized_bits_per_scalar(bits: int, group: int = RTN_GROUP, meta_bits: int 
 def quantized_compression_ratio(base_ratio: float, bits: int, group: int = RTN_GROUP) -> float:
     """Compression of a 16-bit factorised cache of ratio `base_ratio` after RTN quantisation of every factor."""
     return base_ratio * 16.0 / quantized_bits_per_scalar(bits, group)
+
+
+# --------------------------------------------------------------------------
+# Randomised cross-layer factorisation  (App. "Custom SVD Kernel": randomised SVD, 16-bit matrix products in the
+# power iterations, shifted Cholesky QR instead of Householder QR)
+#
+# The paper names the ingredients, not the steps.  The steps taken here are the textbook randomised subspace
+# iteration (Halko, Martinsson, Tropp) run on the right side, because X (T x N, N = G d) is tall:
+#   Z <- Omega (N x l, l = r + p);  repeat q + 1 times: Y = X Z; U = X^T Y; Z = orth(U)
+#   Rayleigh-Ritz on span(Z): M = Z^T X^T X Z = P Lambda P^T; V = Z P_r; B = V^T; A = X bf16(V); sigma = sqrt(Lambda).
+# orth = shifted Cholesky QR: G = U^T U + s I, s = shift * max diag(U^T U), G = L L^T, U <- U L^-T, in passes with
+# relative shifts 1e-4, 1e-5 (inside the iteration) and 1e-4, 1e-5, 1e-6, 1e-8, 1e-10 (last iterate).  Matrices that the 16-bit products read are rounded to bf16 first (X is bf16 already).
+# It approximates clf_factorize's optimum; it is compared with it through the residual, never factor by factor.
+# --------------------------------------------------------------------------
+
+
+CHOLQR_SHIFTS = (1e-4, 1e-5, 1e-6, 1e-8, 1e-10)
+
+
+def cholesky_qr(U: np.ndarray, shifts=CHOLQR_SHIFTS) -> np.ndarray:
+    """Orthonormalise the columns of U (n x l) by repeated shifted Cholesky QR (fp64 here); one pass per entry of
+    `shifts` (each relative to the largest diagonal entry of the Gram matrix of that pass)."""
+    Z = np.asarray(U, dtype=np.float64)
+    for shift_rel in shifts:
+        Gm = Z.T @ Z
+        Gm = Gm + shift_rel * Gm.diagonal().max() * np.eye(Gm.shape[0])
+        L = np.linalg.cholesky(Gm)
+        Z = np.linalg.solve(L, Z.T).T                       # Z L^-T
+    return Z
+
+
+def clf_randomized(X_cat: np.ndarray, r: int, omega: np.ndarray, power_iters: int = 2):
+    """Rank-r factorisation of X_cat (T x N, bf16 values) from the test matrix omega (N x l, bf16 values, l >= r).
+    Returns A (T x r), V (N x r) with B = V^T, sigma (r,); A and V hold bf16 values (float32 arrays)."""
+    X = np.asarray(X_cat, dtype=np.float64)
+    Z = np.asarray(omega, dtype=np.float64)
+    for it in range(power_iters + 1):
+        Y = bf16_round((X @ bf16_round(Z.astype(np.float32)).astype(np.float64)).astype(np.float32)).astype(np.float64)
+        U = X.T @ Y
+        # inside the iteration the iterate only has to stay well conditioned (two passes); the last one has to be
+        # orthonormal (five passes, decreasing shifts)
+        Z = cholesky_qr(U, CHOLQR_SHIFTS if it == power_iters else CHOLQR_SHIFTS[:2])
+    Zb = bf16_round(Z.astype(np.float32)).astype(np.float64)
+    W = bf16_round((X @ Zb).astype(np.float32)).astype(np.float64)
+    M = Z.T @ (X.T @ W)
+    M = 0.5 * (M + M.T)
+    lam, P = np.linalg.eigh(M)
+    order = np.argsort(-lam)[:r]
+    V = bf16_round((Z @ P[:, order]).astype(np.float32))
+    A = bf16_round((X @ V.astype(np.float64)).astype(np.float32))
+    return A, V, np.sqrt(np.maximum(lam[order], 0.0))

@@ -82,6 +82,20 @@ static bool encode_rows64(void* out, const void* base, uint64_t rows, uint64_t c
   return r == CUDA_SUCCESS;
 }
 
+// 2-D bf16 tensor [rows][cols] with a row pitch of `pitch` elements, box = box_rows x 64 columns, 128-byte swizzle.
+bool encode_bf16_map(void* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols) {
   return encode_rows64(out, base, rows, cols, kLandmarkBoxRows);
 }
@@ -417,6 +431,66 @@ int xkv_sr_reconstruct_attend_tail(xkv_group* g, int layer_begin, int layer_end,
   if (e == cudaSuccess)
     e = launch_fused(g, layer_begin, layer_end, (const __nv_bfloat16*)q, sel_idx, sel_cnt, k_cap, (__nv_bfloat16*)out,
                      lse, s, TailParts{(const float*)workspace, tail_splits(tail_cap)});
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+static int current_sm100_device(int* device) {
+  int major = 0;
+  cudaError_t e = cudaGetDevice(device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, *device);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return major == 10 ? XKV_OK : XKV_ERR_ARCH;
+}
+
+int xkv_clf_rank_l(const xkv_clf_config* cfg, int32_t* l) {
+  if (!l) return XKV_ERR_INVALID_ARG;
+  int v = 0;
+  const int st = clf_rank_l(cfg, &v);
+  if (st == XKV_OK) *l = v;
+  return st;
+}
+
+int xkv_clf_workspace_bytes(const xkv_clf_config* cfg, uint64_t* bytes) {
+  if (!bytes) return XKV_ERR_INVALID_ARG;
+  return clf_workspace_bytes(cfg, bytes);
+}
+
+int xkv_clf_factorize(const xkv_clf_config* cfg, const void* X, const void* omega, void* workspace,
+                      uint64_t workspace_bytes, void* A, void* B, float* sigma, void* stream) {
+  if (!X || !omega || !workspace || !A || !B) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)X & 15u) || ((uintptr_t)omega & 15u) || ((uintptr_t)workspace & 255u) || ((uintptr_t)A & 15u) ||
+      ((uintptr_t)B & 15u) || ((uintptr_t)sigma & 3u))
+    return XKV_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  int st = clf_workspace_bytes(cfg, &need);                  // also validates cfg
+  if (st != XKV_OK) return st;
+  if (workspace_bytes < need) return XKV_ERR_INVALID_ARG;
+  int device = 0;
+  st = current_sm100_device(&device);
+  if (st != XKV_OK) return st;
+  return clf_factorize(cfg, X, omega, workspace, workspace_bytes, A, B, sigma, device, (cudaStream_t)stream);
+}
+
+int xkv_clf_status(const void* workspace, uint32_t* flags, void* stream) {
+  if (!workspace) return XKV_ERR_INVALID_ARG;
+  unsigned int f = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(&f, workspace, sizeof(f), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) { set_cuda_error(e); return XKV_ERR_CUDA; }
+  if (flags) *flags = f;
+  if (f & XKV_FLAG_TIMEOUT) return XKV_ERR_TIMEOUT;
+  return XKV_OK;
+}
+
+int xkv_debug_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K, float* C, uint32_t* flags, void* stream) {
+  if (!a || !b || !C || !flags || M < 1 || N < 1 || K < 1 || (M % 8) || (K % 8)) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)a & 15u) || ((uintptr_t)b & 15u) || ((uintptr_t)C & 3u)) return XKV_ERR_INVALID_ARG;
+  int device = 0;
+  const int st = current_sm100_device(&device);
+  if (st != XKV_OK) return st;
+  cudaError_t e = clf_gemm(a, b, M, N, K, C, flags, device, (cudaStream_t)stream);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }

@@ -1,0 +1,656 @@
+// Cross-layer factorisation on the GPU (Sec. 3.1, Eq. 1; App. "Custom SVD Kernel": a randomised SVD whose power
+// iterations are 16-bit tensor-core matrix products and whose orthogonalisation is a shifted Cholesky QR).
+//
+// X = [X_l0 ... X_l0+G-1] (T x N, N = G d, bf16) is tall, so the iteration runs on the right side.  With l = r + p:
+//   Z (N x l) <- the random test matrix
+//   repeat q + 1 times:   Y^T = Z^T X^T   (l x T, bf16)          tensor core
+//                         U   = X^T Y     (N x l, fp32)          tensor core
+//                         Z   = U R^-1,  R^T R = U^T U + shift I (shifted Cholesky QR in fp64: two passes inside the
+//                               iteration, five for the last iterate, which has to be orthonormal)
+//   Rayleigh-Ritz:        W^T = Z^T X^T,  U' = X^T W,  M = Z^T U' (= Z^T X^T X Z, l x l),  M = P Lambda P^T (Jacobi)
+//   V = Z P_r (N x r);    B_l = rows of V^T (bf16);   A = X V_bf16 (T x r, tensor core);   sigma = sqrt(Lambda).
+// A = U Sigma and B = V^T of the truncated SVD of X, up to the accuracy of the subspace (checked against the exact
+// optimum sum_{i>r} sigma_i^2, never factor by factor: signs and degenerate subspaces are not unique).
+//
+// One tensor-core kernel serves the three tall products.  It computes C (M x N) = A B^T for A given as [K][M]
+// row-major (an MN-major operand: the M index is contiguous) and B as [N][K] row-major (K-major), the two operand
+// forms the fused decode kernel already uses, so no matrix is ever transposed in memory:
+//   Y^T = Z-as-A (K = N_x)  x  X-as-B;     U = X-as-A (K = T)  x  Y^T-as-B;     A^T = V-as-A  x  X-as-B (stored transposed).
+#include <cuda.h>
+#include <math.h>
+
+#include "xkv_internal.cuh"
+#include "xkv_ptx.cuh"
+
+namespace xkv {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kGemmThreads = 192;                 // warps 0-3 epilogue, 4 TMA producer, 5 MMA issue
+constexpr int kGemmStages = 6;
+constexpr int kGemmStageBytes = 32768;            // A: two slabs of [64 k][64 m] (8 KB each); B: [128 n][64 k] (16 KB)
+constexpr uint32_t kGemmWaitLimit = 1u << 24;
+
+__device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kGemmWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+
+// C[m][n] = sum_k A[k][m] B[n][k].  grid = (ceil(N/128), ceil(M/128)).  TRANS: store C^T (out[n][m]).
+// Out-of-range rows and columns of the operands are zero-filled by the copy engine; stores are guarded.
+template <bool TRANS>
+__global__ void __launch_bounds__(kGemmThreads)
+clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int M, int N, int K,
+                float* __restrict__ Cf, __nv_bfloat16* __restrict__ Cb, long long ldc, unsigned int* __restrict__ flags) {
+  extern __shared__ uint8_t gemm_smem[];
+  __shared__ __align__(8) uint64_t bars[2 * kGemmStages + 1];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_s;
+  const uint32_t base = (smem_u32(gemm_smem) + 1023u) & ~1023u;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n0 = blockIdx.x * 128, m0 = blockIdx.y * 128;
+  const int KB = (K + 63) / 64;
+  const uint32_t bar0 = smem_u32(bars);
+  auto FULL = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+  auto EMPTY = [&](int s) { return bar0 + 8u * (uint32_t)(kGemmStages + s); };
+  const uint32_t ACC = bar0 + 8u * (uint32_t)(2 * kGemmStages);
+  if (tid == 0) {
+    for (int s = 0; s < kGemmStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
+    mbar_init(ACC, 1);
+    abort_s = 0;
+    fence_mbar_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(smem_u32(&tmem_slot), 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  bool ok = true;
+  if (warp == 4) {
+    if (lane == 0) {
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % kGemmStages;
+        if (kb >= kGemmStages && !gemm_wait(EMPTY(s), (uint32_t)((kb / kGemmStages - 1) & 1))) { ok = false; break; }
+        const uint32_t st = base + (uint32_t)s * kGemmStageBytes;
+        mbar_expect_tx(FULL(s), kGemmStageBytes);
+        tma_load_2d(st, &map_a, m0, kb * 64, FULL(s));                 // A: columns m0..m0+63, rows (k) kb*64..+63
+        tma_load_2d(st + 8192, &map_a, m0 + 64, kb * 64, FULL(s));     //    columns m0+64..m0+127
+        tma_load_2d(st + 16384, &map_b, kb * 64, n0, FULL(s));         // B: columns (k) kb*64..+63, rows n0..n0+127
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
+      constexpr uint32_t idesc = idesc_bf16_f32(128, 128) | (1u << 15);   // A is read along its rows (MN-major)
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % kGemmStages;
+        if (!gemm_wait(FULL(s), (uint32_t)((kb / kGemmStages) & 1))) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t st = base + (uint32_t)s * kGemmStageBytes;
+        // A: two 64-column slabs 8192 bytes apart, 8-row groups (along k) 1024 bytes apart; 16 k-rows per step
+        const uint32_t a_lo = ((uint32_t)((st & 0x3FFFFu) >> 4)) | ((uint32_t)(8192 >> 4) << 16);
+        const uint32_t b_lo = (uint32_t)(smem_desc_sw128(st + 16384, 0) & 0xFFFFFFFFull);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_bf16(tmem, desc_hi | (a_lo + (uint32_t)kk * (2048u >> 4)), desc_hi | (b_lo + 2u * (uint32_t)kk), idesc,
+                      (kb | kk) ? 1u : 0u);
+        tc_commit(EMPTY(s));
+      }
+      tc_commit(ACC);
+    }
+  }
+  if (warp >= 4) {                  // a producer or issuer that gave up tells the epilogue not to wait for ever
+    if (!ok && lane == 0) { abort_s = 1; atomicOr(flags, XKV_FLAG_TIMEOUT); }
+  } else {
+    // ---- epilogue: thread = accumulator lane = row m0 + tid
+    bool done = false;
+    for (uint32_t i = 0; i < kGemmWaitLimit && !done; ++i) {
+      done = mbar_try_wait(ACC, 0);
+      if (!done && (i & 1023u) == 1023u && *(volatile int*)&abort_s) break;
+    }
+    if (done) {
+      tc_fence_after();
+      const int m = m0 + tid;
+      const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+#pragma unroll 1
+      for (int cb = 0; cb < 4; ++cb) {
+        float v[32];
+        tmem_ld32(tmem + lane_base + (uint32_t)(cb * 32), v);
+        tc_wait_ld();
+        if (m < M) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int n = n0 + cb * 32 + i;
+            if (n < N) {
+              const long long at = TRANS ? (long long)n * ldc + m : (long long)m * ldc + n;
+              if (Cf) Cf[at] = v[i];
+              if (Cb) Cb[at] = __float2bfloat16(v[i]);
+            }
+          }
+        }
+      }
+    } else if (tid == 0) {
+      atomicOr(flags, XKV_FLAG_TIMEOUT);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// The small matrices (l x l, N x l) in fp32 on the ordinary cores.
+namespace {
+
+// C (m x n, ldc) = op(A) B with B (k x n, ldb) row-major and op(A) = A^T for A (k x m, lda) if TA, else A (m x k, lda).
+// 64 x 64 tiles, 256 threads, 4 x 4 outputs per thread.
+// TO = double accumulates in double (the Gram matrices of the Cholesky QR, whose condition number is the square of
+// the iterate's).
+template <bool TA, typename TO>
+__global__ void __launch_bounds__(256)
+sgemm_small_kernel(const float* __restrict__ A, const float* __restrict__ B, TO* __restrict__ C, int m, int n, int k,
+                   int lda, int ldb, int ldc) {
+  __shared__ float As[16][64 + 4], Bs[16][64 + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  TO acc[4][4] = {};
+  for (int k0 = 0; k0 < k; k0 += 16) {
+    for (int i = tid; i < 16 * 64; i += 256) {
+      const int kk = TA ? i / 64 : i % 16, mm = TA ? i % 64 : i / 16;
+      const int gk = k0 + kk, gm = m0 + mm;
+      As[kk][mm] = (gk < k && gm < m) ? (TA ? A[(size_t)gk * lda + gm] : A[(size_t)gm * lda + gk]) : 0.0f;
+      const int bk = i / 64, bn = i % 64;
+      Bs[bk][bn] = (k0 + bk < k && n0 + bn < n) ? B[(size_t)(k0 + bk) * ldb + n0 + bn] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += (TO)a[i] * (TO)b[j];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gm = m0 + ty * 4 + i, gn = n0 + tx * 4 + j;
+      if (gm < m && gn < n) C[(size_t)gm * ldc + gn] = acc[i][j];
+    }
+}
+
+// Blocked Cholesky factorisation (fp64) of the symmetric l x l matrix G + shift_rel * max_diag(G) * I, lower factor in
+// place, in panels of 32 columns: factor the diagonal block, solve the panel below it, update the trailing matrix.
+constexpr int kCholNb = 32;
+
+__global__ void __launch_bounds__(1024)
+chol_shift_kernel(double* __restrict__ G, int l, double shift_rel) {
+  __shared__ double red[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  double mx = 0.0;
+  for (int i = tid; i < l; i += 1024) mx = fmax(mx, G[(size_t)i * l + i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) red[warp] = mx;
+  __syncthreads();
+  mx = red[lane];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  for (int i = tid; i < l; i += 1024) G[(size_t)i * l + i] += shift_rel * mx;
+}
+
+// Diagonal block [kb, kb+nb): unblocked factorisation in shared memory (one CTA of 32 x 32 threads).  A pivot that
+// is not positive (breakdown) is replaced by a tiny one and reported in flags.
+__global__ void __launch_bounds__(1024)
+chol_diag_kernel(double* __restrict__ G, int l, int kb, int nb, unsigned int* __restrict__ flags) {
+  __shared__ double a[kCholNb][kCholNb + 1];
+  const int i = threadIdx.y, j = threadIdx.x;
+  a[i][j] = (i < nb && j < nb) ? G[(size_t)(kb + i) * l + kb + j] : (i == j ? 1.0 : 0.0);
+  __syncthreads();
+  for (int c = 0; c < nb; ++c) {
+    if (i == c && j == c) {
+      double d = a[c][c];
+      if (!(d > 0.0)) { atomicOr(flags, XKV_FLAG_CLF_BREAKDOWN); d = 1e-300; }
+      a[c][c] = sqrt(d);
+    }
+    __syncthreads();
+    if (j == c && i > c) a[i][c] /= a[c][c];
+    __syncthreads();
+    if (j > c && i >= j) a[i][j] -= a[i][c] * a[j][c];
+    __syncthreads();
+  }
+  if (i < nb && j < nb && j <= i) G[(size_t)(kb + i) * l + kb + j] = a[i][j];
+}
+
+// Panel below the diagonal block: row i of L21 solves x L11^T = A21[i] (one thread per row).
+__global__ void __launch_bounds__(128)
+chol_panel_kernel(double* __restrict__ G, int l, int kb, int nb) {
+  __shared__ double L11[kCholNb][kCholNb + 1];
+  for (int e = threadIdx.x; e < kCholNb * kCholNb; e += 128) {
+    const int r = e / kCholNb, c = e % kCholNb;
+    L11[r][c] = (r < nb && c <= r) ? G[(size_t)(kb + r) * l + kb + c] : 0.0;
+  }
+  __syncthreads();
+  const int i = kb + nb + blockIdx.x * 128 + threadIdx.x;
+  if (i >= l) return;
+  double x[kCholNb];
+  double* row = G + (size_t)i * l + kb;
+#pragma unroll
+  for (int c = 0; c < kCholNb; ++c) x[c] = c < nb ? row[c] : 0.0;
+#pragma unroll
+  for (int c = 0; c < kCholNb; ++c) {
+    if (c < nb) {
+      double v = x[c];
+#pragma unroll
+      for (int t = 0; t < kCholNb; ++t) if (t < c) v -= x[t] * L11[c][t];
+      x[c] = v / L11[c][c];
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < kCholNb; ++c) if (c < nb) row[c] = x[c];
+}
+
+// Trailing update of the lower triangle: G[i][k] -= sum_t L21[i][t] L21[k][t]; one 32 x 32 tile per CTA.
+__global__ void __launch_bounds__(1024)
+chol_update_kernel(double* __restrict__ G, int l, int kb, int nb) {
+  if (blockIdx.x > blockIdx.y) return;                                 // upper triangle: not needed
+  __shared__ double Li[kCholNb][kCholNb + 1], Lk[kCholNb][kCholNb + 1];
+  const int t0 = kb + nb;
+  const int i = t0 + blockIdx.y * kCholNb + threadIdx.y, k = t0 + blockIdx.x * kCholNb + threadIdx.x;
+  const int ii = t0 + blockIdx.y * kCholNb + threadIdx.x;              // the row this thread loads for the tiles
+  const int kk = t0 + blockIdx.x * kCholNb + threadIdx.x;
+  // thread (y, x) loads element (row x of the tile, column y of the panel)
+  Li[threadIdx.x][threadIdx.y] = (ii < l && threadIdx.y < nb) ? G[(size_t)ii * l + kb + threadIdx.y] : 0.0;
+  Lk[threadIdx.x][threadIdx.y] = (kk < l && threadIdx.y < nb) ? G[(size_t)kk * l + kb + threadIdx.y] : 0.0;
+  __syncthreads();
+  if (i < l && k <= i) {
+    double acc = 0.0;
+#pragma unroll
+    for (int t = 0; t < kCholNb; ++t) acc += Li[threadIdx.y][t] * Lk[threadIdx.x][t];
+    G[(size_t)i * l + k] -= acc;
+  }
+}
+
+// Z (n x l) = U L^-T for the lower factor L: row by row, z_j = (u_j - sum_{i<j} z_i L[j][i]) / L[j][j] (fp64).  One warp
+// per row; the row lives in shared memory.  Also writes the bf16 copy the tensor-core products read.
+constexpr int kSolveWarps = 4;
+__global__ void __launch_bounds__(kSolveWarps * 32)
+trsolve_rows_kernel(const float* __restrict__ U, const double* __restrict__ L, float* __restrict__ Z,
+                    __nv_bfloat16* __restrict__ Zb, int n, int l) {
+  extern __shared__ double zrow[];                   // [kSolveWarps][l]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row = blockIdx.x * kSolveWarps + warp;
+  if (row >= n) return;
+  double* z = zrow + (size_t)warp * l;
+  for (int j = lane; j < l; j += 32) z[j] = (double)U[(size_t)row * l + j];
+  __syncwarp();
+  for (int j = 0; j < l; ++j) {
+    const double* Lj = L + (size_t)j * l;
+    double s = 0.0;
+    for (int i = lane; i < j; i += 32) s += z[i] * Lj[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) z[j] = (z[j] - s) / Lj[j];
+    __syncwarp();
+  }
+  for (int j = lane; j < l; j += 32) {
+    Z[(size_t)row * l + j] = (float)z[j];
+    if (Zb) Zb[(size_t)row * l + j] = __float2bfloat16((float)z[j]);
+  }
+}
+
+}  // namespace
+
+namespace {
+
+// Eigen-decomposition of the symmetric l x l matrix M by cyclic Jacobi rotations in the round-robin (tournament)
+// order: every round rotates l/2 disjoint index pairs at once, as three kernels (the rotations of the round; columns
+// p, q of M and of P for every row; rows p, q of M for every column) so that the work of a round spreads over
+// the SMs.  A check per sweep sets *done once the off-diagonal weight is below working precision; every kernel
+// returns at once after that.  On return the eigenvalues are on the diagonal of M, the eigenvectors the columns of P.
+constexpr int kJacobiMaxPairs = 1024;
+constexpr int kJacobiSweeps = 12;
+
+__global__ void jacobi_init_kernel(float* __restrict__ P, int l, int* __restrict__ done) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e == 0) *done = 0;
+  if (e < l * l) P[e] = (e / l == e % l) ? 1.0f : 0.0f;
+}
+
+__global__ void __launch_bounds__(1024)
+jacobi_check_kernel(const float* __restrict__ M, int l, int* __restrict__ done) {
+  __shared__ float red[64];
+  if (*done) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float off = 0.0f, all = 0.0f;
+  for (int e = tid; e < l * l; e += 1024) {
+    const float v = M[e];
+    all += v * v;
+    if (e / l != e % l) off += v * v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { off += __shfl_xor_sync(0xffffffffu, off, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
+  if (lane == 0) { red[warp] = off; red[32 + warp] = all; }
+  __syncthreads();
+  if (tid == 0) {
+    float o2 = 0.0f, a2 = 0.0f;
+    for (int w = 0; w < 32; ++w) { o2 += red[w]; a2 += red[32 + w]; }
+    if (o2 <= 1e-13f * a2) *done = 1;
+  }
+}
+
+__global__ void jacobi_rot_kernel(const float* __restrict__ M, int l, int t, float2* __restrict__ cs, int2* __restrict__ pq,
+                                  const int* __restrict__ done) {
+  if (*done) return;
+  const int n = (l + 1) & ~1, np = n / 2;
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= np) return;
+  int p, q;
+  if (k == 0) { p = n - 1; q = t; }
+  else { p = (t + k) % (n - 1); q = (t - k + n - 1) % (n - 1); }
+  if (p > q) { const int x = p; p = q; q = x; }
+  float c = 1.0f, s = 0.0f;
+  if (q < l) {
+    const float app = M[(size_t)p * l + p], aqq = M[(size_t)q * l + q], apq = M[(size_t)p * l + q];
+    if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * sqrtf(fabsf(app * aqq))) {
+      const float tau = (aqq - app) / (2.0f * apq);
+      const float tt = (tau >= 0.0f ? 1.0f : -1.0f) / (fabsf(tau) + sqrtf(1.0f + tau * tau));
+      c = rsqrtf(1.0f + tt * tt);
+      s = tt * c;
+    }
+  } else {
+    q = -1;                                           // the padding index: nothing to rotate
+  }
+  cs[k] = make_float2(c, s);
+  pq[k] = make_int2(p, q);
+}
+
+// columns p, q of M and of P, every row
+__global__ void jacobi_cols_kernel(float* __restrict__ M, float* __restrict__ P, int l, const float2* __restrict__ cs,
+                                   const int2* __restrict__ pq, const int* __restrict__ done) {
+  if (*done) return;
+  const int np = ((l + 1) & ~1) / 2;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= l * np) return;
+  const int i = e / np, k = e - i * np;
+  const int2 ix = pq[k];
+  const float2 r = cs[k];
+  if (ix.y < 0 || r.y == 0.0f) return;
+  float* row = M + (size_t)i * l;
+  const float x = row[ix.x], y = row[ix.y];
+  row[ix.x] = r.x * x - r.y * y;
+  row[ix.y] = r.y * x + r.x * y;
+  float* prow = P + (size_t)i * l;
+  const float u = prow[ix.x], v = prow[ix.y];
+  prow[ix.x] = r.x * u - r.y * v;
+  prow[ix.y] = r.y * u + r.x * v;
+}
+
+// rows p, q of M, every column
+__global__ void jacobi_rows_kernel(float* __restrict__ M, int l, const float2* __restrict__ cs, const int2* __restrict__ pq,
+                                   const int* __restrict__ done) {
+  if (*done) return;
+  const int np = ((l + 1) & ~1) / 2;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= np * l) return;
+  const int k = e / l, j = e - k * l;
+  const int2 ix = pq[k];
+  const float2 r = cs[k];
+  if (ix.y < 0 || r.y == 0.0f) return;
+  const float x = M[(size_t)ix.x * l + j], y = M[(size_t)ix.y * l + j];
+  M[(size_t)ix.x * l + j] = r.x * x - r.y * y;
+  M[(size_t)ix.y * l + j] = r.y * x + r.x * y;
+}
+
+// The r largest eigenvalues (ties to the lower index) and their eigenvectors as the columns of Psel (l x r);
+// sigma = sqrt(lambda).
+__global__ void __launch_bounds__(1024)
+eig_select_kernel(const float* __restrict__ M, const float* __restrict__ P, int l, int r, float* __restrict__ Psel,
+                  float* __restrict__ sigma) {
+  extern __shared__ int rank_s[];                      // [l]
+  const int tid = threadIdx.x;
+  for (int i = tid; i < l; i += 1024) {
+    const float li = M[(size_t)i * l + i];
+    int rk = 0;
+    for (int j = 0; j < l; ++j) {
+      const float lj = M[(size_t)j * l + j];
+      rk += (lj > li || (lj == li && j < i)) ? 1 : 0;
+    }
+    rank_s[i] = rk;
+    if (rk < r && sigma) sigma[rk] = sqrtf(fmaxf(li, 0.0f));
+  }
+  __syncthreads();
+  for (int e = tid; e < l * l; e += 1024) {
+    const int row = e / l, i = e % l;
+    const int rk = rank_s[i];
+    if (rk < r) Psel[(size_t)row * r + rk] = P[e];
+  }
+}
+
+// V (N x r, fp32) -> its bf16 copy and the per-layer matrices B [G][r][d], B[g][m][j] = V[g d + j][m].
+__global__ void clf_finish_kernel(const float* __restrict__ V, int G, int d, int r, __nv_bfloat16* __restrict__ Vb,
+                                  __nv_bfloat16* __restrict__ B) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)G * d * r;
+  if (idx >= total) return;
+  const int m = (int)(idx % r);
+  const long long row = idx / r;                       // g d + j
+  const int g = (int)(row / d), j = (int)(row % d);
+  const __nv_bfloat16 v = __float2bfloat16(V[idx]);
+  Vb[idx] = v;
+  B[((size_t)g * r + m) * d + j] = v;
+}
+
+}  // namespace
+
+namespace {
+
+__global__ void symmetrize_kernel(float* __restrict__ M, int l) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= l * l) return;
+  const int i = e / l, j = e % l;
+  if (i < j) {
+    const float v = 0.5f * (M[(size_t)i * l + j] + M[(size_t)j * l + i]);
+    M[(size_t)i * l + j] = v;
+    M[(size_t)j * l + i] = v;
+  }
+}
+
+struct ClfPlan {
+  int T, Tp, N, r, l, q;
+  size_t off_flags, off_zb, off_yt, off_u, off_z, off_g, off_m, off_p, off_ps, off_v, off_vb, off_cs, off_pq, total;
+};
+
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+bool make_plan(const xkv_clf_config* c, ClfPlan* p) {
+  p->T = c->T; p->Tp = (c->T + 7) & ~7; p->N = c->G * c->d; p->r = c->r; p->q = c->power_iters;
+  const int over = c->oversample > 0 ? c->oversample : 32;
+  p->l = (c->r + over + 63) & ~63;
+  if (p->l > p->N) p->l = p->N & ~63;
+  if (p->l < c->r || p->l < 64 || p->l / 2 > kJacobiMaxPairs) return false;
+  size_t o = 0;
+  p->off_flags = o; o = align_up(o + 256);
+  p->off_zb = o; o = align_up(o + (size_t)p->N * p->l * 2);
+  p->off_yt = o; o = align_up(o + (size_t)p->l * p->Tp * 2);
+  p->off_u = o; o = align_up(o + (size_t)p->N * p->l * 4);
+  p->off_z = o; o = align_up(o + (size_t)p->N * p->l * 4);
+  p->off_g = o; o = align_up(o + (size_t)p->l * p->l * 8);      // the Gram matrix / Cholesky factor, fp64
+  p->off_m = o; o = align_up(o + (size_t)p->l * p->l * 4);
+  p->off_p = o; o = align_up(o + (size_t)p->l * p->l * 4);
+  p->off_ps = o; o = align_up(o + (size_t)p->l * p->r * 4);
+  p->off_v = o; o = align_up(o + (size_t)p->N * p->r * 4);
+  p->off_vb = o; o = align_up(o + (size_t)p->N * p->r * 2);
+  p->off_cs = o; o = align_up(o + (size_t)kJacobiMaxPairs * 8);
+  p->off_pq = o; o = align_up(o + (size_t)kJacobiMaxPairs * 8);
+  p->total = o;
+  return true;
+}
+
+int check_clf_config(const xkv_clf_config* c) {
+  if (!c || c->struct_size != sizeof(xkv_clf_config)) return XKV_ERR_INVALID_ARG;
+  if (c->T < 1 || c->T >= (1 << 24) || c->G < 1 || c->d < 8 || c->r < 8 || c->power_iters < 0 || c->power_iters > 8 ||
+      c->oversample < 0)
+    return XKV_ERR_INVALID_ARG;
+  if (c->r % 8 || (c->G * (long long)c->d) % 64 || c->G * (long long)c->d > (1 << 20)) return XKV_ERR_INVALID_ARG;
+  if (c->r > c->G * c->d) return XKV_ERR_INVALID_ARG;
+  return XKV_OK;
+}
+
+template <bool TRANS>
+cudaError_t launch_gemm(const void* a, int a_rows_k, int a_cols_m, int a_pitch, const void* b, int b_rows_n, int b_cols_k,
+                        int b_pitch, float* Cf, __nv_bfloat16* Cb, long long ldc, unsigned int* flags, int device,
+                        cudaStream_t s) {
+  CUtensorMap ma, mb;
+  if (!encode_bf16_map(&ma, a, (uint64_t)a_rows_k, (uint64_t)a_cols_m, (uint64_t)a_pitch, 64) ||
+      !encode_bf16_map(&mb, b, (uint64_t)b_rows_n, (uint64_t)b_cols_k, (uint64_t)b_pitch, 128))
+    return cudaErrorInvalidValue;
+  const size_t smem = 1024 + (size_t)kGemmStages * kGemmStageBytes;
+  cudaError_t e = ensure_dyn_smem<clf_gemm_kernel<TRANS>>(smem, device);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((b_rows_n + 127) / 128, (a_cols_m + 127) / 128);
+  clf_gemm_kernel<TRANS><<<grid, kGemmThreads, smem, s>>>(ma, mb, a_cols_m, b_rows_n, a_rows_k, Cf, Cb, ldc, flags);
+  count_launch(kFamClf);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int clf_rank_l(const xkv_clf_config* c, int* l) {
+  int st = check_clf_config(c);
+  if (st != XKV_OK) return st;
+  ClfPlan p;
+  if (!make_plan(c, &p)) return XKV_ERR_UNSUPPORTED;
+  *l = p.l;
+  return XKV_OK;
+}
+
+int clf_workspace_bytes(const xkv_clf_config* c, uint64_t* bytes) {
+  int st = check_clf_config(c);
+  if (st != XKV_OK) return st;
+  ClfPlan p;
+  if (!make_plan(c, &p)) return XKV_ERR_UNSUPPORTED;
+  *bytes = p.total;
+  return XKV_OK;
+}
+
+// Debug/test entry of the tensor-core product alone: C (M x N, fp32) = A B^T, A bf16 [K][M], B bf16 [N][K].
+cudaError_t clf_gemm(const void* a, const void* b, int M, int N, int K, float* C, unsigned int* flags, int device, cudaStream_t s) {
+  return launch_gemm<false>(a, K, M, M, b, N, K, K, C, nullptr, N, flags, device, s);
+}
+
+int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, void* workspace, uint64_t workspace_bytes,
+                  void* A_out, void* B_out, float* sigma, int device, cudaStream_t s) {
+  int st = check_clf_config(c);
+  if (st != XKV_OK) return st;
+  ClfPlan p;
+  if (!make_plan(c, &p)) return XKV_ERR_UNSUPPORTED;
+  if (workspace_bytes < p.total) return XKV_ERR_INVALID_ARG;
+  uint8_t* w = (uint8_t*)workspace;
+  unsigned int* flags = (unsigned int*)(w + p.off_flags);
+  __nv_bfloat16* Zb = (__nv_bfloat16*)(w + p.off_zb);
+  __nv_bfloat16* Yt = (__nv_bfloat16*)(w + p.off_yt);
+  float* U = (float*)(w + p.off_u);
+  float* Z = (float*)(w + p.off_z);
+  double* Gm = (double*)(w + p.off_g);
+  float2* jcs = (float2*)(w + p.off_cs);
+  int2* jpq = (int2*)(w + p.off_pq);
+  int* jdone = (int*)(flags + 1);
+  float* Mm = (float*)(w + p.off_m);
+  float* Pm = (float*)(w + p.off_p);
+  float* Ps = (float*)(w + p.off_ps);
+  float* V = (float*)(w + p.off_v);
+  __nv_bfloat16* Vb = (__nv_bfloat16*)(w + p.off_vb);
+  const int N = p.N, l = p.l, r = p.r, T = p.T;
+  cudaError_t e = cudaMemsetAsync(flags, 0, 256, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(Zb, omega, (size_t)N * l * 2, cudaMemcpyDeviceToDevice, s);
+  const dim3 g_ll((l + 63) / 64, (l + 63) / 64);
+  // Y^T = Z^T X^T  then  U = X^T Y
+  auto two_products = [&]() -> cudaError_t {
+    cudaError_t e2 = launch_gemm<false>(Zb, N, l, l, X, T, N, N, nullptr, Yt, p.Tp, flags, device, s);
+    if (e2 != cudaSuccess) return e2;
+    return launch_gemm<false>(X, T, N, N, Yt, l, T, p.Tp, U, nullptr, l, flags, device, s);
+  };
+  // Z = orth(src) by three passes of shifted Cholesky QR.  The Gram matrix is accumulated, factorised and solved
+  // in fp64: its condition number is the square of the iterate's, which after a multiplication by X^T X spans the
+  // whole range between the largest singular value and the noise floor.
+  const size_t solve_smem = (size_t)kSolveWarps * l * sizeof(double);
+  e = e == cudaSuccess ? ensure_dyn_smem<trsolve_rows_kernel>(solve_smem, device) : e;
+  // Every pass divides the condition number by about shift^-1/2; the iterate of a power iteration only has to stay
+  // well conditioned (two passes), the last one has to be orthonormal (five passes with decreasing shifts: the
+  // columns of U that lie in the noise floor are 10^8 times smaller than the leading ones).
+  static const double kShifts[5] = {1e-4, 1e-5, 1e-6, 1e-8, 1e-10};
+  auto cholqr = [&](const float* src, int passes) -> cudaError_t {
+    for (int pass = 0; pass < passes; ++pass) {
+      const float* in = pass == 0 ? src : Z;
+      sgemm_small_kernel<true, double><<<g_ll, 256, 0, s>>>(in, in, Gm, l, l, N, l, l, l);
+      const double shift_rel = kShifts[pass];
+      chol_shift_kernel<<<1, 1024, 0, s>>>(Gm, l, shift_rel);
+      int launches = 2;
+      for (int kb = 0; kb < l; kb += kCholNb) {
+        const int nb = l - kb < kCholNb ? l - kb : kCholNb;
+        chol_diag_kernel<<<1, dim3(kCholNb, kCholNb), 0, s>>>(Gm, l, kb, nb, flags);
+        const int rem = l - kb - nb;
+        ++launches;
+        if (rem > 0) {
+          chol_panel_kernel<<<(rem + 127) / 128, 128, 0, s>>>(Gm, l, kb, nb);
+          const int tiles = (rem + kCholNb - 1) / kCholNb;
+          chol_update_kernel<<<dim3(tiles, tiles), dim3(kCholNb, kCholNb), 0, s>>>(Gm, l, kb, nb);
+          launches += 2;
+        }
+      }
+      trsolve_rows_kernel<<<(N + kSolveWarps - 1) / kSolveWarps, kSolveWarps * 32, solve_smem, s>>>(in, Gm, Z, Zb, N, l);
+      count_launch(kFamClf, launches + 1);
+    }
+    return cudaGetLastError();
+  };
+  for (int it = 0; it <= p.q && e == cudaSuccess; ++it) {
+    e = two_products();
+    if (e == cudaSuccess) e = cholqr(U, it == p.q ? 5 : 2);
+  }
+  if (e == cudaSuccess) e = two_products();              // W = X Z and U' = X^T W for the Rayleigh-Ritz step
+  if (e == cudaSuccess) {
+    sgemm_small_kernel<true, float><<<g_ll, 256, 0, s>>>(Z, U, Mm, l, l, N, l, l, l);
+    symmetrize_kernel<<<(l * l + 255) / 256, 256, 0, s>>>(Mm, l);
+    jacobi_init_kernel<<<(l * l + 255) / 256, 256, 0, s>>>(Pm, l, jdone);
+    const int n_even = (l + 1) & ~1, np = n_even / 2;
+    for (int sweep = 0; sweep < kJacobiSweeps; ++sweep) {
+      jacobi_check_kernel<<<1, 1024, 0, s>>>(Mm, l, jdone);
+      for (int t = 0; t < n_even - 1; ++t) {
+        jacobi_rot_kernel<<<(np + 127) / 128, 128, 0, s>>>(Mm, l, t, jcs, jpq, jdone);
+        jacobi_cols_kernel<<<(l * np + 255) / 256, 256, 0, s>>>(Mm, Pm, l, jcs, jpq, jdone);
+        jacobi_rows_kernel<<<(l * np + 255) / 256, 256, 0, s>>>(Mm, l, jcs, jpq, jdone);
+      }
+      count_launch(kFamClf, 1 + 3 * (n_even - 1));
+    }
+    eig_select_kernel<<<1, 1024, (size_t)l * sizeof(int), s>>>(Mm, Pm, l, r, Ps, sigma);
+    sgemm_small_kernel<false, float><<<dim3((r + 63) / 64, (N + 63) / 64), 256, 0, s>>>(Z, Ps, V, N, r, l, l, r, r);
+    const long long tot = (long long)N * r;
+    clf_finish_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(V, c->G, c->d, r, Vb, (__nv_bfloat16*)B_out);
+    count_launch(kFamClf, 6);
+    e = cudaGetLastError();
+  }
+  // A = X V_bf16, stored [T][r]
+  if (e == cudaSuccess) e = launch_gemm<true>(Vb, N, r, r, X, T, N, N, nullptr, (__nv_bfloat16*)A_out, r, flags, device, s);
+  if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
+  return XKV_OK;
+}
+
+}  // namespace xkv

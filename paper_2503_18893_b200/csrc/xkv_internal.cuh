@@ -93,7 +93,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 enum KernelFamily {
   kFamScan = XKV_KERNEL_SCAN, kFamTopk = XKV_KERNEL_TOPK, kFamFused = XKV_KERNEL_FUSED, kFamMerge = XKV_KERNEL_MERGE,
   kFamTile = XKV_KERNEL_TILE, kFamTailTc = XKV_KERNEL_TAIL_TC, kFamTailCuda = XKV_KERNEL_TAIL_CUDA,
-  kFamLandmarks = XKV_KERNEL_LANDMARKS, kFamPrep = XKV_KERNEL_PREP, kFamDense = XKV_KERNEL_DENSE, kFamCount = XKV_KERNEL_FAMILIES
+  kFamLandmarks = XKV_KERNEL_LANDMARKS, kFamPrep = XKV_KERNEL_PREP, kFamDense = XKV_KERNEL_DENSE, kFamClf = XKV_KERNEL_CLF, kFamCount = XKV_KERNEL_FAMILIES
 };
 void count_launch(KernelFamily family, int n = 1);
 
@@ -134,6 +134,8 @@ int select_static(const xkv_select_static_config* c, int l0, int l1, const void*
                   int32_t* sel_cnt, cudaStream_t s);
 // xkv_api.cu: tensor map over [rows][cols] bf16 landmarks, kLandmarkBoxRows-row boxes of 64 columns, 128-byte swizzle
 bool encode_landmark_map(void* out, const void* base, uint64_t rows, uint64_t cols);
+// the same for a general bf16 matrix [rows][cols] with a row pitch (elements) and box_rows-row boxes of 64 columns
+bool encode_bf16_map(void* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows);
 
 // xkv_attend.cu
 size_t attend_part_floats(const xkv_group* grp);
@@ -160,6 +162,14 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
 cudaError_t launch_quantize_rtn4(const __nv_bfloat16* x, long long rows, int cols, void* codes, void* meta, cudaStream_t s);
 cudaError_t launch_dequantize_rtn4(const void* codes, const void* meta, long long rows, int cols, __nv_bfloat16* x,
                                    cudaStream_t s);
+
+// xkv_clf.cu
+int clf_rank_l(const xkv_clf_config* c, int* l);
+int clf_workspace_bytes(const xkv_clf_config* c, uint64_t* bytes);
+int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, void* workspace, uint64_t workspace_bytes,
+                  void* A_out, void* B_out, float* sigma, int device, cudaStream_t s);
+cudaError_t clf_gemm(const void* a, const void* b, int M, int N, int K, float* C, unsigned int* flags, int device,
+                     cudaStream_t s);
 
 // xkv_fused.cu
 int fused_slots(const xkv_group* grp);

@@ -120,7 +120,9 @@ _lib.xkv_debug_launch_counts.restype = ctypes.c_int
 _lib.xkv_debug_set_fault_injection.argtypes = [_P, ctypes.c_uint32]
 _lib.xkv_debug_set_fault_injection.restype = ctypes.c_int
 
-XKV_KERNEL_FAMILIES = ("scan", "topk", "fused", "merge", "tile", "tail_tc", "tail_cuda", "landmarks", "prep", "dense")
+XKV_KERNEL_FAMILIES = ("scan", "topk", "fused", "merge", "tile", "tail_tc", "tail_cuda", "landmarks", "prep", "dense",
+                       "clf")
+XKV_FLAG_CLF_BREAKDOWN = 4
 XKV_INJECT_SCAN_NO_LOAD = 1
 XKV_INJECT_FUSED_NO_B = 2
 
@@ -319,6 +321,67 @@ def xkv_group_set_quantized_bases(grp: Group, codes_k, meta_k, codes_v, meta_v, 
     if st != XKV_OK:
         raise XKVError(st, "xkv_group_set_quantized_bases")
     grp.quantized = (codes_k, meta_k, codes_v, meta_v)      # keep the borrowed tensors alive with the handle
+
+
+class xkv_clf_config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("T", ctypes.c_int32), ("G", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("r", ctypes.c_int32), ("oversample", ctypes.c_int32), ("power_iters", ctypes.c_int32)]
+
+
+_lib.xkv_clf_rank_l.argtypes = [ctypes.POINTER(xkv_clf_config), ctypes.POINTER(ctypes.c_int32)]
+_lib.xkv_clf_rank_l.restype = ctypes.c_int
+_lib.xkv_clf_workspace_bytes.argtypes = [ctypes.POINTER(xkv_clf_config), ctypes.POINTER(ctypes.c_uint64)]
+_lib.xkv_clf_workspace_bytes.restype = ctypes.c_int
+_lib.xkv_clf_factorize.argtypes = [ctypes.POINTER(xkv_clf_config), _P, _P, _P, ctypes.c_uint64, _P, _P, _P, _P]
+_lib.xkv_clf_factorize.restype = ctypes.c_int
+_lib.xkv_clf_status.argtypes = [_P, ctypes.POINTER(ctypes.c_uint32), _P]
+_lib.xkv_clf_status.restype = ctypes.c_int
+_lib.xkv_debug_gemm.argtypes = [_P, _P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P]
+_lib.xkv_debug_gemm.restype = ctypes.c_int
+
+
+def make_clf_config(*, T, G, d, r, oversample=0, power_iters=2) -> xkv_clf_config:
+    return xkv_clf_config(ctypes.sizeof(xkv_clf_config), T, G, d, r, oversample, power_iters)
+
+
+def xkv_clf_rank_l(cfg: xkv_clf_config) -> int:
+    l = ctypes.c_int32()
+    st = _lib.xkv_clf_rank_l(ctypes.byref(cfg), ctypes.byref(l))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_clf_rank_l")
+    return l.value
+
+
+def xkv_clf_workspace_bytes(cfg: xkv_clf_config) -> int:
+    b = ctypes.c_uint64()
+    st = _lib.xkv_clf_workspace_bytes(ctypes.byref(cfg), ctypes.byref(b))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_clf_workspace_bytes")
+    return b.value
+
+
+def xkv_clf_factorize(cfg: xkv_clf_config, X, omega, workspace, A, B, sigma=None, stream=None) -> None:
+    """Cross-layer factorisation of X bf16 [T][G*d] (include/xkv.h); A bf16 [T][r], B bf16 [G][r][d], sigma fp32 [r]."""
+    st = _lib.xkv_clf_factorize(ctypes.byref(cfg), _ptr(X), _ptr(omega), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _ptr(A), _ptr(B), _ptr(sigma),
+                                _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_clf_factorize")
+
+
+def xkv_clf_status(workspace, stream=None):
+    f = ctypes.c_uint32()
+    st = _lib.xkv_clf_status(_ptr(workspace), ctypes.byref(f), _stream(stream))
+    return st, f.value
+
+
+def xkv_debug_gemm(a, b, C, flags, stream=None) -> None:
+    """C (M x N, fp32) = A B^T for a bf16 [K][M] and b bf16 [N][K] on the tensor core (diagnostic)."""
+    K, M = a.shape
+    N = b.shape[0]
+    st = _lib.xkv_debug_gemm(_ptr(a), _ptr(b), M, N, K, _ptr(C), _ptr(flags), _stream(stream))
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_debug_gemm")
 
 
 def xkv_dense_workspace_bytes(grp: Group, cap: int) -> int:

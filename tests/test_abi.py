@@ -126,3 +126,18 @@ def test_quantisation_entry_points_check_their_arguments_on_the_host(xkv):
     assert L.xkv_quantize_rtn(0x1000, 4, 64, 9, 0x2000, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG
     assert L.xkv_dequantize_rtn(0x1008, 0x2000, 4, 64, 4, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG    # alignment
     assert L.xkv_group_set_quantized_bases(None, None, None, None, None, 4) == xkv.XKV_ERR_INVALID_ARG
+
+
+def test_clf_config_is_checked_on_the_host(xkv):
+    ok = xkv.make_clf_config(T=131072, G=4, d=1024, r=512)
+    assert xkv.xkv_clf_rank_l(ok) == 576                      # r + 32 rounded up to a multiple of 64
+    assert xkv.xkv_clf_workspace_bytes(ok) > 131072 * 576 * 2
+    for bad in (dict(T=0), dict(r=12), dict(d=100, G=1), dict(r=8192), dict(power_iters=9)):
+        kw = dict(T=4096, G=2, d=128, r=64)
+        kw.update(bad)
+        with pytest.raises(xkv.XKVError) as e:
+            xkv.xkv_clf_workspace_bytes(xkv.make_clf_config(**kw))
+        assert e.value.status == xkv.XKV_ERR_INVALID_ARG, bad
+    with pytest.raises(xkv.XKVError) as e:                    # l beyond what the eigen-solver's tables hold
+        xkv.xkv_clf_workspace_bytes(xkv.make_clf_config(T=4096, G=4, d=1024, r=2048, oversample=64))
+    assert e.value.status == xkv.XKV_ERR_UNSUPPORTED

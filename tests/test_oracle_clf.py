@@ -95,3 +95,57 @@ def test_bf16_round_ties_to_even_and_exact_values():
     import torch
     y = np.random.default_rng(5).standard_normal(1000).astype(np.float32)
     np.testing.assert_array_equal(O.bf16_round(y), torch.from_numpy(y).bfloat16().float().numpy())
+
+
+# ---- the randomised factorisation (App. "Custom SVD Kernel"): pinned against the exact one above
+
+def _decaying(T, N, rank, noise, seed):
+    rng = np.random.default_rng(seed)
+    s = 1.0 / np.arange(1, rank + 1)
+    X = (rng.standard_normal((T, rank)) * s) @ rng.standard_normal((rank, N)) / np.sqrt(rank)
+    X += noise * np.sqrt((X ** 2).mean()) * rng.standard_normal((T, N))
+    return O.bf16_round(X.astype(np.float32)).astype(np.float64)
+
+
+def test_cholesky_qr_gives_an_orthonormal_basis_of_the_same_span():
+    rng = np.random.default_rng(0)
+    U = rng.standard_normal((300, 40)) * np.logspace(0, -7, 40)          # condition number 1e7
+    Z = O.cholesky_qr(U)
+    assert np.abs(Z.T @ Z - np.eye(40)).max() < 1e-8
+    # same column space: projecting U on span(Z) changes nothing
+    assert np.abs(Z @ (Z.T @ U) - U).max() < 1e-9 * np.abs(U).max()
+    # against the library's Householder QR: identical projector
+    Q, _ = np.linalg.qr(U)
+    assert np.abs(Z @ Z.T - Q @ Q.T).max() < 1e-6
+
+
+def test_randomized_factorisation_is_close_to_the_optimum_and_b_is_orthonormal():
+    X = _decaying(1500, 256, 48, 0.01, 1)
+    r, l = 64, 128
+    omega = O.bf16_round(np.random.default_rng(2).standard_normal((256, l)).astype(np.float32))
+    A, V, sig = O.clf_randomized(X, r, omega, power_iters=2)
+    sv = np.linalg.svd(X, compute_uv=False)
+    res = ((X - A.astype(np.float64) @ V.astype(np.float64).T) ** 2).sum()
+    assert res <= 1.15 * (sv[r:] ** 2).sum()      # Eckart-Young optimum; the flat noise tail is what the 32 extra directions cannot order
+    assert np.abs(V.T.astype(np.float64) @ V - np.eye(r)).max() < 1e-2    # bf16 storage
+    np.testing.assert_allclose(sig[:48], sv[:48], rtol=1e-2)
+    # more power iterations never hurt, none at all is worse
+    A0, V0, _ = O.clf_randomized(X, r, omega, power_iters=0)
+    res0 = ((X - A0.astype(np.float64) @ V0.astype(np.float64).T) ** 2).sum()
+    assert res <= res0 * 1.001
+
+
+def test_randomized_factorisation_recovers_exactly_low_rank_input():
+    rng = np.random.default_rng(3)
+    X = O.bf16_round((rng.standard_normal((800, 20)) @ rng.standard_normal((20, 128)) / 4).astype(np.float32)).astype(np.float64)
+    omega = O.bf16_round(rng.standard_normal((128, 64)).astype(np.float32))
+    A, V, sig = O.clf_randomized(X, 32, omega, power_iters=1)
+    res = ((X - A.astype(np.float64) @ V.astype(np.float64).T) ** 2).sum() / (X ** 2).sum()
+    assert res < 1e-4                                                     # rounding of X, A and V to bf16 only
+    # with l = N the subspace is everything and the result is the exact truncated SVD up to that rounding
+    om_full = O.bf16_round(rng.standard_normal((128, 128)).astype(np.float32))
+    Xn = _decaying(600, 128, 128, 0.0, 4)
+    A2, V2, _ = O.clf_randomized(Xn, 32, om_full, power_iters=0)
+    sv = np.linalg.svd(Xn, compute_uv=False)
+    res2 = ((Xn - A2.astype(np.float64) @ V2.astype(np.float64).T) ** 2).sum()
+    assert abs(res2 / (sv[32:] ** 2).sum() - 1.0) < 2e-2
