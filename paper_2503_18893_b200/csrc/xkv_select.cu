@@ -160,12 +160,13 @@ constexpr int kTopkCand = 256;    // at most this many keys are ranked against o
 // Keys of this thread's 16 consecutive chunks of one super-block (0 beyond n_c; callers mask by index).
 // sign == 0: the array already holds keys (the landmark scan writes them); else it holds floats and the key is
 // that of sign * value.
-__device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, float sign, uint32_t (&key)[kTopkItems]) {
+template <int ITEMS>
+__device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, int n_c, float sign, uint32_t (&key)[ITEMS]) {
   const bool keyed = sign == 0.0f;
-  if (j0 + kTopkItems <= n_c && ((n_c & 3) == 0)) {
+  if (j0 + ITEMS <= n_c && ((n_c & 3) == 0)) {
     const float4* p = reinterpret_cast<const float4*>(S + j0);
 #pragma unroll
-    for (int i = 0; i < kTopkItems / 4; ++i) {
+    for (int i = 0; i < ITEMS / 4; ++i) {
       const float4 v = p[i];
       const float f[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -173,7 +174,7 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ S, int j0, i
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < kTopkItems; ++i) {
+    for (int i = 0; i < ITEMS; ++i) {
       const float f = (j0 + i < n_c) ? S[j0 + i] : 0.0f;
       key[i] = (j0 + i < n_c) ? (keyed ? __float_as_uint(f) : score_key(f * sign)) : 0u;
     }
@@ -542,11 +543,10 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 // maxima -- are >= it), and with k_ch a few percent of n_c only a few percent of the keys pass it.  The keys >= P
 // go to a list in shared memory (key, chunk index); the exact k_ch-th largest key is then found on the list by
 // the radix select of topk_kernel; membership goes to a bitmap over the chunks (united with the head's outlier
-// chunks), whose prefix popcounts give the ascending output positions.  GPT = 16 disables the filter (P = the
-// smallest key): chosen by the host when there are fewer groups than k_ch.  The result is identical to
-// topk_kernel's for every input; only the amount of work differs.
-constexpr int kPivotListMax = kTopkThreads * kTopkItems;    // every key may pass (all keys equal)
-
+// chunks), whose prefix popcounts give the ascending output positions.  GPT = 0 disables the filter (P = the
+// smallest key): chosen by the host when there are fewer groups than k_ch.  ITEMS = 16 keys per thread serve
+// n_c <= 16384 chunks, ITEMS = 32 (keys read twice instead of held in registers) n_c <= 32768.  The result is
+// identical to topk_kernel's for every input; only the amount of work differs.
 // Bin (counted from the top) that holds the `need`-th largest of the keys counted in hist[0..kTopkBins), by a
 // suffix sum over the bins; thread t owns bins 2t, 2t+1.  Results in sh[0] = bin, sh[1] = rank wanted inside the
 // bin, sh[2] = keys in the bin.  Contains barriers: call it from all threads.
@@ -581,11 +581,13 @@ __device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, ui
   __syncthreads();
 }
 
-template <int GPT>
+template <int GPT, int ITEMS>
 __global__ void __launch_bounds__(kTopkThreads, 1)
 topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out, float sign,
                   int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
   extern __shared__ __align__(16) uint8_t pivot_smem[];
+  constexpr int kPivotListMax = kTopkThreads * ITEMS;                              // every key may pass (all keys equal)
+  static_assert(kPivotListMax <= 65536 && kPivotListMax / 32 <= kTopkThreads, "16-bit chunk index, one bitmap word per thread");
   uint32_t* list_key = reinterpret_cast<uint32_t*>(pivot_smem);                    // [kPivotListMax]; later the chunk list
   uint16_t* list_idx = reinterpret_cast<uint16_t*>(list_key + kPivotListMax);      // [kPivotListMax]
   __shared__ __align__(16) uint32_t hist[kTopkBins];
@@ -601,19 +603,19 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
   const float* __restrict__ S = dev.pooled + prob * dev.n_c;
   int32_t* __restrict__ out = sel_idx + prob * k_cap;
   const int n_c = dev.n_c, c = dev.c, T = dev.T;
-  constexpr int NW = kPivotListMax / 32;                               // words of a bitmap (512)
-  constexpr int NG = GPT == 16 ? 1 : GPT;                              // group maxima kept per thread
-  constexpr int GS = kTopkItems / NG;                                  // keys per group
+  constexpr int NW = kPivotListMax / 32;                               // words of a bitmap
+  constexpr int NG = GPT == 0 ? 1 : GPT;                               // group maxima kept per thread
+  constexpr int GS = ITEMS / NG;                                       // keys per group
 
   grid_dependency_wait();                      // the pooled scores come from the kernel launched before
   grid_dependency_launch();
-  const int j0 = tid * kTopkItems;
+  const int j0 = tid * ITEMS;
   const bool all = (k_ch >= n_c);
   uint32_t thr = 0, need_eq = 0;
   for (int w = tid; w < NW; w += kTopkThreads) { take_w[w] = 0u; eq_w[w] = 0u; }
   if (tid == 0) sh_n = 0;
   if (!all) {
-    uint32_t key[kTopkItems];
+    uint32_t key[ITEMS];
     load_keys(S, j0, n_c, sign, key);
     // ---- extrema of this thread's keys and of its groups
     uint32_t kmin = 0xffffffffu, kmax = 0u;
@@ -621,10 +623,10 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
 #pragma unroll
     for (int g = 0; g < NG; ++g) gmax[g] = 0u;
 #pragma unroll
-    for (int i = 0; i < kTopkItems; ++i) {
+    for (int i = 0; i < ITEMS; ++i) {
       if (j0 + i < n_c) {
         kmin = min(kmin, key[i]); kmax = max(kmax, key[i]);
-        if (GPT != 16) gmax[i / GS] = max(gmax[i / GS], key[i]);
+        if (GPT != 0) gmax[i / GS] = max(gmax[i / GS], key[i]);
       }
     }
 #pragma unroll
@@ -643,7 +645,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
     }
     // ---- pivot: lower edge of the bin that holds the k_ch-th largest group maximum
     uint32_t P = kmin;
-    if (GPT != 16) {
+    if (GPT != 0) {
       const uint32_t span1 = kmax - kmin;
       const int bits1 = 32 - __clz(span1);
       const int sh1 = bits1 > 11 ? bits1 - 11 : 0;
@@ -658,9 +660,10 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
     }
     // ---- the keys >= P, with their chunk index, to the list (one shared-memory atomic per warp)
     {
+      if (ITEMS > 16) load_keys(S, j0, n_c, sign, key);   // 32 keys are not held across the barriers above: read them again
       uint32_t cm = 0;
 #pragma unroll
-      for (int i = 0; i < kTopkItems; ++i) {
+      for (int i = 0; i < ITEMS; ++i) {
         if (j0 + i < n_c && key[i] >= P) cm |= 1u << i;
       }
       const uint32_t mine_c = (uint32_t)__popc(cm);
@@ -676,7 +679,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
         wbase = __shfl_sync(0xffffffffu, wbase, 31);
         uint32_t at = wbase + inc - mine_c;
 #pragma unroll
-        for (int i = 0; i < kTopkItems; ++i) {
+        for (int i = 0; i < ITEMS; ++i) {
           if ((cm >> i) & 1u) { list_key[at] = key[i]; list_idx[at] = (uint16_t)(j0 + i); ++at; }
         }
       }
@@ -834,24 +837,33 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
 static cudaError_t launch_topk(const GroupDev& dev, int device, int problems, int l0, int k_ch, int k_cap,
                                const int32_t* outliers, int n_out, float sign, int32_t* sel_idx, int32_t* sel_cnt,
                                cudaStream_t s) {
-  if (dev.n_c > kTopkThreads * kTopkItems)
+  if (dev.n_c > kTopkThreads * 32)
     return launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, outliers, n_out,
                       sign, sel_idx, sel_cnt);
-  // groups per thread: the fewest with at least k_ch groups in all (16 = no filter)
-  const size_t smem = (size_t)kPivotListMax * (sizeof(uint32_t) + sizeof(uint16_t));
+  // keys per thread: 16 up to 16384 chunks, 32 beyond; groups per thread: the fewest with at least k_ch groups in all
+  // (0 = no filter)
+  const int items = dev.n_c <= kTopkThreads * 16 ? 16 : 32;
+  const size_t smem = (size_t)kTopkThreads * items * (sizeof(uint32_t) + sizeof(uint16_t));
   cudaError_t e;
-#define XKV_PIVOT(GPT)                                                                                         \
-  do {                                                                                                         \
-    e = ensure_dyn_smem<topk_pivot_kernel<GPT>>(smem, device);                                                 \
-    if (e == cudaSuccess)                                                                                      \
-      e = launch_pdl(topk_pivot_kernel<GPT>, dim3(problems), dim3(kTopkThreads), smem, s, dev, l0, k_ch, k_cap, \
-                     outliers, n_out, sign, sel_idx, sel_cnt);                                                 \
+#define XKV_PIVOT(GPT, ITEMS)                                                                                         \
+  do {                                                                                                                \
+    e = ensure_dyn_smem<topk_pivot_kernel<GPT, ITEMS>>(smem, device);                                                 \
+    if (e == cudaSuccess)                                                                                             \
+      e = launch_pdl(topk_pivot_kernel<GPT, ITEMS>, dim3(problems), dim3(kTopkThreads), smem, s, dev, l0, k_ch, k_cap, \
+                     outliers, n_out, sign, sel_idx, sel_cnt);                                                        \
   } while (0)
-  auto groups = [&](int gpt) { return (dev.n_c + kTopkItems / gpt - 1) / (kTopkItems / gpt); };
-  if (groups(1) >= k_ch) XKV_PIVOT(1);
-  else if (groups(2) >= k_ch) XKV_PIVOT(2);
-  else if (groups(4) >= k_ch) XKV_PIVOT(4);
-  else XKV_PIVOT(16);
+  auto groups = [&](int gpt) { return (dev.n_c + items / gpt - 1) / (items / gpt); };
+  if (items == 16) {
+    if (groups(1) >= k_ch) XKV_PIVOT(1, 16);
+    else if (groups(2) >= k_ch) XKV_PIVOT(2, 16);
+    else if (groups(4) >= k_ch) XKV_PIVOT(4, 16);
+    else XKV_PIVOT(0, 16);
+  } else {
+    if (groups(1) >= k_ch) XKV_PIVOT(1, 32);
+    else if (groups(2) >= k_ch) XKV_PIVOT(2, 32);
+    else if (groups(4) >= k_ch) XKV_PIVOT(4, 32);
+    else XKV_PIVOT(0, 32);
+  }
 #undef XKV_PIVOT
   return e;
 }

@@ -212,9 +212,11 @@ def test_small_ranks_and_many_tiles_do_not_stall():
     g.close()
 
 
-def test_more_chunks_than_one_topk_superblock():
-    """n_c = 17501 > 16384: the top-k kernel re-reads the pooled scores instead of caching them in registers."""
-    s = synth.config(1, T=140001, k=3000, r_k=8, r_v=8)
+@pytest.mark.parametrize("T", [140001, 300001])
+def test_more_chunks_than_one_topk_superblock(T):
+    """n_c = 17501: 32 keys per thread in the list-based top-k; n_c = 37501: the kernel that re-reads the pooled
+    scores super-block by super-block."""
+    s = synth.config(1, T=T, k=3000, r_k=8, r_v=8)
     inp = C.case_from_factors(s)
     oidx, ocnt, _, _ = C.oracle_step(s, inp, 0, problems=[(0, 0, 0), (1, 0, 1)])
     g = C.GpuCase(s, inp)
@@ -263,11 +265,12 @@ def test_selection_with_static_outliers_union():
     g.close()
 
 
-def test_outliers_with_more_chunks_than_one_superblock():
-    s = synth.config(1, T=8 * 20000, k=256, H_kv=1, H_q=2, G=1, r_k=16, r_v=16)     # n_c = 20000 > 16384
+@pytest.mark.parametrize("n_c", [20000, 40000])
+def test_outliers_with_more_chunks_than_one_superblock(n_c):
+    s = synth.config(1, T=8 * n_c, k=256, H_kv=1, H_q=2, G=1, r_k=16, r_v=16)       # both multi-super-block top-k kernels
     inp = C.case_from_factors(s)
     n_out = 7
-    outl = np.array([[[[0, 16383, 16384, 19999, 5, 5, 12345]]]], dtype=np.int32)
+    outl = np.array([[[[0, 16383, 16384, n_c - 1, 5, 5, 12345]]]], dtype=np.int32)
     g = C.GpuCase(s, inp)
     o_dev = torch.from_numpy(outl).cuda()
     g.xkv.xkv_group_set_outliers(g.grp, o_dev, n_out)
