@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--groups", type=int, default=None, help="number of windows (default: the config's)")
     ap.add_argument("--tail", type=int, default=0,
                     help="rows of uncompressed generated tokens attended to besides the selected rows (default none)")
-    ap.add_argument("--quant", type=int, default=0, choices=[0, 4],
+    ap.add_argument("--quant", type=int, default=0, choices=[0, 3, 4],
                     help="gather the token bases from b-bit round-to-nearest codes (0: bf16 bases, the headline)")
     ap.add_argument("--op", default="decode", choices=["decode", "landmarks", "clf"],
                     help="decode: the hot path (default).  landmarks: the prefill-side Algorithm 1 kernel alone "
@@ -554,8 +554,8 @@ def measure_point(shape, args, world, rank, local_rank, dist, with_cpu=True, wit
         n = cpu_problems or args.cpu_problems or min(n_all, 32)
         oinp = wl.inputs[0]
         if getattr(args, "quant", 0):       # the oracle works on what the codes stand for
-            oinp = workload.GroupInputs(xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_k, args.quant), args.quant),
-                                        xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_v, args.quant), args.quant),
+            oinp = workload.GroupInputs(xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_k, args.quant), bits=args.quant),
+                                        xkv.xkv_dequantize_rtn(*xkv.xkv_quantize_rtn(oinp.A_v, args.quant), bits=args.quant),
                                         oinp.B_k, oinp.B_v, oinp.landmarks, oinp.q)
         dt, np_, cores, ores = oracle_sample(shape, oinp, n, spread=(n < n_all))
         line["cpu_baseline"] = {"value": (np_ / n_all) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",

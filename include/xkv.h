@@ -218,7 +218,11 @@ XKV_API int xkv_debug_gemm(const void* a, const void* b, int32_t M, int32_t N, i
  * codes  [rows][cols/2] bytes, 16-byte aligned.  Inside every 32-bit word (scalars e0..e7) nibble k of the low half
  *        is e_2k and nibble k of the high half is e_2k+1.
  * meta   uint32 [rows][cols/32]: scale in the low 16 bits, offset in the high 16 bits.
- * bits   4 (the only width with a storage format here; else UNSUPPORTED).
+ * bits   4, or 3 (the paper's other setting: 8.03x -> 32.12x).  With 3 bits the step is (max - min)/7, codes clip at
+ *        7, and a group is ONE 16-byte record in `codes` ([rows][cols/32] records, cols/2 bytes per row as for 4 bits;
+ *        `meta` is not used and may be NULL): {meta word, w0, w1, w2}; word w_j holds scalars 10j..10j+9 as five
+ *        pairs, (w_j >> 3k) & 0x00070007 = (e_10j+2k, e_10j+2k+1); bits 15 of w0, w1, w2 hold scalar 30 and bits 31
+ *        scalar 31, least significant bit in w0.  Other widths: UNSUPPORTED.
  * xkv_dequantize_rtn writes x_hat (for the small per-layer matrices B, which a handle takes as bf16).
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
  */
@@ -227,12 +231,13 @@ XKV_API int xkv_dequantize_rtn(const void* codes, const void* meta, int64_t rows
                                void* stream);
 
 /*
- * From now on xkv_sr_reconstruct_attend (and the _tail variant) gathers the token bases from 4-bit codes and
- * dequantises them on the way into shared memory (Eq. 3 on x_hat); a gathered row costs r/2 + r/8 bytes instead
- * of 2r.  The handle's A_k / A_v (which xkv_group_create then accepts as NULL) are no longer read.
+ * From now on xkv_sr_reconstruct_attend (and the _tail variant) gathers the token bases from 4-bit or 3-bit codes and
+ * dequantises them on the way into shared memory (Eq. 3 on x_hat); a gathered row costs r/2 + r/8 bytes (4 bits) or
+ * r/2 bytes (3 bits) instead of 2r.  The handle's A_k / A_v (which xkv_group_create then accepts as NULL) are no longer read.
  * codes_k, meta_k  quantised A_k: [batch][T][r_k/2] bytes and uint32 [batch][T][r_k/32] (layout of xkv_quantize_rtn
  *                  with rows = batch*T), device, BORROWED until the handle is destroyed; likewise codes_v, meta_v.
- * bits             4; r_k and r_v must be multiples of 32.  All-NULL pointers switch back to the bf16 bases.
+ * bits             4 or 3 (with 3 the meta pointers are not used and may be NULL); r_k and r_v must be multiples of 32.
+ *                  All-NULL pointers switch back to the bf16 bases.
  * Errors: INVALID_ARG, UNSUPPORTED (ranks, or a shape the tensor-core path does not cover).
  */
 XKV_API int xkv_group_set_quantized_bases(xkv_group* grp, const void* codes_k, const void* meta_k, const void* codes_v,

@@ -495,25 +495,30 @@ int xkv_debug_gemm(const void* a, const void* b, int32_t M, int32_t N, int32_t K
   return XKV_OK;
 }
 
-static int check_rtn_args(const void* a, const void* b, const void* c3, int64_t rows, int32_t cols, int32_t bits) {
-  if (!a || !b || !c3 || rows < 0 || cols < 32 || cols % 32 != 0) return XKV_ERR_INVALID_ARG;
-  if (((uintptr_t)a & 15u) || ((uintptr_t)b & 15u) || ((uintptr_t)c3 & 15u)) return XKV_ERR_INVALID_ARG;
-  if (bits != 4) return (bits >= 1 && bits <= 8) ? XKV_ERR_UNSUPPORTED : XKV_ERR_INVALID_ARG;
+// x and codes are required; meta only for 4 bits (the 3-bit records carry their scale and offset)
+static int check_rtn_args(const void* x, const void* codes, const void* meta, int64_t rows, int32_t cols, int32_t bits) {
+  if (bits < 1 || bits > 8) return XKV_ERR_INVALID_ARG;
+  if (!x || !codes || rows < 0 || cols < 32 || cols % 32 != 0) return XKV_ERR_INVALID_ARG;
+  if (((uintptr_t)x & 15u) || ((uintptr_t)codes & 15u) || ((uintptr_t)meta & 15u)) return XKV_ERR_INVALID_ARG;
+  if (bits != 4 && bits != 3) return XKV_ERR_UNSUPPORTED;
+  if (bits == 4 && !meta) return XKV_ERR_INVALID_ARG;
   return XKV_OK;
 }
 
 int xkv_quantize_rtn(const void* x, int64_t rows, int32_t cols, int32_t bits, void* codes, void* meta, void* stream) {
   const int st = check_rtn_args(x, codes, meta, rows, cols, bits);
   if (st != XKV_OK) return st;
-  cudaError_t e = launch_quantize_rtn4((const __nv_bfloat16*)x, rows, cols, codes, meta, (cudaStream_t)stream);
+  cudaError_t e = bits == 4 ? launch_quantize_rtn4((const __nv_bfloat16*)x, rows, cols, codes, meta, (cudaStream_t)stream)
+                            : launch_quantize_rtn3((const __nv_bfloat16*)x, rows, cols, codes, (cudaStream_t)stream);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }
 
 int xkv_dequantize_rtn(const void* codes, const void* meta, int64_t rows, int32_t cols, int32_t bits, void* x, void* stream) {
-  const int st = check_rtn_args(codes, meta, x, rows, cols, bits);
+  const int st = check_rtn_args(x, codes, meta, rows, cols, bits);
   if (st != XKV_OK) return st;
-  cudaError_t e = launch_dequantize_rtn4(codes, meta, rows, cols, (__nv_bfloat16*)x, (cudaStream_t)stream);
+  cudaError_t e = bits == 4 ? launch_dequantize_rtn4(codes, meta, rows, cols, (__nv_bfloat16*)x, (cudaStream_t)stream)
+                            : launch_dequantize_rtn3(codes, rows, cols, (__nv_bfloat16*)x, (cudaStream_t)stream);
   if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return XKV_ERR_CUDA; }
   return XKV_OK;
 }
@@ -522,15 +527,17 @@ int xkv_group_set_quantized_bases(xkv_group* g, const void* codes_k, const void*
                                   const void* meta_v, int32_t bits) {
   if (!g) return XKV_ERR_INVALID_ARG;
   if (!codes_k && !meta_k && !codes_v && !meta_v) {
-    g->dev.Aq_k = g->dev.Aq_v = nullptr; g->dev.Am_k = g->dev.Am_v = nullptr;
+    g->dev.Aq_k = g->dev.Aq_v = nullptr; g->dev.Am_k = g->dev.Am_v = nullptr; g->dev.quant_bits = 0;
     return XKV_OK;
   }
-  if (!codes_k || !meta_k || !codes_v || !meta_v) return XKV_ERR_INVALID_ARG;
+  if (bits < 1 || bits > 8) return XKV_ERR_INVALID_ARG;
+  if (bits != 4 && bits != 3) return XKV_ERR_UNSUPPORTED;
+  if (!codes_k || !codes_v || (bits == 4 && (!meta_k || !meta_v))) return XKV_ERR_INVALID_ARG;
   if (((uintptr_t)codes_k | (uintptr_t)meta_k | (uintptr_t)codes_v | (uintptr_t)meta_v) & 15u) return XKV_ERR_INVALID_ARG;
-  if (bits != 4) return (bits >= 1 && bits <= 8) ? XKV_ERR_UNSUPPORTED : XKV_ERR_INVALID_ARG;
   if (g->cfg.r_k % 32 != 0 || g->cfg.r_v % 32 != 0 || !fused_supported(g)) return XKV_ERR_UNSUPPORTED;
   g->dev.Aq_k = (const uint8_t*)codes_k; g->dev.Am_k = (const uint32_t*)meta_k;
   g->dev.Aq_v = (const uint8_t*)codes_v; g->dev.Am_v = (const uint32_t*)meta_v;
+  g->dev.quant_bits = bits;
   return XKV_OK;
 }
 

@@ -216,9 +216,9 @@ __host__ __device__ constexpr int ring_slots() {
 
 // NR: query heads per KV head rounded up to 4, 8 or 16.  WB: most 128-column blocks of r_v (registers of the
 // value epilogue): NR * WB <= 64.
-// QUANT: the token bases are gathered from 4-bit codes (xkv_group_set_quantized_bases) and dequantised by the
-// producer warps on their way into the rings.
-template <int DH, int NR, int WB, bool PROF, bool QUANT>
+// QUANT = 4 or 3: the token bases are gathered from 4-bit or 3-bit codes (xkv_group_set_quantized_bases) and
+// dequantised by the producer warps on their way into the rings; 0: bf16 bases.
+template <int DH, int NR, int WB, bool PROF, int QUANT>
 __global__ void __launch_bounds__(kThreads, 1)
 sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched sc, const __nv_bfloat16* __restrict__ q,
                 const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt) {
@@ -417,8 +417,9 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         const bool in = col0 < r;                          // false in a padding slab: zeros are stored
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
+          // 4 bits: 16 bytes of codes and a separate scale/offset word; 3 bits: one 16-byte record {meta, w0, w1, w2}
           cw[i] = in ? __ldg(reinterpret_cast<const uint4*>(Cb + (size_t)rw[i] * (size_t)(r >> 1) + (col0 >> 1))) : make_uint4(0, 0, 0, 0);
-          mw[i] = in ? __ldg(Mb + (size_t)rw[i] * (size_t)(r >> 5) + (col0 >> 5)) : 0u;
+          if (QUANT == 4) mw[i] = in ? __ldg(Mb + (size_t)rw[i] * (size_t)(r >> 5) + (col0 >> 5)) : 0u;
         }
       };
       auto store = [&](const uint4 (&cw)[8], const uint32_t (&mw)[8]) -> bool {
@@ -436,12 +437,17 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         for (int i = 0; i < 8; ++i) {
           const uint32_t j = rq + 16u * (uint32_t)i;       // tile row
           const uint32_t w[4] = {cw[i].x, cw[i].y, cw[i].z, cw[i].w};
+          uint32_t o[16];
+          if (QUANT == 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) dequant_word(w[u], mw[i], &o[4 * u]);
+          } else {
+            dequant_group3(w[0], w[1], w[2], w[3], o);
+          }
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            uint32_t o[4];
-            dequant_word(w[u], mw[i], o);
             const uint32_t a = st + j * 128u + (((u0 + (uint32_t)u) ^ (j & 7u)) << 4);
-            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o[4 * u]), "r"(o[4 * u + 1]), "r"(o[4 * u + 2]), "r"(o[4 * u + 3]) : "memory");
           }
         }
         asm volatile("cp.async.wait_all;" ::: "memory");   // the staged rotary rows of this tile (key stream) have landed too
@@ -534,7 +540,7 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
         mbar_arrive(BAR(bl.posfull + pb));
       }
       if (!wait_bar(ctx, BAR(bl.posfull + pb), (uint32_t)((it >> 2) & 1), ps + 2)) { ok = false; break; }
-      if constexpr (QUANT) {
+      if constexpr (QUANT != 0) {
         uint32_t rw[8];
         load_rows_q(rw);
         if (!kstream) mbar_arrive(BAR(bl.vfree + pb));     // this thread is done with the position buffer
@@ -1082,17 +1088,21 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   cudaError_t e;
   if (grp->prof) {     // the variant with the diagnostic counters compiled in
     if (dev.Aq_k) return cudaErrorNotSupported;        // no diagnostic variant of the quantised gather
-    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, true, false>>(smem, grp->device);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, true, 0>>(smem, grp->device);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(sr_fused_kernel<DH, NR, WB, true, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, true, 0>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+  } else if (dev.Aq_k && dev.quant_bits == 3) {
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, 3>>(smem, grp->device);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, 3>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   } else if (dev.Aq_k) {
-    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, true>>(smem, grp->device);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, 4>>(smem, grp->device);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, true>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, 4>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   } else {
-    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, false>>(smem, grp->device);
+    e = ensure_dyn_smem<sr_fused_kernel<DH, NR, WB, false, 0>>(smem, grp->device);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, false>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
+    e = launch_pdl(sr_fused_kernel<DH, NR, WB, false, 0>, dim3(sc.n_ctas), dim3(kThreads), smem, s, mk, dev, sc, q, sel_idx, sel_cnt);
   }
   count_launch(kFamFused);
   if (e != cudaSuccess) return e;

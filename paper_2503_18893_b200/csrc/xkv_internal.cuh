@@ -40,7 +40,8 @@ struct GroupDev {
   unsigned int* flags;              // device flag word
   const int32_t* outliers;          // [G][batch][H_kv][n_out] static outlier chunk ids (Algorithm 2 line 5), or nullptr
   int n_out;
-  const uint8_t* Aq_k;              // 4-bit codes of A_k [batch][T][r_k/2], or nullptr (then the bf16 bases are gathered)
+  int quant_bits;                   // 0: bf16 bases; 4: codes + scale/offset words; 3: 16-byte records in Aq_* (Am_* unused)
+  const uint8_t* Aq_k;              // codes of A_k [batch][T][r_k/2], or nullptr (then the bf16 bases are gathered)
   const uint8_t* Aq_v;              // [batch][T][r_v/2]
   const uint32_t* Am_k;             // scale/offset words [batch][T][r_k/32]
   const uint32_t* Am_v;             // [batch][T][r_v/32]
@@ -162,6 +163,8 @@ cudaError_t launch_tail_partials(const xkv_group* grp, int l0, int l1, const __n
 cudaError_t launch_quantize_rtn4(const __nv_bfloat16* x, long long rows, int cols, void* codes, void* meta, cudaStream_t s);
 cudaError_t launch_dequantize_rtn4(const void* codes, const void* meta, long long rows, int cols, __nv_bfloat16* x,
                                    cudaStream_t s);
+cudaError_t launch_quantize_rtn3(const __nv_bfloat16* x, long long rows, int cols, void* rec, cudaStream_t s);
+cudaError_t launch_dequantize_rtn3(const void* rec, long long rows, int cols, __nv_bfloat16* x, cudaStream_t s);
 
 // xkv_clf.cu
 int clf_rank_l(const xkv_clf_config* c, int* l);

@@ -186,6 +186,26 @@ __device__ __forceinline__ void dequant_word(uint32_t w, uint32_t meta, uint32_t
   }
 }
 
+// The 3-bit format: a group of 32 scalars is one 16-byte record {meta, w0, w1, w2}.  Word w_j holds scalars
+// 10j .. 10j+9 as five pairs, (w_j >> 3k) & 0x00070007 = (e_10j+2k, e_10j+2k+1); bits 15 and 31 of the three words
+// together hold scalars 30 (bits 15) and 31 (bits 31), least significant bit in w0.  Sixteen registers of two bf16.
+__device__ __forceinline__ void dequant_group3(uint32_t meta, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t* out16) {
+  const uint32_t s2 = __byte_perm(meta, meta, 0x1010);
+  const uint32_t z2 = __byte_perm(meta, meta, 0x3232);
+  const uint32_t w[3] = {w0, w1, w2};
+  auto one = [&](uint32_t pair, int at) {
+    uint32_t n, x;
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(n) : "r"(pair | 0x43004300u), "r"(0x43004300u));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(x) : "r"(n), "r"(s2), "r"(z2));
+    out16[at] = x;
+  };
+#pragma unroll
+  for (int j = 0; j < 3; ++j)
+#pragma unroll
+    for (int k = 0; k < 5; ++k) one((w[j] >> (3 * k)) & 0x00070007u, 5 * j + k);
+  one(((w0 >> 15) & 0x00010001u) | ((w1 >> 14) & 0x00020002u) | ((w2 >> 13) & 0x00040004u), 15);
+}
+
 // Programmatic dependent launch: block until the kernel this one depends on has completed and flushed its writes
 // (a no-op when the kernel was not launched with the programmatic-serialization attribute).
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -294,11 +294,12 @@ def xkv_sr_reconstruct_attend_tail(grp: Group, layer_begin: int, layer_end: int,
 
 def xkv_quantize_rtn(x, bits: int = 4, stream=None):
     """RTN-quantise a bf16 device tensor [..., cols] along its last axis in groups of 32 (include/xkv.h).
-    Returns (codes uint8 [..., cols/2], meta int32 [..., cols/32]) device tensors."""
+    Returns (codes uint8 [..., cols/2], meta int32 [..., cols/32] or None for 3 bits) device tensors."""
     cols = x.shape[-1]
     rows = x.numel() // cols
     codes = torch.empty(x.shape[:-1] + (cols // 2,), dtype=torch.uint8, device=x.device)
-    meta = torch.empty(x.shape[:-1] + (cols // 32,), dtype=torch.int32, device=x.device)
+    # 4 bits: one scale/offset word per group beside the codes; 3 bits: the 16-byte records hold them (meta is None)
+    meta = torch.empty(x.shape[:-1] + (cols // 32,), dtype=torch.int32, device=x.device) if bits == 4 else None
     st = _lib.xkv_quantize_rtn(_ptr(x), rows, cols, bits, _ptr(codes), _ptr(meta), _stream(stream))
     if st != XKV_OK:
         raise XKVError(st, "xkv_quantize_rtn")

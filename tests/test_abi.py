@@ -122,7 +122,8 @@ def test_launch_counters_by_family(xkv):
 def test_quantisation_entry_points_check_their_arguments_on_the_host(xkv):
     L = xkv._lib
     assert L.xkv_quantize_rtn(0x1000, 4, 48, 4, 0x2000, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG      # cols % 32
-    assert L.xkv_quantize_rtn(0x1000, 4, 64, 3, 0x2000, 0x3000, None) == xkv.XKV_ERR_UNSUPPORTED      # no 3-bit format
+    assert L.xkv_quantize_rtn(0x1000, 4, 64, 5, 0x2000, 0x3000, None) == xkv.XKV_ERR_UNSUPPORTED      # no 5-bit format
+    assert L.xkv_quantize_rtn(0x1000, 4, 64, 4, 0x2000, None, None) == xkv.XKV_ERR_INVALID_ARG        # 4 bits need meta
     assert L.xkv_quantize_rtn(0x1000, 4, 64, 9, 0x2000, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG
     assert L.xkv_dequantize_rtn(0x1008, 0x2000, 4, 64, 4, 0x3000, None) == xkv.XKV_ERR_INVALID_ARG    # alignment
     assert L.xkv_group_set_quantized_bases(None, None, None, None, None, 4) == xkv.XKV_ERR_INVALID_ARG
