@@ -321,102 +321,169 @@ trsolve_rows_kernel(const float* __restrict__ U, const double* __restrict__ L, f
 namespace {
 
 // Eigen-decomposition of the symmetric l x l matrix M by cyclic Jacobi rotations in the round-robin (tournament)
-// order: every round rotates l/2 disjoint index pairs at once, as three kernels (the rotations of the round; columns
-// p, q of M and of P for every row; rows p, q of M for every column) so that the work of a round spreads over
-// the SMs.  A check per sweep sets *done once the off-diagonal weight is below working precision; every kernel
-// returns at once after that.  On return the eigenvalues are on the diagonal of M, the eigenvectors the columns of P.
+// order: every round rotates l/2 disjoint index pairs at once.  A check per sweep ends the sweeps once the
+// off-diagonal weight is below working precision.  On return the eigenvalues are on the diagonal of M, the
+// eigenvectors the columns of P.
 constexpr int kJacobiMaxPairs = 1024;
 constexpr int kJacobiSweeps = 12;
 
-__global__ void jacobi_init_kernel(float* __restrict__ P, int l, int* __restrict__ done) {
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e == 0) *done = 0;
-  if (e < l * l) P[e] = (e / l == e % l) ? 1.0f : 0.0f;
+// The sweeps are one cooperative kernel.  All CTAs are resident at once, so a round needs no kernel boundary (as
+// three launches per round the ~7000 rounds of a 576 x 576 matrix were launch bound: 63 ms against 13 ms): every round reads the
+// matrices of the previous round (M, P in buffer `cur`) and writes the other buffer, and one grid-wide barrier
+// separates the rounds.  A round: every CTA works out the l/2 rotations of the round from M (cheap, and saves a
+// second barrier), then the grid updates M block by block -- the 2 x 2 block (rows p_a, q_a; columns p_b, q_b)
+// takes the column rotation of pair b and then the row rotation of pair a --
+// and rotates the column pairs of P.  Reads bypass L1 (other SMs wrote the data), the barrier is an arrival
+// counter that only grows plus a generation word; its wait is bounded like every wait of the library: a CTA that
+// gives up raises XKV_FLAG_TIMEOUT and the abort word, and every other CTA leaves at its next wait.
+constexpr int kJacobiCoopThreads = 512;
+constexpr unsigned kJacobiSpinLimit = 1u << 18;   // polls of a barrier that normally opens within microseconds
+
+struct JacobiSync {          // words of the workspace's flag block
+  unsigned int* flags;       // status word
+  unsigned int* count;       // arrivals so far (monotonic)
+  unsigned int* gen;         // barriers completed
+  unsigned int* abort;       // a CTA gave up
+};
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned int* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-__global__ void __launch_bounds__(1024)
-jacobi_check_kernel(const float* __restrict__ M, int l, int* __restrict__ done) {
-  __shared__ float red[64];
-  if (*done) return;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float off = 0.0f, all = 0.0f;
-  for (int e = tid; e < l * l; e += 1024) {
-    const float v = M[e];
-    all += v * v;
-    if (e / l != e % l) off += v * v;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) { off += __shfl_xor_sync(0xffffffffu, off, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
-  if (lane == 0) { red[warp] = off; red[32 + warp] = all; }
+// Returns false when the barrier was abandoned (by this CTA or another one).  `my_gen` counts this CTA's barriers.
+__device__ __forceinline__ bool jacobi_grid_barrier(const JacobiSync& sy, unsigned& my_gen, int* ok_s) {
   __syncthreads();
-  if (tid == 0) {
-    float o2 = 0.0f, a2 = 0.0f;
-    for (int w = 0; w < 32; ++w) { o2 += red[w]; a2 += red[32 + w]; }
-    if (o2 <= 1e-13f * a2) *done = 1;
-  }
-}
-
-__global__ void jacobi_rot_kernel(const float* __restrict__ M, int l, int t, float2* __restrict__ cs, int2* __restrict__ pq,
-                                  const int* __restrict__ done) {
-  if (*done) return;
-  const int n = (l + 1) & ~1, np = n / 2;
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= np) return;
-  int p, q;
-  if (k == 0) { p = n - 1; q = t; }
-  else { p = (t + k) % (n - 1); q = (t - k + n - 1) % (n - 1); }
-  if (p > q) { const int x = p; p = q; q = x; }
-  float c = 1.0f, s = 0.0f;
-  if (q < l) {
-    const float app = M[(size_t)p * l + p], aqq = M[(size_t)q * l + q], apq = M[(size_t)p * l + q];
-    if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * sqrtf(fabsf(app * aqq))) {
-      const float tau = (aqq - app) / (2.0f * apq);
-      const float tt = (tau >= 0.0f ? 1.0f : -1.0f) / (fabsf(tau) + sqrtf(1.0f + tau * tau));
-      c = rsqrtf(1.0f + tt * tt);
-      s = tt * c;
+  if (threadIdx.x == 0) {
+    ++my_gen;
+    __threadfence();
+    bool ok = true;
+    if (atomicAdd(sy.count, 1u) == gridDim.x * my_gen - 1u) {
+      st_release_u32(sy.gen, my_gen);                      // last to arrive: open the barrier
+    } else {
+      unsigned i = 0;
+      while (ld_acquire_u32(sy.gen) < my_gen) {
+        if (++i >= kJacobiSpinLimit || ld_acquire_u32(sy.abort) != 0u) { ok = false; break; }
+      }
     }
-  } else {
-    q = -1;                                           // the padding index: nothing to rotate
+    if (!ok) { atomicOr(sy.flags, XKV_FLAG_TIMEOUT); atomicExch(sy.abort, 1u); }
+    __threadfence();
+    *ok_s = ok ? 1 : 0;
   }
-  cs[k] = make_float2(c, s);
-  pq[k] = make_int2(p, q);
+  __syncthreads();
+  return *ok_s != 0;
 }
 
-// columns p, q of M and of P, every row
-__global__ void jacobi_cols_kernel(float* __restrict__ M, float* __restrict__ P, int l, const float2* __restrict__ cs,
-                                   const int2* __restrict__ pq, const int* __restrict__ done) {
-  if (*done) return;
-  const int np = ((l + 1) & ~1) / 2;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= l * np) return;
-  const int i = e / np, k = e - i * np;
-  const int2 ix = pq[k];
-  const float2 r = cs[k];
-  if (ix.y < 0 || r.y == 0.0f) return;
-  float* row = M + (size_t)i * l;
-  const float x = row[ix.x], y = row[ix.y];
-  row[ix.x] = r.x * x - r.y * y;
-  row[ix.y] = r.y * x + r.x * y;
-  float* prow = P + (size_t)i * l;
-  const float u = prow[ix.x], v = prow[ix.y];
-  prow[ix.x] = r.x * u - r.y * v;
-  prow[ix.y] = r.y * u + r.x * v;
-}
-
-// rows p, q of M, every column
-__global__ void jacobi_rows_kernel(float* __restrict__ M, int l, const float2* __restrict__ cs, const int2* __restrict__ pq,
-                                   const int* __restrict__ done) {
-  if (*done) return;
-  const int np = ((l + 1) & ~1) / 2;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= np * l) return;
-  const int k = e / l, j = e - k * l;
-  const int2 ix = pq[k];
-  const float2 r = cs[k];
-  if (ix.y < 0 || r.y == 0.0f) return;
-  const float x = M[(size_t)ix.x * l + j], y = M[(size_t)ix.y * l + j];
-  M[(size_t)ix.x * l + j] = r.x * x - r.y * y;
-  M[(size_t)ix.y * l + j] = r.y * x + r.x * y;
+__global__ void __launch_bounds__(kJacobiCoopThreads, 1)
+jacobi_coop_kernel(float* __restrict__ M0, float* __restrict__ M1, float* __restrict__ P0, float* __restrict__ P1, int l,
+                   float2* __restrict__ partial, JacobiSync sy) {
+  __shared__ float2 cs_s[kJacobiMaxPairs];
+  __shared__ int2 pq_s[kJacobiMaxPairs];
+  __shared__ int ok_s;
+  __shared__ float2 red_s[kJacobiCoopThreads / 32];
+  __shared__ int done_s;
+  const int tid = threadIdx.x, nb = gridDim.x;
+  const int np = l / 2;                                   // l is even (a multiple of 64)
+  const long long gtid = (long long)blockIdx.x * kJacobiCoopThreads + tid, gstride = (long long)nb * kJacobiCoopThreads;
+  unsigned my_gen = 0;
+  for (long long e = gtid; e < (long long)l * l; e += gstride) P0[e] = (e / l == e % l) ? 1.0f : 0.0f;
+  int cur = 0;
+  bool alive = jacobi_grid_barrier(sy, my_gen, &ok_s);
+  for (int sweep = 0; alive && sweep < kJacobiSweeps; ++sweep) {
+    // ---- off-diagonal weight of M: per-CTA partial sums, then every CTA adds them up in the same order
+    {
+      const float* M = cur ? M1 : M0;
+      float off = 0.0f, all = 0.0f;
+      for (long long e = gtid; e < (long long)l * l; e += gstride) {
+        const float v = __ldcg(M + e);
+        all += v * v;
+        if (e / l != e % l) off += v * v;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) { off += __shfl_xor_sync(0xffffffffu, off, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
+      if ((tid & 31) == 0) red_s[tid >> 5] = make_float2(off, all);
+      __syncthreads();
+      if (tid == 0) {
+        float o2 = 0.0f, a2 = 0.0f;
+        for (int w = 0; w < kJacobiCoopThreads / 32; ++w) { o2 += red_s[w].x; a2 += red_s[w].y; }
+        partial[(sweep & 1) * nb + blockIdx.x] = make_float2(o2, a2);
+      }
+      alive = jacobi_grid_barrier(sy, my_gen, &ok_s);
+      if (!alive) break;
+      if (tid == 0) {
+        float o2 = 0.0f, a2 = 0.0f;
+        for (int b = 0; b < nb; ++b) { const float2 v = __ldcg(partial + (sweep & 1) * nb + b); o2 += v.x; a2 += v.y; }
+        done_s = (o2 <= 1e-13f * a2) ? 1 : 0;
+      }
+      __syncthreads();
+      if (done_s) break;                                  // the same decision in every CTA
+    }
+    for (int t = 0; alive && t < l - 1; ++t) {
+      const float* M = cur ? M1 : M0;
+      const float* P = cur ? P1 : P0;
+      float* Mn = cur ? M0 : M1;
+      float* Pn = cur ? P0 : P1;
+      for (int k = tid; k < np; k += kJacobiCoopThreads) {
+        int p, q;
+        if (k == 0) { p = l - 1; q = t; }
+        else { p = (t + k) % (l - 1); q = (t - k + l - 1) % (l - 1); }
+        if (p > q) { const int x = p; p = q; q = x; }
+        float c = 1.0f, sn = 0.0f;
+        const float app = __ldcg(M + (size_t)p * l + p), aqq = __ldcg(M + (size_t)q * l + q), apq = __ldcg(M + (size_t)p * l + q);
+        if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * sqrtf(fabsf(app * aqq))) {
+          const float tau = (aqq - app) / (2.0f * apq);
+          const float tt = (tau >= 0.0f ? 1.0f : -1.0f) / (fabsf(tau) + sqrtf(1.0f + tau * tau));
+          c = rsqrtf(1.0f + tt * tt);
+          sn = tt * c;
+        }
+        cs_s[k] = make_float2(c, sn);
+        pq_s[k] = make_int2(p, q);
+      }
+      __syncthreads();
+      // M: 2 x 2 blocks (pair a of rows, pair b of columns)
+      for (long long it = gtid; it < (long long)np * np; it += gstride) {
+        const int ka = (int)(it / np), kb = (int)(it - (long long)ka * np);
+        const int2 ra = pq_s[ka], cb = pq_s[kb];
+        const float2 ja = cs_s[ka], jb = cs_s[kb];
+        const float* r0 = M + (size_t)ra.x * l;
+        const float* r1 = M + (size_t)ra.y * l;
+        float x0 = __ldcg(r0 + cb.x), y0 = __ldcg(r0 + cb.y), x1 = __ldcg(r1 + cb.x), y1 = __ldcg(r1 + cb.y);
+        if (jb.y != 0.0f) {                               // columns p_b, q_b
+          const float u0 = jb.x * x0 - jb.y * y0, v0 = jb.y * x0 + jb.x * y0;
+          const float u1 = jb.x * x1 - jb.y * y1, v1 = jb.y * x1 + jb.x * y1;
+          x0 = u0; y0 = v0; x1 = u1; y1 = v1;
+        }
+        if (ja.y != 0.0f) {                               // rows p_a, q_a
+          const float u0 = ja.x * x0 - ja.y * x1, u1 = ja.y * x0 + ja.x * x1;
+          const float v0 = ja.x * y0 - ja.y * y1, v1 = ja.y * y0 + ja.x * y1;
+          x0 = u0; x1 = u1; y0 = v0; y1 = v1;
+        }
+        float* w0 = Mn + (size_t)ra.x * l;
+        float* w1 = Mn + (size_t)ra.y * l;
+        w0[cb.x] = x0; w0[cb.y] = y0; w1[cb.x] = x1; w1[cb.y] = y1;
+      }
+      // P: column pairs, every row
+      for (long long it = gtid; it < (long long)l * np; it += gstride) {
+        const int i = (int)(it / np), k = (int)(it - (long long)i * np);
+        const int2 ix = pq_s[k];
+        const float2 j = cs_s[k];
+        const float u = __ldcg(P + (size_t)i * l + ix.x), v = __ldcg(P + (size_t)i * l + ix.y);
+        float nu = u, nv = v;
+        if (j.y != 0.0f) { nu = j.x * u - j.y * v; nv = j.y * u + j.x * v; }
+        Pn[(size_t)i * l + ix.x] = nu;
+        Pn[(size_t)i * l + ix.y] = nv;
+      }
+      alive = jacobi_grid_barrier(sy, my_gen, &ok_s);
+      cur ^= 1;
+    }
+  }
+  if (alive && cur == 1) {                                // the callers read buffer 0
+    for (long long e = gtid; e < (long long)l * l; e += gstride) { M0[e] = __ldcg(M1 + e); P0[e] = __ldcg(P1 + e); }
+  }
 }
 
 // The r largest eigenvalues (ties to the lower index) and their eigenvectors as the columns of Psel (l x r);
@@ -475,7 +542,7 @@ __global__ void symmetrize_kernel(float* __restrict__ M, int l) {
 
 struct ClfPlan {
   int T, Tp, N, r, l, q;
-  size_t off_flags, off_zb, off_yt, off_u, off_z, off_g, off_m, off_p, off_ps, off_v, off_vb, off_cs, off_pq, total;
+  size_t off_flags, off_zb, off_yt, off_u, off_z, off_g, off_m, off_p, off_ps, off_v, off_vb, off_cs, off_m2, off_p2, total;
 };
 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -498,8 +565,9 @@ bool make_plan(const xkv_clf_config* c, ClfPlan* p) {
   p->off_ps = o; o = align_up(o + (size_t)p->l * p->r * 4);
   p->off_v = o; o = align_up(o + (size_t)p->N * p->r * 4);
   p->off_vb = o; o = align_up(o + (size_t)p->N * p->r * 2);
-  p->off_cs = o; o = align_up(o + (size_t)kJacobiMaxPairs * 8);
-  p->off_pq = o; o = align_up(o + (size_t)kJacobiMaxPairs * 8);
+  p->off_cs = o; o = align_up(o + (size_t)2 * 1024 * 8);            // per-CTA partial sums of the Jacobi convergence check
+  p->off_m2 = o; o = align_up(o + (size_t)p->l * p->l * 4);      // second buffers of the one-kernel Jacobi sweeps
+  p->off_p2 = o; o = align_up(o + (size_t)p->l * p->l * 4);
   p->total = o;
   return true;
 }
@@ -570,9 +638,6 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   float* U = (float*)(w + p.off_u);
   float* Z = (float*)(w + p.off_z);
   double* Gm = (double*)(w + p.off_g);
-  float2* jcs = (float2*)(w + p.off_cs);
-  int2* jpq = (int2*)(w + p.off_pq);
-  int* jdone = (int*)(flags + 1);
   float* Mm = (float*)(w + p.off_m);
   float* Pm = (float*)(w + p.off_p);
   float* Ps = (float*)(w + p.off_ps);
@@ -629,23 +694,30 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   if (e == cudaSuccess) {
     sgemm_small_kernel<true, float><<<g_ll, 256, 0, s>>>(Z, U, Mm, l, l, N, l, l, l);
     symmetrize_kernel<<<(l * l + 255) / 256, 256, 0, s>>>(Mm, l);
-    jacobi_init_kernel<<<(l * l + 255) / 256, 256, 0, s>>>(Pm, l, jdone);
-    const int n_even = (l + 1) & ~1, np = n_even / 2;
-    for (int sweep = 0; sweep < kJacobiSweeps; ++sweep) {
-      jacobi_check_kernel<<<1, 1024, 0, s>>>(Mm, l, jdone);
-      for (int t = 0; t < n_even - 1; ++t) {
-        jacobi_rot_kernel<<<(np + 127) / 128, 128, 0, s>>>(Mm, l, t, jcs, jpq, jdone);
-        jacobi_cols_kernel<<<(l * np + 255) / 256, 256, 0, s>>>(Mm, Pm, l, jcs, jpq, jdone);
-        jacobi_rows_kernel<<<(l * np + 255) / 256, 256, 0, s>>>(Mm, l, jcs, jpq, jdone);
+    {
+      int per_sm = 0, sms = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_coop_kernel, kJacobiCoopThreads, 0);
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+      if (e == cudaSuccess && per_sm < 1) e = cudaErrorLaunchOutOfResources;
+      if (e == cudaSuccess) {
+        float* M2 = (float*)(w + p.off_m2);
+        float* P2 = (float*)(w + p.off_p2);
+        float2* partial = (float2*)(w + p.off_cs);
+        JacobiSync sy{flags, flags + 8, flags + 9, flags + 10};      // zeroed with the flag block above
+        int l_arg = l;
+        void* args[] = {&Mm, &M2, &Pm, &P2, &l_arg, &partial, &sy};
+        e = cudaLaunchCooperativeKernel((const void*)jacobi_coop_kernel, dim3(sms), dim3(kJacobiCoopThreads), args, 0, s);
+        count_launch(kFamClf, 1);
       }
-      count_launch(kFamClf, 1 + 3 * (n_even - 1));
     }
-    eig_select_kernel<<<1, 1024, (size_t)l * sizeof(int), s>>>(Mm, Pm, l, r, Ps, sigma);
-    sgemm_small_kernel<false, float><<<dim3((r + 63) / 64, (N + 63) / 64), 256, 0, s>>>(Z, Ps, V, N, r, l, l, r, r);
-    const long long tot = (long long)N * r;
-    clf_finish_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(V, c->G, c->d, r, Vb, (__nv_bfloat16*)B_out);
-    count_launch(kFamClf, 6);
-    e = cudaGetLastError();
+    if (e == cudaSuccess) {
+      eig_select_kernel<<<1, 1024, (size_t)l * sizeof(int), s>>>(Mm, Pm, l, r, Ps, sigma);
+      sgemm_small_kernel<false, float><<<dim3((r + 63) / 64, (N + 63) / 64), 256, 0, s>>>(Z, Ps, V, N, r, l, l, r, r);
+      const long long tot = (long long)N * r;
+      clf_finish_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(V, c->G, c->d, r, Vb, (__nv_bfloat16*)B_out);
+      count_launch(kFamClf, 5);
+      e = cudaGetLastError();
+    }
   }
   // A = X V_bf16, stored [T][r]
   if (e == cudaSuccess) e = launch_gemm<true>(Vb, N, r, r, X, T, N, N, nullptr, (__nv_bfloat16*)A_out, r, flags, device, s);
