@@ -335,7 +335,8 @@ XKV_API uint64_t xkv_kernel_launch_count(void);
 #define XKV_KERNEL_PREP 8      /* handle set-up: repacking, rotary tables */
 #define XKV_KERNEL_DENSE 9     /* merge of dense-attention partials (xkv_dense_attend) */
 #define XKV_KERNEL_CLF 10      /* cross-layer factorisation (xkv_clf_factorize) */
-#define XKV_KERNEL_FAMILIES 11
+#define XKV_KERNEL_MERGE_MULTI 11 /* the same merge with one CTA per group of query heads (windows of many problems) */
+#define XKV_KERNEL_FAMILIES 12
 XKV_API int xkv_debug_launch_counts(uint64_t* counts);
 
 /*

@@ -1061,6 +1061,160 @@ merge_segments_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __r
   }
 }
 
+// The same merge for windows with many problems: one CTA per (problem, group of HG query heads), 512 threads.
+// With one CTA per head a window of 128 problems x 7 heads is six waves of CTAs that each read the problem's B_v
+// block again; here every B_v row a thread fetches serves all HG heads.  Same arithmetic per head as above; the
+// sum over the rows of B_v is folded by one shuffle and one pass through shared memory.
+constexpr int kMergeMultiThreads = 512;
+template <int DH, int HG>
+__global__ void __launch_bounds__(kMergeMultiThreads)
+merge_segments_multi_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+  extern __shared__ float m_s[];                      // [HG][r4] weighted sums of basis rows, [HG][warps][DH] partial outputs
+  __shared__ float wgt_s[HG][kMergeMaxSeg];
+  __shared__ float twgt_s[HG][kTailMaxSplit];
+  __shared__ float ML_s[HG][2];
+  constexpr int TPR = DH / 8, RPP = kMergeMultiThreads / TPR, NW = kMergeMultiThreads / 32;
+  const int n_rep = dev.n_rep, r = dev.r_v, r4 = (r + 3) & ~3;
+  float* w_s = m_s;
+  float* red = m_s + HG * r4;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ngrp = (n_rep + HG - 1) / HG;
+  const int h0 = (blockIdx.x % ngrp) * HG, py = blockIdx.x / ngrp;
+  const int nh = min(HG, n_rep - h0);
+  const int per_layer = dev.batch * dev.H_kv;
+  const int g = py % dev.H_kv, b = (py / dev.H_kv) % dev.batch, l = sc.l0 + py / per_layer;
+  const long long prob = ((long long)l * dev.batch + b) * dev.H_kv + g;
+  const long long first = (long long)py * sc.tpp;
+  const int c0 = cta_of_tile(first, sc.n_ctas, sc.n_tiles), c1 = cta_of_tile(first + sc.tpp - 1, sc.n_ctas, sc.n_tiles);
+  const int nseg = min(c1 - c0 + 1, kMergeMaxSeg);
+  const size_t stride = (size_t)n_rep * (r + 2);
+  const int rg = tid / TPR, dg = tid % TPR;
+  const size_t ld = (size_t)dev.H_kv * DH;
+  const __nv_bfloat16* Bv = dev.B_v + (((size_t)b * dev.G + l) * r) * ld + (size_t)g * DH + dg * 8;
+  constexpr int kPre = HG <= 4 ? 8 : 4;               // rows of B_v requested before the partials are waited for
+  uint4 pre[kPre];
+#pragma unroll
+  for (int i = 0; i < kPre; ++i) {
+    const int m = rg + i * RPP;
+    pre[i] = m < r ? *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld) : make_uint4(0, 0, 0, 0);
+  }
+  grid_dependency_wait();
+  grid_dependency_launch();
+  const float* part0 = dev.part + ((size_t)prob * sc.n_slots) * stride + (size_t)h0 * (r + 2);
+  const int nts = tail.part ? min(tail.n_split, kTailMaxSplit) : 0;
+  const size_t tstride = (size_t)n_rep * (DH + 2);
+  const float* tpart0 = tail.part ? tail.part + ((size_t)py * tail.n_split) * tstride + (size_t)h0 * (DH + 2) : nullptr;
+  if (warp < nh) {                                    // warp h: maxima, weights of the segments, denominator of head h0 + h
+    const float* part = part0 + (size_t)warp * (r + 2);
+    const float* tpart = tpart0 ? tpart0 + (size_t)warp * (DH + 2) : nullptr;
+    constexpr int kPer = (kMergeMaxSeg + 31) / 32;
+    float sm[kPer], sl[kPer];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int sg = lane + 32 * i;
+      sm[i] = sg < nseg ? __ldcg(part + sg * stride + r) : -INFINITY;
+      sl[i] = sg < nseg ? __ldcg(part + sg * stride + r + 1) : 0.0f;
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) mx = fmaxf(mx, sm[i]);
+    for (int sg = lane; sg < nts; sg += 32) mx = fmaxf(mx, tpart[sg * tstride + DH]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float Ls = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int sg = lane + 32 * i;
+      if (sg < nseg) {
+        const float w = (sm[i] == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(sm[i] - mx);
+        wgt_s[warp][sg] = w;
+        Ls += w * sl[i];
+      }
+    }
+    for (int sg = lane; sg < nts; sg += 32) {
+      const float ms = tpart[sg * tstride + DH];
+      const float w = (ms == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(ms - mx);
+      twgt_s[warp][sg] = w;
+      Ls += w * tpart[sg * tstride + DH + 1];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
+    if (lane == 0) { ML_s[warp][0] = mx; ML_s[warp][1] = Ls; }
+  }
+  __syncthreads();
+  // weighted sums of the segments' partial sums, one rank column per thread and pass, segments in ascending order
+  for (int col = tid; col < r; col += kMergeMultiThreads) {
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+      if (h < nh) {
+        const float* part = part0 + (size_t)h * (r + 2) + col;
+        float acc = 0.0f;
+#pragma unroll 4
+        for (int sg = 0; sg < nseg; ++sg) acc = fmaf(wgt_s[h][sg], __ldcg(part + sg * stride), acc);
+        w_s[h * r4 + col] = acc;
+      }
+    }
+  }
+  __syncthreads();
+  float acc[HG][8];
+#pragma unroll
+  for (int h = 0; h < HG; ++h)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[h][e] = 0.0f;
+  auto add_row = [&](const uint4& v, int m) {
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+    float x[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(u[e] << 16); x[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u); }
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+      const float w = h < nh ? w_s[h * r4 + m] : 0.0f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[h][e] = fmaf(w, x[e], acc[h][e]);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kPre; ++i) {
+    const int m = rg + i * RPP;
+    if (m < r) add_row(pre[i], m);
+  }
+#pragma unroll 2
+  for (int m = rg + kPre * RPP; m < r; m += RPP) add_row(*reinterpret_cast<const uint4*>(Bv + (size_t)m * ld), m);
+  // a warp holds two row groups (lanes 0..15 and 16..31 with the same columns): fold them, then one partial per warp
+#pragma unroll
+  for (int h = 0; h < HG; ++h)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[h][e] += __shfl_xor_sync(0xffffffffu, acc[h][e], TPR);
+  static_assert(TPR == 16 || TPR == 8, "row groups per warp");
+  if constexpr (TPR == 8) {
+#pragma unroll
+    for (int h = 0; h < HG; ++h)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[h][e] += __shfl_xor_sync(0xffffffffu, acc[h][e], 16);
+  }
+  if (lane < TPR) {
+#pragma unroll
+    for (int h = 0; h < HG; ++h)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) red[(h * NW + warp) * DH + lane * 8 + e] = acc[h][e];
+  }
+  __syncthreads();
+  for (int o = tid; o < nh * DH; o += kMergeMultiThreads) {
+    const int h = o / DH, d = o - h * DH;
+    float v = 0.0f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) v += red[(h * NW + w) * DH + d];
+    if (tpart0) {
+      const float* tpart = tpart0 + (size_t)h * (DH + 2);
+      for (int sg = 0; sg < nts; ++sg) v = fmaf(twgt_s[h][sg], tpart[sg * tstride + d], v);
+    }
+    const float M = ML_s[h][0], L = ML_s[h][1];
+    const long long qh = ((long long)l * dev.batch + b) * dev.H_q + (long long)g * n_rep + h0 + h;
+    out[qh * DH + d] = __float2bfloat16(L > 0.0f ? v / L : 0.0f);
+    if (lse && d == 0) lse[qh] = L > 0.0f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
+}
+
 template <int DH, int NR>
 constexpr size_t fused_smem_bytes() {
   return 1024 + (size_t)(ring_slots<DH, NR>() + kNB) * kSlabBytes + misc_smem_bytes<DH, NR>();
@@ -1106,12 +1260,24 @@ cudaError_t launch_fused_t(const xkv_group* grp, int l0, int l1, const __nv_bflo
   }
   count_launch(kFamFused);
   if (e != cudaSuccess) return e;
-  const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
-  e = ensure_dyn_smem<merge_segments_kernel<DH>>(msmem, grp->device);
+  // one CTA per query head while those CTAs fit the SMs about twice over; beyond that one CTA per group of heads
+  constexpr int HG = NR <= 4 ? 4 : 8;
+  bool multi = false;
+  if ((long long)problems * dev.n_rep <= 2LL * grp->sm_count) {
+    const size_t msmem = sizeof(float) * (((size_t)dev.r_v + 3) / 4 * 4 + (size_t)(kMergeThreads / (DH / 8)) * DH);
+    e = ensure_dyn_smem<merge_segments_kernel<DH>>(msmem, grp->device);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, tail, out, lse);
+  } else {
+    const size_t msmem = sizeof(float) * ((size_t)HG * (((size_t)dev.r_v + 3) / 4 * 4) + (size_t)HG * (kMergeMultiThreads / 32) * DH);
+    const int ngrp = (dev.n_rep + HG - 1) / HG;
+    e = ensure_dyn_smem<merge_segments_multi_kernel<DH, HG>>(msmem, grp->device);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(merge_segments_multi_kernel<DH, HG>, dim3(problems * ngrp), dim3(kMergeMultiThreads), msmem, s, dev, sc, tail, out, lse);
+    multi = true;
+  }
   if (e != cudaSuccess) return e;
-  e = launch_pdl(merge_segments_kernel<DH>, dim3(problems * dev.n_rep), dim3(kMergeThreads), msmem, s, dev, sc, tail, out, lse);
-  if (e != cudaSuccess) return e;
-  count_launch(kFamMerge);
+  count_launch(multi ? kFamMergeMulti : kFamMerge);
   return cudaGetLastError();
 }
 

@@ -94,7 +94,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 enum KernelFamily {
   kFamScan = XKV_KERNEL_SCAN, kFamTopk = XKV_KERNEL_TOPK, kFamFused = XKV_KERNEL_FUSED, kFamMerge = XKV_KERNEL_MERGE,
   kFamTile = XKV_KERNEL_TILE, kFamTailTc = XKV_KERNEL_TAIL_TC, kFamTailCuda = XKV_KERNEL_TAIL_CUDA,
-  kFamLandmarks = XKV_KERNEL_LANDMARKS, kFamPrep = XKV_KERNEL_PREP, kFamDense = XKV_KERNEL_DENSE, kFamClf = XKV_KERNEL_CLF, kFamCount = XKV_KERNEL_FAMILIES
+  kFamLandmarks = XKV_KERNEL_LANDMARKS, kFamPrep = XKV_KERNEL_PREP, kFamDense = XKV_KERNEL_DENSE, kFamClf = XKV_KERNEL_CLF, kFamMergeMulti = XKV_KERNEL_MERGE_MULTI,
+  kFamCount = XKV_KERNEL_FAMILIES
 };
 void count_launch(KernelFamily family, int n = 1);
 
@@ -107,7 +108,17 @@ inline cudaError_t ensure_dyn_smem(size_t bytes, int device) {
   static std::atomic<size_t> have[kMaxDevices];
   if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
   if (have[device].load(std::memory_order_acquire) >= bytes && bytes > 0) return cudaSuccess;
-  if (bytes <= 48 * 1024) return cudaSuccess;          // the default limit covers it
+  // the default limit of 48 KB covers static and dynamic shared memory together
+  static std::atomic<long> static_bytes{-1};
+  long st = static_bytes.load(std::memory_order_acquire);
+  if (st < 0) {
+    cudaFuncAttributes attr;
+    const cudaError_t ea = cudaFuncGetAttributes(&attr, Kernel);
+    if (ea != cudaSuccess) return ea;
+    st = (long)attr.sharedSizeBytes;
+    static_bytes.store(st, std::memory_order_release);
+  }
+  if (bytes + (size_t)st <= 48 * 1024) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) have[device].store(bytes, std::memory_order_release);
   return e;

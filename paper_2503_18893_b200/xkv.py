@@ -121,7 +121,7 @@ _lib.xkv_debug_set_fault_injection.argtypes = [_P, ctypes.c_uint32]
 _lib.xkv_debug_set_fault_injection.restype = ctypes.c_int
 
 XKV_KERNEL_FAMILIES = ("scan", "topk", "fused", "merge", "tile", "tail_tc", "tail_cuda", "landmarks", "prep", "dense",
-                       "clf")
+                       "clf", "merge_multi")
 XKV_FLAG_CLF_BREAKDOWN = 4
 XKV_INJECT_SCAN_NO_LOAD = 1
 XKV_INJECT_FUSED_NO_B = 2
