@@ -82,7 +82,7 @@ __device__ __forceinline__ void score_pass(uint32_t tile, const float* __restric
 }
 
 // grid.x = ceil(n_c / kScoreRows) tiles, grid.y = (layers in call) * batch * H_kv problems.
-template <int DH>
+template <int DH, int HMAX>
 __global__ void __launch_bounds__(kScoreThreads)
 score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const __nv_bfloat16* __restrict__ q,
                   int l0) {
@@ -136,9 +136,17 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
   }
   float best0 = -INFINITY, best1 = -INFINITY;
   const int row0 = threadIdx.x;
-  for (int h0 = 0; h0 < dev.n_rep; h0 += 4) {
-    const int hb = min(4, dev.n_rep - h0);
+  // heads in passes of HMAX: a pass reads the tile once for all its heads.  The kernel for up to four heads per
+  // KV head is kept apart from the wider one: its code is smaller, and the scan is sensitive to that.
+  for (int h0 = 0; h0 < dev.n_rep; h0 += HMAX) {
+    const int hb = min(HMAX, dev.n_rep - h0);
     const float* qh = qs + h0 * DH;
+    if constexpr (HMAX == 8) {
+      if (hb == 8) { score_pass<DH, 8>(tile, qh, row0, dev.sel_scale, best0, best1); continue; }
+      if (hb == 7) { score_pass<DH, 7>(tile, qh, row0, dev.sel_scale, best0, best1); continue; }
+      if (hb == 6) { score_pass<DH, 6>(tile, qh, row0, dev.sel_scale, best0, best1); continue; }
+      if (hb == 5) { score_pass<DH, 5>(tile, qh, row0, dev.sel_scale, best0, best1); continue; }
+    }
     if (hb == 4) score_pass<DH, 4>(tile, qh, row0, dev.sel_scale, best0, best1);
     else if (hb == 3) score_pass<DH, 3>(tile, qh, row0, dev.sel_scale, best0, best1);
     else if (hb == 2) score_pass<DH, 2>(tile, qh, row0, dev.sel_scale, best0, best1);
@@ -881,15 +889,18 @@ static cudaError_t launch_select_dev(const GroupDev& dev, const CUtensorMap& tma
   const size_t smem = 1024 + (size_t)(dev.d_h / 64) * kScoreRows * 128 + (size_t)dev.n_rep * dev.d_h * 4;
   dim3 grid(tiles, problems);
   cudaError_t e;
+#define XKV_SCAN(DH, HMAX)                                                                              \
+  do {                                                                                                  \
+    e = ensure_dyn_smem<score_pool_kernel<DH, HMAX>>(smem, device);                                     \
+    if (e != cudaSuccess) return e;                                                                     \
+    e = launch_pdl(score_pool_kernel<DH, HMAX>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0); \
+  } while (0)
   if (dev.d_h == 128) {
-    e = ensure_dyn_smem<score_pool_kernel<128>>(smem, device);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(score_pool_kernel<128>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
+    if (dev.n_rep <= 4) XKV_SCAN(128, 4); else XKV_SCAN(128, 8);
   } else {
-    e = ensure_dyn_smem<score_pool_kernel<64>>(smem, device);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(score_pool_kernel<64>, grid, dim3(kScoreThreads), smem, s, tmap, dev, q, l0);
+    if (dev.n_rep <= 4) XKV_SCAN(64, 4); else XKV_SCAN(64, 8);
   }
+#undef XKV_SCAN
   count_launch(kFamScan);
   if (e != cudaSuccess) return e;
   e = launch_topk(dev, device, problems, l0, k_ch, k_cap, dev.outliers, dev.n_out, 0.0f, sel_idx, sel_cnt, s);
