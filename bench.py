@@ -345,6 +345,7 @@ def run_clf(args):
         if i >= args.warmup:
             ts.append(e0.elapsed_time(e1))
     st, flags = xkv.xkv_clf_status(ws)
+    jacobi_sweeps = int(ws[:256].view(torch.int32)[11].item())       # diagnostic word of the workspace's flag block
     # residual against the optimum
     N = s.G * s.d
     gram = torch.zeros((N, N), dtype=torch.float64, device="cuda")
@@ -364,7 +365,7 @@ def run_clf(args):
                       "residual_over_optimum": res / optimum, "relative_residual": res / float(ev.sum()),
                       "orthonormality_max_dev": float((Vm @ Vm.T - torch.eye(r, device="cuda", dtype=torch.float64)).abs().max()),
                       "sigma_max_rel_err": float(((sig.double() - ev[:r].sqrt()).abs() / ev[0].sqrt()).max()),
-                      "status": st, "flags": flags}))
+                      "jacobi_sweeps": jacobi_sweeps, "status": st, "flags": flags}))
     return 0
 
 

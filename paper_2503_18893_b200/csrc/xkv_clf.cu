@@ -195,7 +195,7 @@ sgemm_small_kernel(const float* __restrict__ A, const float* __restrict__ B, TO*
     }
 }
 
-// C (m x n, fp64) = A^T B for fp32 A (k x m) and B (k x n) on the fp64 tensor-core path (mma.sync m8n8k4): the Gram
+// C (m x n, fp64 or rounded to fp32) = A^T B for fp32 A (k x m) and B (k x n) on the fp64 tensor-core path (mma.sync m8n8k4): the Gram
 // matrices of the Cholesky QR, accumulated in fp64 because their condition number is the square of the iterate's.
 // (A scalar fp64 kernel with 4 x 4 outputs per thread spent 0.79 ms on a 576 x 576 x 4096 product, this one 0.33 ms.)  64 x 64 tiles, 8 warps of 16 x 32, chunks of 32 rows
 // widened to fp64 on their way into shared memory; m, n multiples of 64, k a multiple of 32.
@@ -204,8 +204,9 @@ __device__ __forceinline__ void dmma_8x8x4(double (&d)[2], double a, double b) {
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
 }
+template <typename TO>
 __global__ void __launch_bounds__(256)
-dgemm_tn_mma_kernel(const float* __restrict__ A, const float* __restrict__ B, double* __restrict__ C, int k, int lda,
+dgemm_tn_mma_kernel(const float* __restrict__ A, const float* __restrict__ B, TO* __restrict__ C, int k, int lda,
                     int ldb, int ldc) {
   __shared__ double As[32][kDgemmLd], Bs[32][kDgemmLd];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -254,9 +255,9 @@ dgemm_tn_mma_kernel(const float* __restrict__ A, const float* __restrict__ B, do
   for (int i = 0; i < 2; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      double* dst = C + (size_t)(m0 + wm + 8 * i + (lane >> 2)) * ldc + n0 + wn + 8 * j + 2 * (lane & 3);
-      dst[0] = acc[i][j][0];
-      dst[1] = acc[i][j][1];
+      TO* dst = C + (size_t)(m0 + wm + 8 * i + (lane >> 2)) * ldc + n0 + wn + 8 * j + 2 * (lane & 3);
+      dst[0] = (TO)acc[i][j][0];
+      dst[1] = (TO)acc[i][j][1];
     }
 }
 
@@ -380,6 +381,123 @@ trsolve_rows_kernel(const float* __restrict__ U, const double* __restrict__ L, f
   }
 }
 
+// ---- the triangular solve Z = U L^-T in 64-column blocks on the fp64 tensor-core path ----
+// Z[:, J] = (U[:, J] - sum_{I<J} Z[:, I] L[J, I]^T) inv(L[J, J])^T.  The inverses of the 64 x 64 diagonal blocks come
+// from a small kernel (one thread per column of the inverse, forward substitution); the solve keeps 32 rows of Z in
+// fp64 in shared memory per CTA and streams the blocks of L through a 64 x 64 staging tile.
+constexpr int kTriBlock = 64;
+__global__ void __launch_bounds__(kTriBlock)
+tri_inv_diag_kernel(const double* __restrict__ L, int l, double* __restrict__ Xinv) {
+  __shared__ double Xs[kTriBlock][kTriBlock + 1];
+  const int c = threadIdx.x, jb = blockIdx.x * kTriBlock;
+  const double* Lb = L + (size_t)jb * l + jb;
+  for (int j = 0; j < kTriBlock; ++j) {
+    double x = 0.0;
+    if (j >= c) {
+      double s0 = (j == c) ? 1.0 : 0.0, s1 = 0.0;
+      const double* Lj = Lb + (size_t)j * l;
+      int i = c;
+      for (; i + 1 < j; i += 2) { s0 -= Lj[i] * Xs[i][c]; s1 -= Lj[i + 1] * Xs[i + 1][c]; }
+      if (i < j) s0 -= Lj[i] * Xs[i][c];
+      x = (s0 + s1) / Lj[j];
+    }
+    Xs[j][c] = x;                                    // a thread only ever reads its own column
+  }
+  __syncthreads();
+  double* out = Xinv + (size_t)blockIdx.x * kTriBlock * kTriBlock;
+  for (int e = c; e < kTriBlock * kTriBlock; e += kTriBlock) out[e] = Xs[e / kTriBlock][e % kTriBlock];
+}
+
+constexpr int kTriRows = 32;                         // rows of Z per CTA
+__global__ void __launch_bounds__(256)
+trsolve_mma_kernel(const float* __restrict__ U, const double* __restrict__ L, const double* __restrict__ Xinv,
+                   float* __restrict__ Z, __nv_bfloat16* __restrict__ Zb, int n, int l) {
+  extern __shared__ double tri_s[];
+  const int ldz = l + 4;                             // 4 mod 16 doubles: fragment loads are conflict free
+  double* Zs = tri_s;                                // [kTriRows][ldz]
+  double* Ls = tri_s + (size_t)kTriRows * ldz;       // [64][kDgemmLd]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 1) * 16, wn = (warp >> 1) * 16;
+  const int row0 = blockIdx.x * kTriRows;
+  const int fr = lane >> 2, fc = lane & 3;
+  auto stage = [&](const double* src, int ld) {      // 64 x 64 block, row-major
+    for (int e = tid; e < kTriBlock * kTriBlock; e += 256) Ls[(e >> 6) * kDgemmLd + (e & 63)] = src[(size_t)(e >> 6) * ld + (e & 63)];
+  };
+  const int nb = l / kTriBlock;
+  for (int J = 0; J < nb; ++J) {
+    double acc[2][2][2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int r = row0 + wm + 8 * i + fr;
+        const float2 u = r < n ? *reinterpret_cast<const float2*>(U + (size_t)r * l + J * kTriBlock + wn + 8 * j + 2 * fc)
+                               : make_float2(0.0f, 0.0f);
+        acc[i][j][0] = (double)u.x;
+        acc[i][j][1] = (double)u.y;
+      }
+    for (int I = 0; I < J; ++I) {
+      __syncthreads();                               // the staging tile and the last block of Z are free / written
+      stage(L + (size_t)J * kTriBlock * l + (size_t)I * kTriBlock, l);
+      __syncthreads();
+#pragma unroll 4
+      for (int kk = 0; kk < kTriBlock; kk += 4) {
+        double a[2], b[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) a[i] = -Zs[(size_t)(wm + 8 * i + fr) * ldz + I * kTriBlock + kk + fc];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) b[j] = Ls[(wn + 8 * j + fr) * kDgemmLd + kk + fc];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+          for (int j = 0; j < 2; ++j) dmma_8x8x4(acc[i][j], a[i], b[j]);
+      }
+    }
+    __syncthreads();
+    // the right-hand side of the diagonal step goes through the block's own columns of Zs
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        double* d = Zs + (size_t)(wm + 8 * i + fr) * ldz + J * kTriBlock + wn + 8 * j + 2 * fc;
+        d[0] = acc[i][j][0];
+        d[1] = acc[i][j][1];
+        acc[i][j][0] = 0.0;
+        acc[i][j][1] = 0.0;
+      }
+    stage(Xinv + (size_t)J * kTriBlock * kTriBlock, kTriBlock);
+    __syncthreads();
+#pragma unroll 4
+    for (int kk = 0; kk < kTriBlock; kk += 4) {
+      double a[2], b[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) a[i] = Zs[(size_t)(wm + 8 * i + fr) * ldz + J * kTriBlock + kk + fc];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) b[j] = Ls[(wn + 8 * j + fr) * kDgemmLd + kk + fc];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) dmma_8x8x4(acc[i][j], a[i], b[j]);
+    }
+    __syncthreads();                                 // every warp has read the right-hand side
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int rl = wm + 8 * i + fr, col = J * kTriBlock + wn + 8 * j + 2 * fc;
+        double* d = Zs + (size_t)rl * ldz + col;
+        d[0] = acc[i][j][0];
+        d[1] = acc[i][j][1];
+        const int r = row0 + rl;
+        if (r < n) {
+          const float z0 = (float)acc[i][j][0], z1 = (float)acc[i][j][1];
+          *reinterpret_cast<float2*>(Z + (size_t)r * l + col) = make_float2(z0, z1);
+          if (Zb) *reinterpret_cast<__nv_bfloat162*>(Zb + (size_t)r * l + col) = __floats2bfloat162_rn(z0, z1);
+        }
+      }
+  }
+}
+
 }  // namespace
 
 namespace {
@@ -457,6 +575,7 @@ jacobi_coop_kernel(float* __restrict__ M0, float* __restrict__ M1, float* __rest
   for (long long e = gtid; e < (long long)l * l; e += gstride) P0[e] = (e / l == e % l) ? 1.0f : 0.0f;
   int cur = 0;
   bool alive = jacobi_grid_barrier(sy, my_gen, &ok_s);
+  int sweeps_done = 0;
   for (int sweep = 0; alive && sweep < kJacobiSweeps; ++sweep) {
     // ---- off-diagonal weight of M: per-CTA partial sums, then every CTA adds them up in the same order
     {
@@ -486,16 +605,91 @@ jacobi_coop_kernel(float* __restrict__ M0, float* __restrict__ M1, float* __rest
       __syncthreads();
       if (done_s) break;                                  // the same decision in every CTA
     }
+    ++sweeps_done;
     for (int t = 0; alive && t < l - 1; ++t) {
       const float* M = cur ? M1 : M0;
       const float* P = cur ? P1 : P0;
       float* Mn = cur ? M0 : M1;
       float* Pn = cur ? P0 : P1;
-      for (int k = tid; k < np; k += kJacobiCoopThreads) {
+      // pair k of round t (round-robin order), smaller index first
+      auto pair_of = [&](int k) -> int2 {
         int p, q;
         if (k == 0) { p = l - 1; q = t; }
         else { p = (t + k) % (l - 1); q = (t - k + l - 1) % (l - 1); }
-        if (p > q) { const int x = p; p = q; q = x; }
+        return p < q ? make_int2(p, q) : make_int2(q, p);
+      };
+      // M: 2 x 2 blocks (pair a of rows, pair b of columns); P: column pairs, every row; kBatch items of each per
+      // pass.  The loads of the first pass are issued before the rotations are worked out -- their addresses
+      // depend on the round only -- so that a round of a 576 x 576 matrix is one trip to L2, not three.
+      constexpr int kBatch = 4;
+      const long long nM = (long long)np * np, nP = (long long)l * np;
+      float x0[kBatch], y0[kBatch], x1[kBatch], y1[kBatch], pu[kBatch], pv[kBatch];
+      int ka[kBatch], kb[kBatch], pi[kBatch], pk[kBatch];
+      auto load_m = [&](long long base) {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const long long it = base + u * gstride;
+          ka[u] = -1;
+          if (it < nM) {
+            ka[u] = (int)(it / np); kb[u] = (int)(it - (long long)ka[u] * np);
+            const int2 ra = pair_of(ka[u]), cb = pair_of(kb[u]);
+            const float* r0 = M + (size_t)ra.x * l;
+            const float* r1 = M + (size_t)ra.y * l;
+            x0[u] = __ldcg(r0 + cb.x); y0[u] = __ldcg(r0 + cb.y); x1[u] = __ldcg(r1 + cb.x); y1[u] = __ldcg(r1 + cb.y);
+          }
+        }
+      };
+      auto load_p = [&](long long base) {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const long long it = base + u * gstride;
+          pi[u] = -1;
+          if (it < nP) {
+            pi[u] = (int)(it / np); pk[u] = (int)(it - (long long)pi[u] * np);
+            const int2 ix = pair_of(pk[u]);
+            pu[u] = __ldcg(P + (size_t)pi[u] * l + ix.x); pv[u] = __ldcg(P + (size_t)pi[u] * l + ix.y);
+          }
+        }
+      };
+      auto finish_m = [&]() {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          if (ka[u] < 0) continue;
+          const int2 ra = pq_s[ka[u]], cb = pq_s[kb[u]];
+          const float2 ja = cs_s[ka[u]], jb = cs_s[kb[u]];
+          float a0 = x0[u], b0 = y0[u], a1 = x1[u], b1 = y1[u];
+          if (jb.y != 0.0f) {                             // columns p_b, q_b
+            const float u0 = jb.x * a0 - jb.y * b0, v0 = jb.y * a0 + jb.x * b0;
+            const float u1 = jb.x * a1 - jb.y * b1, v1 = jb.y * a1 + jb.x * b1;
+            a0 = u0; b0 = v0; a1 = u1; b1 = v1;
+          }
+          if (ja.y != 0.0f) {                             // rows p_a, q_a
+            const float u0 = ja.x * a0 - ja.y * a1, u1 = ja.y * a0 + ja.x * a1;
+            const float v0 = ja.x * b0 - ja.y * b1, v1 = ja.y * b0 + ja.x * b1;
+            a0 = u0; a1 = u1; b0 = v0; b1 = v1;
+          }
+          float* w0 = Mn + (size_t)ra.x * l;
+          float* w1 = Mn + (size_t)ra.y * l;
+          w0[cb.x] = a0; w0[cb.y] = b0; w1[cb.x] = a1; w1[cb.y] = b1;
+        }
+      };
+      auto finish_p = [&]() {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          if (pi[u] < 0) continue;
+          const int2 ix = pq_s[pk[u]];
+          const float2 j = cs_s[pk[u]];
+          float nu = pu[u], nv = pv[u];
+          if (j.y != 0.0f) { nu = j.x * pu[u] - j.y * pv[u]; nv = j.y * pu[u] + j.x * pv[u]; }
+          Pn[(size_t)pi[u] * l + ix.x] = nu;
+          Pn[(size_t)pi[u] * l + ix.y] = nv;
+        }
+      };
+      load_m(gtid);
+      load_p(gtid);
+      for (int k = tid; k < np; k += kJacobiCoopThreads) {
+        const int2 ix = pair_of(k);
+        const int p = ix.x, q = ix.y;
         float c = 1.0f, sn = 0.0f;
         const float app = __ldcg(M + (size_t)p * l + p), aqq = __ldcg(M + (size_t)q * l + q), apq = __ldcg(M + (size_t)p * l + q);
         if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * sqrtf(fabsf(app * aqq))) {
@@ -505,46 +699,18 @@ jacobi_coop_kernel(float* __restrict__ M0, float* __restrict__ M1, float* __rest
           sn = tt * c;
         }
         cs_s[k] = make_float2(c, sn);
-        pq_s[k] = make_int2(p, q);
+        pq_s[k] = ix;
       }
       __syncthreads();
-      // M: 2 x 2 blocks (pair a of rows, pair b of columns)
-      for (long long it = gtid; it < (long long)np * np; it += gstride) {
-        const int ka = (int)(it / np), kb = (int)(it - (long long)ka * np);
-        const int2 ra = pq_s[ka], cb = pq_s[kb];
-        const float2 ja = cs_s[ka], jb = cs_s[kb];
-        const float* r0 = M + (size_t)ra.x * l;
-        const float* r1 = M + (size_t)ra.y * l;
-        float x0 = __ldcg(r0 + cb.x), y0 = __ldcg(r0 + cb.y), x1 = __ldcg(r1 + cb.x), y1 = __ldcg(r1 + cb.y);
-        if (jb.y != 0.0f) {                               // columns p_b, q_b
-          const float u0 = jb.x * x0 - jb.y * y0, v0 = jb.y * x0 + jb.x * y0;
-          const float u1 = jb.x * x1 - jb.y * y1, v1 = jb.y * x1 + jb.x * y1;
-          x0 = u0; y0 = v0; x1 = u1; y1 = v1;
-        }
-        if (ja.y != 0.0f) {                               // rows p_a, q_a
-          const float u0 = ja.x * x0 - ja.y * x1, u1 = ja.y * x0 + ja.x * x1;
-          const float v0 = ja.x * y0 - ja.y * y1, v1 = ja.y * y0 + ja.x * y1;
-          x0 = u0; x1 = u1; y0 = v0; y1 = v1;
-        }
-        float* w0 = Mn + (size_t)ra.x * l;
-        float* w1 = Mn + (size_t)ra.y * l;
-        w0[cb.x] = x0; w0[cb.y] = y0; w1[cb.x] = x1; w1[cb.y] = y1;
-      }
-      // P: column pairs, every row
-      for (long long it = gtid; it < (long long)l * np; it += gstride) {
-        const int i = (int)(it / np), k = (int)(it - (long long)i * np);
-        const int2 ix = pq_s[k];
-        const float2 j = cs_s[k];
-        const float u = __ldcg(P + (size_t)i * l + ix.x), v = __ldcg(P + (size_t)i * l + ix.y);
-        float nu = u, nv = v;
-        if (j.y != 0.0f) { nu = j.x * u - j.y * v; nv = j.y * u + j.x * v; }
-        Pn[(size_t)i * l + ix.x] = nu;
-        Pn[(size_t)i * l + ix.y] = nv;
-      }
+      finish_m();
+      finish_p();
+      for (long long base = gtid + kBatch * gstride; base < nM; base += kBatch * gstride) { load_m(base); finish_m(); }
+      for (long long base = gtid + kBatch * gstride; base < nP; base += kBatch * gstride) { load_p(base); finish_p(); }
       alive = jacobi_grid_barrier(sy, my_gen, &ok_s);
       cur ^= 1;
     }
   }
+  if (blockIdx.x == 0 && tid == 0) sy.abort[1] = (unsigned)sweeps_done;   // diagnostic: sweeps that ran
   if (alive && cur == 1) {                                // the callers read buffer 0
     for (long long e = gtid; e < (long long)l * l; e += gstride) { M0[e] = __ldcg(M1 + e); P0[e] = __ldcg(P1 + e); }
   }
@@ -606,7 +772,7 @@ __global__ void symmetrize_kernel(float* __restrict__ M, int l) {
 
 struct ClfPlan {
   int T, Tp, N, r, l, q;
-  size_t off_flags, off_zb, off_yt, off_u, off_z, off_g, off_m, off_p, off_ps, off_v, off_vb, off_cs, off_m2, off_p2, total;
+  size_t off_flags, off_zb, off_yt, off_u, off_z, off_g, off_m, off_p, off_ps, off_v, off_vb, off_cs, off_m2, off_p2, off_xinv, total;
 };
 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -632,6 +798,7 @@ bool make_plan(const xkv_clf_config* c, ClfPlan* p) {
   p->off_cs = o; o = align_up(o + (size_t)2 * 1024 * 8);            // per-CTA partial sums of the Jacobi convergence check
   p->off_m2 = o; o = align_up(o + (size_t)p->l * p->l * 4);      // second buffers of the one-kernel Jacobi sweeps
   p->off_p2 = o; o = align_up(o + (size_t)p->l * p->l * 4);
+  p->off_xinv = o; o = align_up(o + (size_t)p->l * kTriBlock * 8);   // inverses of the diagonal blocks of a Cholesky factor
   p->total = o;
   return true;
 }
@@ -722,6 +889,11 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   // whole range between the largest singular value and the noise floor.
   const size_t solve_smem = (size_t)kSolveWarps * l * sizeof(double);
   e = e == cudaSuccess ? ensure_dyn_smem<trsolve_rows_kernel>(solve_smem, device) : e;
+  const size_t tri_smem = ((size_t)kTriRows * (l + 4) + (size_t)kTriBlock * kDgemmLd) * sizeof(double);
+  // the blocked solve keeps 32 rows of Z in shared memory: sketches wider than about 700 columns take the row-wise kernel
+  const bool mma_solve = (getenv("XKV_CLF_SOLVE_ROWS") == nullptr) && tri_smem <= 227u * 1024u;
+  if (mma_solve) e = e == cudaSuccess ? ensure_dyn_smem<trsolve_mma_kernel>(tri_smem, device) : e;
+  double* Xinv = (double*)(w + p.off_xinv);
   // Every pass divides the condition number by about shift^-1/2; the iterate of a power iteration only has to stay
   // well conditioned (two passes), the last one has to be orthonormal (five passes with decreasing shifts: the
   // columns of U that lie in the noise floor are 10^8 times smaller than the leading ones).
@@ -729,7 +901,7 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   auto cholqr = [&](const float* src, int passes) -> cudaError_t {
     for (int pass = 0; pass < passes; ++pass) {
       const float* in = pass == 0 ? src : Z;
-      dgemm_tn_mma_kernel<<<g_ll, 256, 0, s>>>(in, in, Gm, N, l, l, l);
+      dgemm_tn_mma_kernel<double><<<g_ll, 256, 0, s>>>(in, in, Gm, N, l, l, l);
       const double shift_rel = kShifts[pass];
       chol_shift_kernel<<<1, 1024, 0, s>>>(Gm, l, shift_rel);
       int launches = 2;
@@ -745,7 +917,13 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
           launches += 2;
         }
       }
-      trsolve_rows_kernel<<<(N + kSolveWarps - 1) / kSolveWarps, kSolveWarps * 32, solve_smem, s>>>(in, Gm, Z, Zb, N, l);
+      if (!mma_solve) {
+        trsolve_rows_kernel<<<(N + kSolveWarps - 1) / kSolveWarps, kSolveWarps * 32, solve_smem, s>>>(in, Gm, Z, Zb, N, l);
+      } else {
+        tri_inv_diag_kernel<<<l / kTriBlock, kTriBlock, 0, s>>>(Gm, l, Xinv);
+        trsolve_mma_kernel<<<(N + kTriRows - 1) / kTriRows, 256, tri_smem, s>>>(in, Gm, Xinv, Z, Zb, N, l);
+        ++launches;
+      }
       count_launch(kFamClf, launches + 1);
     }
     return cudaGetLastError();
@@ -756,7 +934,7 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   }
   if (e == cudaSuccess) e = two_products();              // W = X Z and U' = X^T W for the Rayleigh-Ritz step
   if (e == cudaSuccess) {
-    sgemm_small_kernel<true, float><<<g_ll, 256, 0, s>>>(Z, U, Mm, l, l, N, l, l, l);
+    dgemm_tn_mma_kernel<float><<<g_ll, 256, 0, s>>>(Z, U, Mm, N, l, l, l);     // M = Z^T U', accumulated in fp64
     symmetrize_kernel<<<(l * l + 255) / 256, 256, 0, s>>>(Mm, l);
     {
       int per_sm = 0, sms = 0;
