@@ -45,12 +45,16 @@ def _factorize_gpu(X, G, d, r, oversample, q, seed):
     return A, B, sig, omega
 
 
-@pytest.mark.parametrize("name,over,r,p,q", [
-    ("tiny_T2048_N256_r64", dict(T=2048), 64, 32, 2),
-    ("ragged_T1001_N256_r40", dict(T=1001), 40, 24, 2),
-    ("N1024_r128_decaying", dict(T=4096, G=4, H_kv=2, d_h=128, rho=64, decay=1.0, noise=0.01, noise_abs=False), 128, 64, 2),
+@pytest.mark.parametrize("name,over,r,p,q,near", [
+    ("tiny_T2048_N256_r64", dict(T=2048), 64, 32, 2, 1.15),
+    ("ragged_T1001_N256_r40", dict(T=1001), 40, 24, 2, 1.15),
+    ("N1024_r128_decaying", dict(T=4096, G=4, H_kv=2, d_h=128, rho=64, decay=1.0, noise=0.01, noise_abs=False), 128, 64, 2, 1.15),
+    # a sketch of 832 columns: wider than the blocked triangular solve holds in shared memory, so the row-wise one
+    # runs.  Two thirds of the kept directions lie in the flat noise tail, which no sketch can order: the bound against
+    # the optimum is loose here, the one against the oracle's run of the same algorithm is what counts.
+    ("N1024_r768_wide_sketch", dict(T=4096, G=4, H_kv=2, d_h=128, rho=512, decay=1.0, noise=0.01, noise_abs=False), 768, 64, 1, 2.0),
 ])
-def test_clf_residual_orthonormality_and_projection(name, over, r, p, q):
+def test_clf_residual_orthonormality_and_projection(name, over, r, p, q, near):
     s = synth.config(1, **over)
     K, _ = synth.make_kv(s)                                           # (G, T, d) bf16
     X = torch.cat([K[l] for l in range(s.G)], dim=1)                  # (T, G d): the layers side by side (Eq. 1)
@@ -64,7 +68,7 @@ def test_clf_residual_orthonormality_and_projection(name, over, r, p, q):
     # the oracle's restatement of the same algorithm on the same test matrix
     Ao, Vo, so = O.clf_randomized(Xf, r, C.f32(omega), q)
     res_o = float(((Xf - Ao.astype(np.float64) @ Vo.astype(np.float64).T) ** 2).sum())
-    assert res <= 1.15 * optimum, (name, res / optimum)               # the randomised subspace is near the optimum
+    assert res <= near * optimum, (name, res / optimum)               # the randomised subspace is near the optimum
     assert res <= 1.03 * res_o, (name, res / res_o)                   # and the fp32/bf16 GPU pipeline loses nothing on fp64
     assert np.abs(V.T @ V - np.eye(r)).max() <= 2e-2                  # orthonormal rows of B (bf16 storage)
     proj = Xf @ V                                                     # A = X B^T
