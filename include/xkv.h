@@ -352,6 +352,16 @@ XKV_API int xkv_debug_launch_counts(uint64_t* counts);
 #define XKV_INJECT_SCAN_NO_LOAD 1u
 #define XKV_INJECT_FUSED_NO_B 2u
 XKV_API int xkv_debug_set_fault_injection(xkv_group* grp, uint32_t mask);
+/*
+ * The same for xkv_clf_factorize, which has no handle: the mask applies to every later call of the process until it
+ * is set back to 0.
+ *   XKV_INJECT_CLF_BARRIER    one CTA of the Jacobi kernel does not arrive at the first grid barrier, and the wait of
+ *                             that kernel's barriers is shortened to about a millisecond; the other CTAs give up,
+ *                             the workspace's flag word gets XKV_FLAG_TIMEOUT (xkv_clf_status returns
+ *                             XKV_ERR_TIMEOUT) and the factors of that call are unspecified.
+ */
+#define XKV_INJECT_CLF_BARRIER 4u
+XKV_API int xkv_debug_set_clf_fault_injection(uint32_t mask);
 
 /*
  * Chunk selection for callers that must not allocate device memory.  (The paper has no counterpart: this is a

@@ -472,6 +472,12 @@ int xkv_clf_factorize(const xkv_clf_config* cfg, const void* X, const void* omeg
   return clf_factorize(cfg, X, omega, workspace, workspace_bytes, A, B, sigma, device, (cudaStream_t)stream);
 }
 
+int xkv_debug_set_clf_fault_injection(uint32_t mask) {
+  if (mask & ~XKV_INJECT_CLF_BARRIER) return XKV_ERR_INVALID_ARG;
+  clf_set_fault_injection(mask);
+  return XKV_OK;
+}
+
 int xkv_clf_status(const void* workspace, uint32_t* flags, void* stream) {
   if (!workspace) return XKV_ERR_INVALID_ARG;
   unsigned int f = 0;

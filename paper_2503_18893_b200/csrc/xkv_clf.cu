@@ -526,6 +526,8 @@ struct JacobiSync {          // words of the workspace's flag block
   unsigned int* count;       // arrivals so far (monotonic)
   unsigned int* gen;         // barriers completed
   unsigned int* abort;       // a CTA gave up
+  unsigned int spin_limit;   // polls of one barrier wait
+  unsigned int skip_first;   // fault injection (tests of the give-up path): CTA 0 passes the first barrier without arriving
 };
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned int* p) {
@@ -544,12 +546,14 @@ __device__ __forceinline__ bool jacobi_grid_barrier(const JacobiSync& sy, unsign
     ++my_gen;
     __threadfence();
     bool ok = true;
-    if (atomicAdd(sy.count, 1u) == gridDim.x * my_gen - 1u) {
+    if (sy.skip_first && blockIdx.x == 0 && my_gen == 1u) {
+      // injected fault: the others never see this arrival, run into their limit and raise the abort word
+    } else if (atomicAdd(sy.count, 1u) == gridDim.x * my_gen - 1u) {
       st_release_u32(sy.gen, my_gen);                      // last to arrive: open the barrier
     } else {
       unsigned i = 0;
       while (ld_acquire_u32(sy.gen) < my_gen) {
-        if (++i >= kJacobiSpinLimit || ld_acquire_u32(sy.abort) != 0u) { ok = false; break; }
+        if (++i >= sy.spin_limit || ld_acquire_u32(sy.abort) != 0u) { ok = false; break; }
       }
     }
     if (!ok) { atomicOr(sy.flags, XKV_FLAG_TIMEOUT); atomicExch(sy.abort, 1u); }
@@ -855,6 +859,9 @@ cudaError_t clf_gemm(const void* a, const void* b, int M, int N, int K, float* C
   return launch_gemm<false>(a, K, M, M, b, N, K, K, C, nullptr, N, flags, device, s);
 }
 
+static std::atomic<unsigned> g_clf_inject{0};
+void clf_set_fault_injection(unsigned mask) { g_clf_inject.store(mask, std::memory_order_relaxed); }
+
 int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, void* workspace, uint64_t workspace_bytes,
                   void* A_out, void* B_out, float* sigma, int device, cudaStream_t s) {
   int st = check_clf_config(c);
@@ -945,7 +952,9 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
         float* M2 = (float*)(w + p.off_m2);
         float* P2 = (float*)(w + p.off_p2);
         float2* partial = (float2*)(w + p.off_cs);
-        JacobiSync sy{flags, flags + 8, flags + 9, flags + 10};      // zeroed with the flag block above
+        const bool inject = (g_clf_inject.load(std::memory_order_relaxed) & XKV_INJECT_CLF_BARRIER) != 0u;
+        JacobiSync sy{flags, flags + 8, flags + 9, flags + 10,            // zeroed with the flag block above
+                      inject ? 1024u : kJacobiSpinLimit, inject ? 1u : 0u};
         int l_arg = l;
         void* args[] = {&Mm, &M2, &Pm, &P2, &l_arg, &partial, &sy};
         e = cudaLaunchCooperativeKernel((const void*)jacobi_coop_kernel, dim3(sms), dim3(kJacobiCoopThreads), args, 0, s);

@@ -180,6 +180,7 @@ cudaError_t launch_dequantize_rtn3(const void* rec, long long rows, int cols, __
 // xkv_clf.cu
 int clf_rank_l(const xkv_clf_config* c, int* l);
 int clf_workspace_bytes(const xkv_clf_config* c, uint64_t* bytes);
+void clf_set_fault_injection(unsigned mask);
 int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, void* workspace, uint64_t workspace_bytes,
                   void* A_out, void* B_out, float* sigma, int device, cudaStream_t s);
 cudaError_t clf_gemm(const void* a, const void* b, int M, int N, int K, float* C, unsigned int* flags, int device,

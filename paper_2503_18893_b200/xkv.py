@@ -125,6 +125,9 @@ XKV_KERNEL_FAMILIES = ("scan", "topk", "fused", "merge", "tile", "tail_tc", "tai
 XKV_FLAG_CLF_BREAKDOWN = 4
 XKV_INJECT_SCAN_NO_LOAD = 1
 XKV_INJECT_FUSED_NO_B = 2
+XKV_INJECT_CLF_BARRIER = 4
+_lib.xkv_debug_set_clf_fault_injection.argtypes = [ctypes.c_uint32]
+_lib.xkv_debug_set_clf_fault_injection.restype = ctypes.c_int
 
 
 class XKVError(RuntimeError):
@@ -152,6 +155,12 @@ def xkv_debug_launch_counts() -> dict:
     if st != XKV_OK:
         raise XKVError(st, "xkv_debug_launch_counts")
     return {n: int(a[i]) for i, n in enumerate(XKV_KERNEL_FAMILIES)}
+
+
+def xkv_debug_set_clf_fault_injection(mask: int) -> None:
+    st = _lib.xkv_debug_set_clf_fault_injection(mask)
+    if st != XKV_OK:
+        raise XKVError(st, "xkv_debug_set_clf_fault_injection")
 
 
 def xkv_debug_set_fault_injection(grp, mask: int) -> None:
