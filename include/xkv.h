@@ -177,7 +177,8 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
  * rank-r factors A = U Sigma (T x r) and B_l (r x d per layer) of X = [X_l0 ... X_l0+G-1] (T x G d), by the
  * randomised SVD the paper describes for prefill (App. "Custom SVD Kernel": power iterations as 16-bit tensor-core
  * matrix products, shifted Cholesky QR instead of Householder QR).  Steps: Z <- omega; (power_iters + 1) times
- * Y = X Z, U = X^T Y, Z = orth(U) (three passes of Cholesky QR with a relative diagonal shift, fp32); then the
+ * Y = X Z, U = X^T Y, Z = orth(U) (two passes of Cholesky QR with a relative diagonal shift, five for the last
+ * iterate; Gram matrix, factor and solve in fp64); then the
  * Rayleigh-Ritz step on span(Z): M = Z^T X^T X Z = P Lambda P^T (Jacobi), V = Z P_r, B = V^T rounded to bf16,
  * A = X bf16(V), sigma = sqrt(Lambda).  The result approximates the optimum of Eq. 1 (it is not unique up to signs and
  * rotations inside equal singular values: compare residuals, never factors).
@@ -190,6 +191,10 @@ XKV_API int xkv_sr_reconstruct_attend_tail(xkv_group* grp, int layer_begin, int 
  * sigma     out fp32 [r], optional.
  * The call allocates nothing and enqueues everything on `stream`.  xkv_clf_status (after the caller has synchronised,
  * or blocking on `stream`) reads the flag word of the workspace: XKV_FLAG_TIMEOUT, XKV_FLAG_CLF_BREAKDOWN.
+ * The first 256 bytes of the workspace are that flag block (32-bit words); besides word 0 (the flags) a caller may
+ * read word 11, the number of Jacobi sweeps the last call ran (a diagnostic: at most 12); the rest is internal.
+ * The Jacobi sweeps are one cooperative launch (all its CTAs resident at once), so the device must not be fully
+ * occupied by kernels that wait for this one.
  * Errors: INVALID_ARG, UNSUPPORTED (l too large for the eigen-solver: l <= 2048), ARCH, CUDA.
  */
 typedef struct {
