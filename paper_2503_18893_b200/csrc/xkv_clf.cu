@@ -29,8 +29,13 @@ namespace {
 using namespace ptx;
 
 constexpr int kGemmThreads = 192;                 // warps 0-3 epilogue, 4 TMA producer, 5 MMA issue
-constexpr int kGemmStages = 6;
-constexpr int kGemmStageBytes = 32768;            // A: two slabs of [64 k][64 m] (8 KB each); B: [128 n][64 k] (16 KB)
+// One stage of the operand ring: A, two slabs of [64 k][64 m] (8 KB each), and B, [BN n][64 k] (BN * 128 bytes).
+// Tiles are 128 x BN with BN = 256, 192 or 128: an N = 128 step reads 8 KB of operands per 64 cycles, all the shared-
+// memory pipe gives, an N = 256 step 12 KB per 128 cycles.  Four stages for the wide tiles (one CTA per SM), three
+// for BN = 128 (two CTAs per SM, so that one's epilogue hides behind the other's products).
+template <int BN> constexpr int gemm_stage_bytes() { return 16384 + BN * 128; }
+template <int BN> constexpr int gemm_stages() { return BN == 128 ? 3 : 4; }
+constexpr int kGemmMaxStages = 4;
 constexpr uint32_t kGemmWaitLimit = 1u << 24;
 
 __device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity) {
@@ -40,19 +45,21 @@ __device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity) {
   return false;
 }
 
-// C[m][n] = sum_k A[k][m] B[n][k].  grid = (ceil(N/128), ceil(M/128)).  TRANS: store C^T (out[n][m]).
+// C[m][n] = sum_k A[k][m] B[n][k].  grid = (ceil(N/BN), ceil(M/128)).  TRANS: store C^T (out[n][m]).
 // Out-of-range rows and columns of the operands are zero-filled by the copy engine; stores are guarded.
-template <bool TRANS>
+template <bool TRANS, int BN>
 __global__ void __launch_bounds__(kGemmThreads)
 clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int M, int N, int K,
                 float* __restrict__ Cf, __nv_bfloat16* __restrict__ Cb, long long ldc, unsigned int* __restrict__ flags) {
   extern __shared__ uint8_t gemm_smem[];
-  __shared__ __align__(8) uint64_t bars[2 * kGemmStages + 1];
+  constexpr int kGemmStages = gemm_stages<BN>(), kGemmStageBytes = gemm_stage_bytes<BN>();
+  constexpr uint32_t kCols = BN <= 128 ? 128u : 256u;      // tensor-memory columns (a power of two)
+  __shared__ __align__(8) uint64_t bars[2 * kGemmMaxStages + 1];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_s;
   const uint32_t base = (smem_u32(gemm_smem) + 1023u) & ~1023u;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n0 = blockIdx.x * 128, m0 = blockIdx.y * 128;
+  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * 128;
   const int KB = (K + 63) / 64;
   const uint32_t bar0 = smem_u32(bars);
   auto FULL = [&](int s) { return bar0 + 8u * (uint32_t)s; };
@@ -65,7 +72,7 @@ clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     fence_mbar_init();
   }
   if (warp == 5) {
-    tmem_alloc(smem_u32(&tmem_slot), 128);
+    tmem_alloc(smem_u32(&tmem_slot), kCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -82,13 +89,13 @@ clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         mbar_expect_tx(FULL(s), kGemmStageBytes);
         tma_load_2d(st, &map_a, m0, kb * 64, FULL(s));                 // A: columns m0..m0+63, rows (k) kb*64..+63
         tma_load_2d(st + 8192, &map_a, m0 + 64, kb * 64, FULL(s));     //    columns m0+64..m0+127
-        tma_load_2d(st + 16384, &map_b, kb * 64, n0, FULL(s));         // B: columns (k) kb*64..+63, rows n0..n0+127
+        tma_load_2d(st + 16384, &map_b, kb * 64, n0, FULL(s));         // B: columns (k) kb*64..+63, rows n0..n0+BN-1
       }
     }
   } else if (warp == 5) {
     if (lane == 0) {
       const uint64_t desc_hi = smem_desc_sw128(0, 0) & 0xFFFFFFFF00000000ull;
-      constexpr uint32_t idesc = idesc_bf16_f32(128, 128) | (1u << 15);   // A is read along its rows (MN-major)
+      constexpr uint32_t idesc = idesc_bf16_f32(128, BN) | (1u << 15);    // A is read along its rows (MN-major)
       for (int kb = 0; kb < KB; ++kb) {
         const int s = kb % kGemmStages;
         if (!gemm_wait(FULL(s), (uint32_t)((kb / kGemmStages) & 1))) { ok = false; break; }
@@ -120,18 +127,39 @@ clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int m = m0 + tid;
       const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
 #pragma unroll 1
-      for (int cb = 0; cb < 4; ++cb) {
+      for (int cb = 0; cb < BN / 32; ++cb) {
         float v[32];
         tmem_ld32(tmem + lane_base + (uint32_t)(cb * 32), v);
         tc_wait_ld();
         if (m < M) {
+          const int nb = n0 + cb * 32;
+          if (!TRANS && nb + 32 <= N && (ldc & 7) == 0) {
+            // a whole run of 32 columns of one row: 16-byte stores (the row pitch keeps them aligned)
+            const long long at = (long long)m * ldc + nb;
+            if (Cf) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int n = n0 + cb * 32 + i;
-            if (n < N) {
-              const long long at = TRANS ? (long long)n * ldc + m : (long long)m * ldc + n;
-              if (Cf) Cf[at] = v[i];
-              if (Cb) Cb[at] = __float2bfloat16(v[i]);
+              for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(Cf + at + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            }
+            if (Cb) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[i], v[i + 1]), h1 = __floats2bfloat162_rn(v[i + 2], v[i + 3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[i + 4], v[i + 5]), h3 = __floats2bfloat162_rn(v[i + 6], v[i + 7]);
+                uint4 u;
+                u.x = *reinterpret_cast<uint32_t*>(&h0); u.y = *reinterpret_cast<uint32_t*>(&h1);
+                u.z = *reinterpret_cast<uint32_t*>(&h2); u.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(Cb + at + i) = u;
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int n = nb + i;
+              if (n < N) {
+                const long long at = TRANS ? (long long)n * ldc + m : (long long)m * ldc + n;
+                if (Cf) Cf[at] = v[i];
+                if (Cb) Cb[at] = __float2bfloat16(v[i]);
+              }
             }
           }
         }
@@ -144,7 +172,7 @@ clf_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   __syncthreads();
   if (warp == 5) {
     tc_fence_after();
-    tmem_dealloc(tmem, 128);
+    tmem_dealloc(tmem, kCols);
   }
 }
 
@@ -817,21 +845,36 @@ int check_clf_config(const xkv_clf_config* c) {
   return XKV_OK;
 }
 
+template <bool TRANS, int BN>
+cudaError_t launch_gemm_bn(const void* a, int a_rows_k, int a_cols_m, int a_pitch, const void* b, int b_rows_n, int b_cols_k,
+                           int b_pitch, float* Cf, __nv_bfloat16* Cb, long long ldc, unsigned int* flags, int device,
+                           cudaStream_t s) {
+  CUtensorMap ma, mb;
+  if (!encode_bf16_map(&ma, a, (uint64_t)a_rows_k, (uint64_t)a_cols_m, (uint64_t)a_pitch, 64) ||
+      !encode_bf16_map(&mb, b, (uint64_t)b_rows_n, (uint64_t)b_cols_k, (uint64_t)b_pitch, BN))
+    return cudaErrorInvalidValue;
+  const size_t smem = 1024 + (size_t)gemm_stages<BN>() * gemm_stage_bytes<BN>();
+  cudaError_t e = ensure_dyn_smem<clf_gemm_kernel<TRANS, BN>>(smem, device);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((b_rows_n + BN - 1) / BN, (a_cols_m + 127) / 128);
+  clf_gemm_kernel<TRANS, BN><<<grid, kGemmThreads, smem, s>>>(ma, mb, a_cols_m, b_rows_n, a_rows_k, Cf, Cb, ldc, flags);
+  count_launch(kFamClf);
+  return cudaGetLastError();
+}
+
+// The tile width that pads N least (the widest on a tie): 576 columns are three tiles of 192, a tall N is tiles of 256.
 template <bool TRANS>
 cudaError_t launch_gemm(const void* a, int a_rows_k, int a_cols_m, int a_pitch, const void* b, int b_rows_n, int b_cols_k,
                         int b_pitch, float* Cf, __nv_bfloat16* Cb, long long ldc, unsigned int* flags, int device,
                         cudaStream_t s) {
-  CUtensorMap ma, mb;
-  if (!encode_bf16_map(&ma, a, (uint64_t)a_rows_k, (uint64_t)a_cols_m, (uint64_t)a_pitch, 64) ||
-      !encode_bf16_map(&mb, b, (uint64_t)b_rows_n, (uint64_t)b_cols_k, (uint64_t)b_pitch, 128))
-    return cudaErrorInvalidValue;
-  const size_t smem = 1024 + (size_t)kGemmStages * kGemmStageBytes;
-  cudaError_t e = ensure_dyn_smem<clf_gemm_kernel<TRANS>>(smem, device);
-  if (e != cudaSuccess) return e;
-  const dim3 grid((b_rows_n + 127) / 128, (a_cols_m + 127) / 128);
-  clf_gemm_kernel<TRANS><<<grid, kGemmThreads, smem, s>>>(ma, mb, a_cols_m, b_rows_n, a_rows_k, Cf, Cb, ldc, flags);
-  count_launch(kFamClf);
-  return cudaGetLastError();
+  const int N = b_rows_n;
+  auto padded = [&](int bn) { return (long long)((N + bn - 1) / bn) * bn; };
+  int bn = 256;
+  if (padded(192) < padded(bn)) bn = 192;
+  if (padded(128) < padded(bn)) bn = 128;
+  if (bn == 256) return launch_gemm_bn<TRANS, 256>(a, a_rows_k, a_cols_m, a_pitch, b, b_rows_n, b_cols_k, b_pitch, Cf, Cb, ldc, flags, device, s);
+  if (bn == 192) return launch_gemm_bn<TRANS, 192>(a, a_rows_k, a_cols_m, a_pitch, b, b_rows_n, b_cols_k, b_pitch, Cf, Cb, ldc, flags, device, s);
+  return launch_gemm_bn<TRANS, 128>(a, a_rows_k, a_cols_m, a_pitch, b, b_rows_n, b_cols_k, b_pitch, Cf, Cb, ldc, flags, device, s);
 }
 
 }  // namespace
