@@ -309,40 +309,61 @@ chol_shift_kernel(double* __restrict__ G, int l, double shift_rel) {
   for (int i = tid; i < l; i += 1024) G[(size_t)i * l + i] += shift_rel * mx;
 }
 
-// Diagonal block [kb, kb+nb): unblocked factorisation in shared memory (one CTA of 32 x 32 threads).  A pivot that
-// is not positive (breakdown) is replaced by a tiny one and reported in flags.
-__global__ void __launch_bounds__(1024)
+// Diagonal block [kb, kb+nb): unblocked factorisation by one warp.  A pivot that is not positive (breakdown) is
+// replaced by a tiny one and reported in flags.
+__global__ void __launch_bounds__(kCholNb)
 chol_diag_kernel(double* __restrict__ G, int l, int kb, int nb, unsigned int* __restrict__ flags) {
-  __shared__ double a[kCholNb][kCholNb + 1];
-  const int i = threadIdx.y, j = threadIdx.x;
-  a[i][j] = (i < nb && j < nb) ? G[(size_t)(kb + i) * l + kb + j] : (i == j ? 1.0 : 0.0);
-  __syncthreads();
-  for (int c = 0; c < nb; ++c) {
-    if (i == c && j == c) {
-      double d = a[c][c];
+  // One warp, lane i holds row i of the block in registers.  Step c: lane c takes the root of its diagonal entry, every
+  // lane below scales its entry of column c, the column goes through shared memory, and every lane takes it out of
+  // the rest of its row (independent multiply-adds).  Roots and quotients go through rsqrt: a step is a chain of
+  // dependent fp64 latencies, and sqrt and division are the longest of them.
+  __shared__ double col[kCholNb];
+  __shared__ double piv;
+  const int i = threadIdx.x;
+  double a[kCholNb];
+#pragma unroll
+  for (int j = 0; j < kCholNb; ++j) a[j] = (i < nb && j < nb && j <= i) ? G[(size_t)(kb + i) * l + kb + j] : (i == j ? 1.0 : 0.0);
+#pragma unroll
+  for (int c = 0; c < kCholNb; ++c) {
+    if (i == c) {
+      double d = a[c];
       if (!(d > 0.0)) { atomicOr(flags, XKV_FLAG_CLF_BREAKDOWN); d = 1e-300; }
-      a[c][c] = sqrt(d);
+      const double y = rsqrt(d);
+      a[c] = d * y;                                   // sqrt(d)
+      piv = y;
     }
-    __syncthreads();
-    if (j == c && i > c) a[i][c] /= a[c][c];
-    __syncthreads();
-    if (j > c && i >= j) a[i][j] -= a[i][c] * a[j][c];
-    __syncthreads();
+    __syncwarp();
+    const double y = piv;
+    if (i > c) a[c] *= y;
+    col[i] = a[c];
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < kCholNb; ++j) {
+      if (j > c && j <= i) a[j] -= a[c] * col[j];
+    }
+    __syncwarp();
   }
-  if (i < nb && j < nb && j <= i) G[(size_t)(kb + i) * l + kb + j] = a[i][j];
+#pragma unroll
+  for (int j = 0; j < kCholNb; ++j) if (i < nb && j < nb && j <= i) G[(size_t)(kb + i) * l + kb + j] = a[j];
 }
 
+constexpr int kCholPanelThreads = 128;             // (one warp per CTA, to spread the rows over more SMs: 24 us instead of 16)
 // Panel below the diagonal block: row i of L21 solves x L11^T = A21[i] (one thread per row).
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kCholPanelThreads)
 chol_panel_kernel(double* __restrict__ G, int l, int kb, int nb) {
   __shared__ double L11[kCholNb][kCholNb + 1];
-  for (int e = threadIdx.x; e < kCholNb * kCholNb; e += 128) {
+  __shared__ double dinv[kCholNb];
+  for (int e = threadIdx.x; e < kCholNb * kCholNb; e += kCholPanelThreads) {
     const int r = e / kCholNb, c = e % kCholNb;
-    L11[r][c] = (r < nb && c <= r) ? G[(size_t)(kb + r) * l + kb + c] : 0.0;
+    const double v = (r < nb && c <= r) ? G[(size_t)(kb + r) * l + kb + c] : 0.0;
+    L11[r][c] = v;
+    if (r == c) dinv[r] = r < nb ? 1.0 / v : 0.0;
   }
   __syncthreads();
-  const int i = kb + nb + blockIdx.x * 128 + threadIdx.x;
+  const int i = kb + nb + blockIdx.x * kCholPanelThreads + threadIdx.x;
   if (i >= l) return;
+  // column sweep: once x_c is known it is taken out of every later entry, so the multiply-adds of a step are
+  // independent of one another (a dot product per entry is one long dependent chain on the fp64 pipe)
   double x[kCholNb];
   double* row = G + (size_t)i * l + kb;
 #pragma unroll
@@ -350,10 +371,9 @@ chol_panel_kernel(double* __restrict__ G, int l, int kb, int nb) {
 #pragma unroll
   for (int c = 0; c < kCholNb; ++c) {
     if (c < nb) {
-      double v = x[c];
+      x[c] *= dinv[c];
 #pragma unroll
-      for (int t = 0; t < kCholNb; ++t) if (t < c) v -= x[t] * L11[c][t];
-      x[c] = v / L11[c][c];
+      for (int t = 0; t < kCholNb; ++t) if (t > c) x[t] -= x[c] * L11[t][c];
     }
   }
 #pragma unroll
@@ -962,11 +982,11 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
       int launches = 2;
       for (int kb = 0; kb < l; kb += kCholNb) {
         const int nb = l - kb < kCholNb ? l - kb : kCholNb;
-        chol_diag_kernel<<<1, dim3(kCholNb, kCholNb), 0, s>>>(Gm, l, kb, nb, flags);
+        chol_diag_kernel<<<1, kCholNb, 0, s>>>(Gm, l, kb, nb, flags);
         const int rem = l - kb - nb;
         ++launches;
         if (rem > 0) {
-          chol_panel_kernel<<<(rem + 127) / 128, 128, 0, s>>>(Gm, l, kb, nb);
+          chol_panel_kernel<<<(rem + kCholPanelThreads - 1) / kCholPanelThreads, kCholPanelThreads, 0, s>>>(Gm, l, kb, nb);
           const int tiles = (rem + kCholNb - 1) / kCholNb;
           chol_update_kernel<<<dim3(tiles, tiles), dim3(kCholNb, kCholNb), 0, s>>>(Gm, l, kb, nb);
           launches += 2;
