@@ -52,25 +52,36 @@ __device__ __forceinline__ void score_pass(uint32_t tile, const float* __restric
   const uint32_t sw = (uint32_t)(row0 & 7);
   const uint32_t a0 = tile + (uint32_t)row0 * 128u;
   const uint32_t a1 = a0 + (uint32_t)kScoreThreads * 128u;
-#pragma unroll 2
+#pragma unroll 4
   for (int cc = 0; cc < DH / 8; ++cc) {
     const uint32_t off = (uint32_t)(cc >> 3) * (kScoreRows * 128u) + ((((uint32_t)cc & 7u) ^ sw) << 4);
     const uint4 va = lds128(a0 + off);
     const uint4 vb = lds128(a1 + off);
     const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
     const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
+    float qv[HB][8];
 #pragma unroll
     for (int h = 0; h < HB; ++h) {
       const float4 q0 = *reinterpret_cast<const float4*>(qs + h * DH + cc * 8);
       const float4 q1 = *reinterpret_cast<const float4*>(qs + h * DH + cc * 8 + 4);
-      const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+      qv[h][0] = q0.x; qv[h][1] = q0.y; qv[h][2] = q0.z; qv[h][3] = q0.w;
+      qv[h][4] = q1.x; qv[h][5] = q1.y; qv[h][6] = q1.z; qv[h][7] = q1.w;
+    }
+    // element by element (ascending i, the canonical order of every sum), all heads and both rows per element: the
+    // 2 * HB multiply-adds of an element are independent of one another
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        // element 2w is the low half of word w, element 2w+1 the high half; ascending i
-        acc0[h] = fmaf(qv[2 * w], __uint_as_float(wa[w] << 16), acc0[h]);
-        acc1[h] = fmaf(qv[2 * w], __uint_as_float(wb[w] << 16), acc1[h]);
-        acc0[h] = fmaf(qv[2 * w + 1], __uint_as_float(wa[w] & 0xffff0000u), acc0[h]);
-        acc1[h] = fmaf(qv[2 * w + 1], __uint_as_float(wb[w] & 0xffff0000u), acc1[h]);
+    for (int w = 0; w < 4; ++w) {
+      const float xa0 = __uint_as_float(wa[w] << 16), xb0 = __uint_as_float(wb[w] << 16);
+      const float xa1 = __uint_as_float(wa[w] & 0xffff0000u), xb1 = __uint_as_float(wb[w] & 0xffff0000u);
+#pragma unroll
+      for (int h = 0; h < HB; ++h) {
+        acc0[h] = fmaf(qv[h][2 * w], xa0, acc0[h]);
+        acc1[h] = fmaf(qv[h][2 * w], xb0, acc1[h]);
+      }
+#pragma unroll
+      for (int h = 0; h < HB; ++h) {
+        acc0[h] = fmaf(qv[h][2 * w + 1], xa1, acc0[h]);
+        acc1[h] = fmaf(qv[h][2 * w + 1], xb1, acc1[h]);
       }
     }
   }
