@@ -175,14 +175,32 @@ __device__ __forceinline__ void key_logits(uint32_t acc, const float2* __restric
 #pragma unroll
         for (int e = 0; e < 4; ++e) { r1[e] = x1[i4 * 4 + e]; r2[e] = x2[i4 * 4 + e]; }
       }
+      // heads in groups of four, element by element inside a group: the four multiply-adds of an element are
+      // independent (one head after the other is a chain of eight dependent ones)
 #pragma unroll
-      for (int h = 0; h < NR; ++h) {
-        const float4 qa = *reinterpret_cast<const float4*>(q_s + h * DH + ii);
-        const float4 qb = *reinterpret_cast<const float4*>(q_s + h * DH + HALF + ii);
-        z[h] = fmaf(qa.x, r1[0], z[h]); z[h] = fmaf(qb.x, r2[0], z[h]);
-        z[h] = fmaf(qa.y, r1[1], z[h]); z[h] = fmaf(qb.y, r2[1], z[h]);
-        z[h] = fmaf(qa.z, r1[2], z[h]); z[h] = fmaf(qb.z, r2[2], z[h]);
-        z[h] = fmaf(qa.w, r1[3], z[h]); z[h] = fmaf(qb.w, r2[3], z[h]);
+      for (int h0 = 0; h0 < NR; h0 += 4) {
+        float4 qa[4], qb[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          qa[h] = *reinterpret_cast<const float4*>(q_s + (h0 + h) * DH + ii);
+          qb[h] = *reinterpret_cast<const float4*>(q_s + (h0 + h) * DH + HALF + ii);
+        }
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qa[h].x, r1[0], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qb[h].x, r2[0], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qa[h].y, r1[1], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qb[h].y, r2[1], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qa[h].z, r1[2], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qb[h].z, r2[2], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qa[h].w, r1[3], z[h0 + h]);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) z[h0 + h] = fmaf(qb[h].w, r2[3], z[h0 + h]);
       }
     }
   }
