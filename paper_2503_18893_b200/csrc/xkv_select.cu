@@ -135,7 +135,31 @@ score_pool_kernel(const __grid_constant__ CUtensorMap tmap, GroupDev dev, const 
   grid_dependency_launch();
   // queries of this KV head, widened to fp32 while the landmarks are in flight
   const __nv_bfloat16* qg = q + (((long long)l * dev.batch + b) * dev.H_q + (long long)g * dev.n_rep) * DH;
-  for (int i = threadIdx.x; i < dev.n_rep * DH; i += kScoreThreads) qs[i] = __bfloat162float(qg[i]);
+  // (all the 16-byte loads of a lane are issued before the first is used: one trip to L2, not one per element)
+  {
+    const uint4* qv = reinterpret_cast<const uint4*>(qg);
+    const int n_pieces = dev.n_rep * (DH / 8);
+    constexpr int kMaxPieces = kMaxRep * (DH / 8) / kScoreThreads;   // at most kMaxRep query heads per KV head
+    uint4 u[kMaxPieces];
+#pragma unroll
+    for (int i = 0; i < kMaxPieces; ++i) {
+      const int pc = threadIdx.x + i * kScoreThreads;
+      u[i] = pc < n_pieces ? qv[pc] : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < kMaxPieces; ++i) {
+      const int pc = threadIdx.x + i * kScoreThreads;
+      if (pc < n_pieces) {
+        float4 a, b;
+        a.x = __uint_as_float(u[i].x << 16); a.y = __uint_as_float(u[i].x & 0xffff0000u);
+        a.z = __uint_as_float(u[i].y << 16); a.w = __uint_as_float(u[i].y & 0xffff0000u);
+        b.x = __uint_as_float(u[i].z << 16); b.y = __uint_as_float(u[i].z & 0xffff0000u);
+        b.z = __uint_as_float(u[i].w << 16); b.w = __uint_as_float(u[i].w & 0xffff0000u);
+        *reinterpret_cast<float4*>(qs + pc * 8) = a;
+        *reinterpret_cast<float4*>(qs + pc * 8 + 4) = b;
+      }
+    }
+  }
   __syncthreads();
 
   if (!mbar_wait_bounded(bar, 0, no_load ? 1024u : kWaitLimit)) {
