@@ -685,10 +685,10 @@ def run_sweep(args, world, rank, local_rank, dist):
 def sweep_table(rows) -> str:
     out = ["| point | windows | SR us / window-step | window-steps/s | tokens/s | bytes_min MB | bound | roofline frac | "
            "select us | attend us | dense us (ours) | dense GB/s | torch SDPA us | SR speed-up over dense | parity (idx "
-           "mismatch / max rel err) |", "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+           "mismatch / max rel err) | SM MHz under load |", "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
     for r in rows:
         if "skipped" in r:
-            out.append(f"| {r['point']} | skipped: {r['skipped']} |" + " |" * 13)
+            out.append(f"| {r['point']} | skipped: {r['skipped']} |" + " |" * 14)
             continue
         sr, d = r["step_roofline"], r.get("dense_attention", {})
         par = r.get("parity", {})
@@ -698,7 +698,9 @@ def sweep_table(rows) -> str:
         out.append(f"| {r['point']} | {r['config']['windows']} | {sr['achieved_us']:.1f} | {r['value']:.0f} | "
                    f"{r['tokens_per_s']:.0f} | {sr['bytes_min_per_group_step'] / 1e6:.1f} | {sr['bound']} | "
                    f"{sr['frac']:.3f} | {r['select_kernel']['us_per_launch']:.1f} | {r['roofline']['us_per_launch']:.1f} | "
-                   f"{dense} | {par.get('idx_mismatch', 'n/a')} / {par.get('max_rel_err', float('nan')):.1e} |")
+                   f"{dense} | {par.get('idx_mismatch', 'n/a')} / {par.get('max_rel_err', float('nan')):.1e} | "
+                   f"{r.get('clocks', {}).get('sm_mhz', float('nan')):.0f}"
+                   f"{' (power cap)' if 'sw_power_cap' in r.get('clocks', {}).get('reasons', []) else ''} |")
     return "\n".join(out) + "\n"
 
 
