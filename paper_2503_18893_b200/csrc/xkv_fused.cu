@@ -798,7 +798,30 @@ sr_fused_kernel(const __grid_constant__ CUtensorMap bk_map, GroupDev dev, Sched 
 #pragma unroll
       for (int h = 0; h < NR; ++h) { m_run[h] = -INFINITY; l_thr[h] = 0.0f; }
       const __nv_bfloat16* qg = q + (((long long)cur.l * dev.batch + cur.b) * dev.H_q + (long long)cur.g * n_rep) * DH;
-      for (int i = j; i < NR * DH; i += 128) q_s[i] = i < n_rep * DH ? __bfloat162float(qg[i]) : 0.0f;
+      // 16-byte pieces, all of a thread's loads issued before the first is used (heads beyond n_rep are zero)
+      {
+        constexpr int kPieces = NR * DH / 8, kPer = (kPieces + 127) / 128;
+        const uint4* qv = reinterpret_cast<const uint4*>(qg);
+        uint4 u[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int pc = j + 128 * i;
+          u[i] = (pc < kPieces && pc * 8 < n_rep * DH) ? __ldg(qv + pc) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int pc = j + 128 * i;
+          if (pc < kPieces) {
+            float4 a, b;
+            a.x = __uint_as_float(u[i].x << 16); a.y = __uint_as_float(u[i].x & 0xffff0000u);
+            a.z = __uint_as_float(u[i].y << 16); a.w = __uint_as_float(u[i].y & 0xffff0000u);
+            b.x = __uint_as_float(u[i].z << 16); b.y = __uint_as_float(u[i].z & 0xffff0000u);
+            b.z = __uint_as_float(u[i].w << 16); b.w = __uint_as_float(u[i].w & 0xffff0000u);
+            *reinterpret_cast<float4*>(q_s + pc * 8) = a;
+            *reinterpret_cast<float4*>(q_s + pc * 8 + 4) = b;
+          }
+        }
+      }
       group_sync();
     };
     while (ok && iter_next(cur, on_leave, on_enter)) {
