@@ -966,7 +966,7 @@ int clf_factorize(const xkv_clf_config* c, const void* X, const void* omega, voi
   e = e == cudaSuccess ? ensure_dyn_smem<trsolve_rows_kernel>(solve_smem, device) : e;
   const size_t tri_smem = ((size_t)kTriRows * (l + 4) + (size_t)kTriBlock * kDgemmLd) * sizeof(double);
   // the blocked solve keeps 32 rows of Z in shared memory: sketches wider than about 700 columns take the row-wise kernel
-  const bool mma_solve = (getenv("XKV_CLF_SOLVE_ROWS") == nullptr) && tri_smem <= 227u * 1024u;
+  const bool mma_solve = tri_smem <= 227u * 1024u;
   if (mma_solve) e = e == cudaSuccess ? ensure_dyn_smem<trsolve_mma_kernel>(tri_smem, device) : e;
   double* Xinv = (double*)(w + p.off_xinv);
   // Every pass divides the condition number by about shift^-1/2; the iterate of a power iteration only has to stay
