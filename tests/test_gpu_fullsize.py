@@ -110,6 +110,17 @@ def test_config5_corners(name, over):
     _check_full_size(s, [(0, 0, 0), (1, 0, 3), (s.G - 1, 0, s.H_kv - 1)])
 
 
+def test_config5_batch16_corner_many_problems():
+    """512 problems in one call (the batch-16 corner of the stress sweep at T = 16K): every index set, and attention on
+    problems of the first, a middle and the last sequence; the merge runs one CTA per problem here."""
+    from paper_2503_18893_b200 import xkv
+    s = synth.config(5, T=16384, r_k=256, r_v=256, k=1024, batch=16)
+    before = xkv.xkv_debug_launch_counts()
+    _check_full_size(s, [(0, 0, 0), (1, 7, 3), (2, 15, 7), (s.G - 1, 15, s.H_kv - 1), (0, 9, 5)])
+    after = xkv.xkv_debug_launch_counts()
+    assert after["merge_multi"] > before["merge_multi"] and after["merge"] == before["merge"]
+
+
 def test_config3_window_with_an_8192_row_uncompressed_tail():
     """The default tail kernel at the headline head width and size: selected rows by the library, then one softmax
     over those rows and 8192 uncompressed rows, on sampled problems."""
