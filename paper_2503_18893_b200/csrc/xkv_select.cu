@@ -591,12 +591,17 @@ topk_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict
 // n_c <= 16384 chunks, ITEMS = 32 (keys read twice instead of held in registers) n_c <= 32768.  The result is
 // identical to topk_kernel's for every input; only the amount of work differs.
 // Bin (counted from the top) that holds the `need`-th largest of the keys counted in hist[0..kTopkBins), by a
-// suffix sum over the bins; thread t owns bins 2t, 2t+1.  Results in sh[0] = bin, sh[1] = rank wanted inside the
-// bin, sh[2] = keys in the bin.  Contains barriers: call it from all threads.
+// suffix sum over the bins; thread t of the TH owns the kTopkBins / TH bins from t * (kTopkBins / TH).  Results in
+// sh[0] = bin, sh[1] = rank wanted inside the bin, sh[2] = keys in the bin.  Contains barriers: call it from all threads.
+template <int TH>
 __device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, uint32_t* warp_tot, uint32_t* sh, int tid) {
+  constexpr int BPT = kTopkBins / TH, NWARP = TH / 32;
+  static_assert(BPT >= 1 && BPT * TH == kTopkBins, "bins per thread");
   const int lane = tid & 31, warp = tid >> 5;
-  const uint32_t h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
-  const uint32_t mine = h0 + h1;
+  uint32_t h[BPT];
+  uint32_t mine = 0;
+#pragma unroll
+  for (int i = 0; i < BPT; ++i) { h[i] = hist[BPT * tid + i]; mine += h[i]; }
   uint32_t suf = mine;                                     // inclusive over higher lanes of the warp
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -606,40 +611,46 @@ __device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, ui
   if (lane == 0) warp_tot[warp] = suf;
   __syncthreads();
   if (warp == 0) {
-    const uint32_t t = warp_tot[lane];
+    const uint32_t t = lane < NWARP ? warp_tot[lane] : 0u;
     uint32_t ws = t;                                       // inclusive over higher warps
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const uint32_t v = __shfl_down_sync(0xffffffffu, ws, o);
       if (lane + o < 32) ws += v;
     }
-    warp_tot[lane] = ws - t;                               // keys in bins of higher warps
+    if (lane < NWARP) warp_tot[lane] = ws - t;             // keys in bins of higher warps
   }
   __syncthreads();
-  const uint32_t above = warp_tot[warp] + (suf - mine);    // keys in bins above 2t+1
+  const uint32_t above = warp_tot[warp] + (suf - mine);    // keys in bins above this thread's
   if (above < need && above + mine >= need) {              // exactly one thread
-    if (above + h1 >= need) { sh[0] = 2 * tid + 1; sh[1] = need - above; sh[2] = h1; }
-    else { sh[0] = 2 * tid; sh[1] = need - above - h1; sh[2] = h0; }
+    uint32_t acc = above;
+#pragma unroll
+    for (int i = BPT - 1; i >= 0; --i) {
+      if (acc < need && acc + h[i] >= need) { sh[0] = (uint32_t)(BPT * tid + i); sh[1] = need - acc; sh[2] = h[i]; }
+      acc += h[i];
+    }
   }
   __syncthreads();
 }
 
-template <int GPT, int ITEMS>
-__global__ void __launch_bounds__(kTopkThreads, 1)
+template <int GPT, int ITEMS, int TH>
+__global__ void __launch_bounds__(TH, 1)
 topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __restrict__ outliers, int n_out, float sign,
                   int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
   extern __shared__ __align__(16) uint8_t pivot_smem[];
-  constexpr int kPivotListMax = kTopkThreads * ITEMS;                              // every key may pass (all keys equal)
-  static_assert(kPivotListMax <= 65536 && kPivotListMax / 32 <= kTopkThreads, "16-bit chunk index, one bitmap word per thread");
+  constexpr int kPivotListMax = TH * ITEMS;                              // every key may pass (all keys equal)
+  static_assert(kPivotListMax <= 65536 && kPivotListMax / 32 <= TH, "16-bit chunk index, one bitmap word per thread");
   uint32_t* list_key = reinterpret_cast<uint32_t*>(pivot_smem);                    // [kPivotListMax]; later the chunk list
   uint16_t* list_idx = reinterpret_cast<uint16_t*>(list_key + kPivotListMax);      // [kPivotListMax]
   __shared__ __align__(16) uint32_t hist[kTopkBins];
   __shared__ uint32_t take_w[kPivotListMax / 32], eq_w[kPivotListMax / 32];        // bitmaps over the chunks
-  __shared__ uint32_t warp_tot[kTopkThreads / 32];
-  __shared__ uint32_t warp_min[kTopkThreads / 32], warp_max[kTopkThreads / 32];
+  __shared__ uint32_t warp_tot[TH / 32];
+  __shared__ uint32_t warp_min[TH / 32], warp_max[TH / 32];
   __shared__ uint32_t sh[4];
   __shared__ uint32_t sh_n;
 
+  constexpr int NWARP = TH / 32;
+  constexpr int kCand = kTopkCand < TH ? kTopkCand : TH;      // every candidate is ranked by a thread of its own
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_layer = dev.batch * dev.H_kv;
   const long long prob = (long long)l0 * per_layer + blockIdx.x;     // [G][batch][H_kv] order
@@ -655,7 +666,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
   const int j0 = tid * ITEMS;
   const bool all = (k_ch >= n_c);
   uint32_t thr = 0, need_eq = 0;
-  for (int w = tid; w < NW; w += kTopkThreads) { take_w[w] = 0u; eq_w[w] = 0u; }
+  for (int w = tid; w < NW; w += TH) { take_w[w] = 0u; eq_w[w] = 0u; }
   if (tid == 0) sh_n = 0;
   if (!all) {
     uint32_t key[ITEMS];
@@ -678,9 +689,9 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
       kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
     }
     if (lane == 0) { warp_min[warp] = kmin; warp_max[warp] = kmax; }
-    for (int i = tid; i < kTopkBins; i += kTopkThreads) hist[i] = 0;
+    for (int i = tid; i < kTopkBins; i += TH) hist[i] = 0;
     __syncthreads();
-    kmin = warp_min[lane]; kmax = warp_max[lane];
+    kmin = lane < NWARP ? warp_min[lane] : 0xffffffffu; kmax = lane < NWARP ? warp_max[lane] : 0u;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
@@ -697,7 +708,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
         if (j0 + g * GS < n_c) atomicAdd(&hist[(gmax[g] - kmin) >> sh1], 1u);    // the group has at least one key
       }
       __syncthreads();
-      find_bin(hist, (uint32_t)k_ch, warp_tot, sh, tid);
+      find_bin<TH>(hist, (uint32_t)k_ch, warp_tot, sh, tid);
       P = kmin + (sh[0] << sh1);
       __syncthreads();
     }
@@ -734,26 +745,26 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
     for (;;) {
       const int bits = 32 - __clz(span);                               // span < 2^bits
       const int shb = bits > 11 ? bits - 11 : 0;
-      for (int i = tid; i < kTopkBins; i += kTopkThreads) hist[i] = 0;
+      for (int i = tid; i < kTopkBins; i += TH) hist[i] = 0;
       __syncthreads();
-      for (int e = tid; e < n_list; e += kTopkThreads) {
+      for (int e = tid; e < n_list; e += TH) {
         const uint32_t rel = list_key[e] - lo;                         // keys below lo wrap to huge values
         if (rel <= span) atomicAdd(&hist[rel >> shb], 1u);
       }
       __syncthreads();
-      find_bin(hist, need, warp_tot, sh, tid);
+      find_bin<TH>(hist, need, warp_tot, sh, tid);
       const uint32_t bsel = sh[0], in_bin = sh[2];
       need = sh[1];
       lo += bsel << shb;
       span = min(span - (bsel << shb), (shb ? (1u << shb) : 1u) - 1u);
       __syncthreads();
       if (shb == 0) { thr = lo; need_eq = need; break; }
-      if (in_bin <= (uint32_t)kTopkCand) {
+      if (in_bin <= (uint32_t)kCand) {
         // few keys are left in the window: collect them and rank them against one another
         uint32_t* cand = hist;
         if (tid == 0) sh[3] = 0;
         __syncthreads();
-        for (int e = tid; e < n_list; e += kTopkThreads) {
+        for (int e = tid; e < n_list; e += TH) {
           const uint32_t kk = list_key[e];
           if (kk - lo <= span) cand[atomicAdd(&sh[3], 1u)] = kk;
         }
@@ -786,7 +797,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
       }
     }
     // ---- membership: keys above the threshold, and (separately) keys equal to it
-    for (int e = tid; e < n_list; e += kTopkThreads) {
+    for (int e = tid; e < n_list; e += TH) {
       const uint32_t kk = list_key[e];
       const uint32_t j = list_idx[e];
       if (kk > thr) atomicOr(&take_w[j >> 5], 1u << (j & 31u));
@@ -794,7 +805,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
     }
   } else {
     __syncthreads();                                                   // the bitmaps are zeroed
-    for (int w = tid; w < NW; w += kTopkThreads) {
+    for (int w = tid; w < NW; w += TH) {
       const int first = w * 32;
       take_w[w] = first + 32 <= n_c ? 0xffffffffu : (first < n_c ? ((1u << (n_c - first)) - 1u) : 0u);
     }
@@ -803,7 +814,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
   if (n_out > 0) {
     __syncthreads();
     const int32_t* outl = outliers + (size_t)prob * (size_t)n_out;     // [G][batch][H_kv][n_out], like sel_idx
-    for (int o = tid; o < n_out; o += kTopkThreads) {
+    for (int o = tid; o < n_out; o += TH) {
       const int jo = outl[o];
       if (jo >= 0 && jo < n_c) atomicOr(&take_w[jo >> 5], 1u << (jo & 31));
     }
@@ -820,21 +831,21 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
     if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-      const uint32_t t = warp_tot[lane];
+      const uint32_t t = lane < NWARP ? warp_tot[lane] : 0u;
       uint32_t ti = t;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const uint32_t v = __shfl_up_sync(0xffffffffu, ti, o);
         if (lane >= o) ti += v;
       }
-      warp_tot[lane] = ti - t;
+      if (lane < NWARP) warp_tot[lane] = ti - t;
       if (lane == 31) sh[3] = ti;
     }
     __syncthreads();
     return inc - mine + warp_tot[warp];
   };
   // keys equal to the threshold: the need_eq with the lowest chunk index are taken (thread w owns word w)
-  static_assert(NW <= kTopkThreads, "one bitmap word per thread");
+  static_assert(NW <= TH, "one bitmap word per thread");
   uint32_t fw = tid < NW ? take_w[tid] : 0u;
   {
     const uint32_t ew = tid < NW ? eq_w[tid] : 0u;
@@ -856,12 +867,12 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
   }
   __syncthreads();
   if (c == 8) {
-    for (uint32_t w = (uint32_t)tid; w < taken * 8u; w += kTopkThreads) {
+    for (uint32_t w = (uint32_t)tid; w < taken * 8u; w += TH) {
       const int row = (int)list_key[w >> 3] * 8 + (int)(w & 7u);
       if (row < T) out[w] = row;
     }
   } else {
-    for (uint32_t w = (uint32_t)tid; w < taken * (uint32_t)c; w += kTopkThreads) {
+    for (uint32_t w = (uint32_t)tid; w < taken * (uint32_t)c; w += TH) {
       const uint32_t e = w / (uint32_t)c, t = w - e * (uint32_t)c;
       const int row = (int)list_key[e] * c + (int)t;
       if (row < T) out[w] = row;
@@ -870,7 +881,7 @@ topk_pivot_kernel(GroupDev dev, int l0, int k_ch, int k_cap, const int32_t* __re
   // whole chunks unless the ragged last chunk was taken (it is then the last one)
   int cnt = (int)taken * c;
   if (taken > 0 && list_key[taken - 1] == (uint32_t)(n_c - 1)) cnt -= (n_c * c - T);
-  for (int i = cnt + tid; i < k_cap; i += kTopkThreads) out[i] = -1;
+  for (int i = cnt + tid; i < k_cap; i += TH) out[i] = -1;
   if (tid == 0 && sel_cnt) sel_cnt[prob] = cnt;
 }
 
@@ -883,30 +894,34 @@ static cudaError_t launch_topk(const GroupDev& dev, int device, int problems, in
   if (dev.n_c > kTopkThreads * 32)
     return launch_pdl(topk_kernel<false>, dim3(problems), dim3(kTopkThreads), 0, s, dev, l0, k_ch, k_cap, outliers, n_out,
                       sign, sel_idx, sel_cnt);
-  // keys per thread: 16 up to 16384 chunks, 32 beyond; groups per thread: the fewest with at least k_ch groups in all
-  // (0 = no filter)
+  // keys per thread: 16 up to 16384 chunks, 32 beyond; threads: the fewest of 128, 256, 512, 1024 that cover the
+  // chunks (a short context needs fewer barriers' worth of warps, and several of its CTAs share an SM); groups per
+  // thread: the fewest with at least k_ch groups in all (0 = no filter)
   const int items = dev.n_c <= kTopkThreads * 16 ? 16 : 32;
-  const size_t smem = (size_t)kTopkThreads * items * (sizeof(uint32_t) + sizeof(uint16_t));
+  const int th = items == 32 ? 1024 : (dev.n_c <= 128 * 16 ? 128 : dev.n_c <= 256 * 16 ? 256 : dev.n_c <= 512 * 16 ? 512 : 1024);
+  const size_t smem = (size_t)th * items * (sizeof(uint32_t) + sizeof(uint16_t));
   cudaError_t e;
-#define XKV_PIVOT(GPT, ITEMS)                                                                                         \
+#define XKV_PIVOT(GPT, ITEMS, TH)                                                                                     \
   do {                                                                                                                \
-    e = ensure_dyn_smem<topk_pivot_kernel<GPT, ITEMS>>(smem, device);                                                 \
+    e = ensure_dyn_smem<topk_pivot_kernel<GPT, ITEMS, TH>>(smem, device);                                             \
     if (e == cudaSuccess)                                                                                             \
-      e = launch_pdl(topk_pivot_kernel<GPT, ITEMS>, dim3(problems), dim3(kTopkThreads), smem, s, dev, l0, k_ch, k_cap, \
+      e = launch_pdl(topk_pivot_kernel<GPT, ITEMS, TH>, dim3(problems), dim3(TH), smem, s, dev, l0, k_ch, k_cap,      \
                      outliers, n_out, sign, sel_idx, sel_cnt);                                                        \
   } while (0)
+#define XKV_PIVOT_G(ITEMS, TH)                                                                                        \
+  do {                                                                                                                \
+    if (groups(1) >= k_ch) XKV_PIVOT(1, ITEMS, TH);                                                                   \
+    else if (groups(2) >= k_ch) XKV_PIVOT(2, ITEMS, TH);                                                              \
+    else if (groups(4) >= k_ch) XKV_PIVOT(4, ITEMS, TH);                                                              \
+    else XKV_PIVOT(0, ITEMS, TH);                                                                                     \
+  } while (0)
   auto groups = [&](int gpt) { return (dev.n_c + items / gpt - 1) / (items / gpt); };
-  if (items == 16) {
-    if (groups(1) >= k_ch) XKV_PIVOT(1, 16);
-    else if (groups(2) >= k_ch) XKV_PIVOT(2, 16);
-    else if (groups(4) >= k_ch) XKV_PIVOT(4, 16);
-    else XKV_PIVOT(0, 16);
-  } else {
-    if (groups(1) >= k_ch) XKV_PIVOT(1, 32);
-    else if (groups(2) >= k_ch) XKV_PIVOT(2, 32);
-    else if (groups(4) >= k_ch) XKV_PIVOT(4, 32);
-    else XKV_PIVOT(0, 32);
-  }
+  if (items == 32) XKV_PIVOT_G(32, 1024);
+  else if (th == 128) XKV_PIVOT_G(16, 128);
+  else if (th == 256) XKV_PIVOT_G(16, 256);
+  else if (th == 512) XKV_PIVOT_G(16, 512);
+  else XKV_PIVOT_G(16, 1024);
+#undef XKV_PIVOT_G
 #undef XKV_PIVOT
   return e;
 }
