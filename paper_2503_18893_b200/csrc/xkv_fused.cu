@@ -1184,14 +1184,24 @@ merge_segments_multi_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat1
   }
   __syncthreads();
   // weighted sums of the segments' partial sums, one rank column per thread and pass, segments in ascending order
+  // (the loads of the first four segments of all heads are issued before the first of them is used: one trip to L2
+  // per column, not one per head and segment)
   for (int col = tid; col < r; col += kMergeMultiThreads) {
+    constexpr int kSegBatch = 4;
+    float v[HG][kSegBatch];
+#pragma unroll
+    for (int h = 0; h < HG; ++h)
+#pragma unroll
+      for (int sg = 0; sg < kSegBatch; ++sg)
+        v[h][sg] = (h < nh && sg < nseg) ? __ldcg(part0 + (size_t)h * (r + 2) + col + sg * stride) : 0.0f;
 #pragma unroll
     for (int h = 0; h < HG; ++h) {
       if (h < nh) {
         const float* part = part0 + (size_t)h * (r + 2) + col;
         float acc = 0.0f;
-#pragma unroll 4
-        for (int sg = 0; sg < nseg; ++sg) acc = fmaf(wgt_s[h][sg], __ldcg(part + sg * stride), acc);
+#pragma unroll
+        for (int sg = 0; sg < kSegBatch; ++sg) if (sg < nseg) acc = fmaf(wgt_s[h][sg], v[h][sg], acc);
+        for (int sg = kSegBatch; sg < nseg; ++sg) acc = fmaf(wgt_s[h][sg], __ldcg(part + sg * stride), acc);
         w_s[h * r4 + col] = acc;
       }
     }
@@ -1219,8 +1229,20 @@ merge_segments_multi_kernel(GroupDev dev, Sched sc, TailParts tail, __nv_bfloat1
     const int m = rg + i * RPP;
     if (m < r) add_row(pre[i], m);
   }
-#pragma unroll 2
-  for (int m = rg + kPre * RPP; m < r; m += RPP) add_row(*reinterpret_cast<const uint4*>(Bv + (size_t)m * ld), m);
+  // the remaining rows four at a time, their loads issued together
+  for (int m0 = rg + kPre * RPP; m0 < r; m0 += 4 * RPP) {
+    uint4 nx[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int m = m0 + u * RPP;
+      nx[u] = m < r ? *reinterpret_cast<const uint4*>(Bv + (size_t)m * ld) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int m = m0 + u * RPP;
+      if (m < r) add_row(nx[u], m);
+    }
+  }
   // a warp holds two row groups (lanes 0..15 and 16..31 with the same columns): fold them, then one partial per warp
 #pragma unroll
   for (int h = 0; h < HG; ++h)
